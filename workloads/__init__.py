@@ -1,0 +1,12 @@
+"""Seeded synthetic inputs and shape descriptions.
+
+This package serves both the CPU oracle and the CUDA library with the same
+bytes.  It contains no arithmetic of the zeroth-order method itself: only
+shape records, a storage-format helper (bf16 rounding) and calls to numpy's
+own random generators.
+"""
+from .spec import ModelSpec, CONFIGS, config  # noqa: F401
+from .synth import (  # noqa: F401
+    bf16_round, to_bf16_bits, from_bf16_bits, make_linear_problem,
+    make_decoder_problem, next_token_labels, label_word_labels,
+)
