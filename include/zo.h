@@ -1,0 +1,205 @@
+/*
+ * zo.h - C ABI of the parallelised zeroth-order (MobiZO-style) gradient estimator
+ *        for NVIDIA B200 (sm_100a).
+ *
+ * One zo_step is one iteration of the paper's Algorithm 1 ("MobiZO Algorithm"):
+ * the q queries (outer loop) and the +/- pair of each query (inner loop) are
+ * folded into ONE forward pass over n = 2q replicas of the shared batch through
+ * Multi-Perturbed LoRA layers ("MP-LoRA" paragraph: Y = X W + (X A) (.) B^(n), W and
+ * A shared, only B perturbed per path), followed by the 2q losses, the q
+ * projected gradients g_i = (l+ - l-) / (2 eps) and the ZO-SGD update
+ * B <- B - lr * (1/q) * sum_i g_i z_i of the trainable LoRA B tensors.
+ * The perturbations z_i are never stored: they are regenerated from the seed
+ * wherever they are needed (seed trick, Background section).
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless its name starts with `host_`.
+ *     The structs zo_config, zo_weights, zo_lora and the pointer arrays inside
+ *     them live in HOST memory and are read during the call only.
+ *   - The library allocates no device memory: the caller passes a workspace of
+ *     zo_workspace_bytes() bytes (256-byte aligned) that must stay valid until
+ *     zo_free(), and owns every tensor and the CUDA stream.
+ *   - Frozen tensors and activations are float32 (ZO_FP32) or bfloat16
+ *     (ZO_BF16); the trainable B tensors are always float32 ("master copy").
+ *   - Layouts are row-major.  Weights are stored [k_out, k_in] (the paper's W
+ *     transposed), LoRA A as [r, k_in] (the paper's A transposed), LoRA B as
+ *     [r, k_out].
+ *   - Replica order: n = 2*i + 0 carries +eps*z_i, n = 2*i + 1 carries -eps*z_i
+ *     (the B[0] / B[1] order of the paper's Algorithm 2).
+ *   - Perturbation stream: Philox4x32-10, key = (seed low, seed high), counter =
+ *     (e >> 2, tensor_id, i, 0), element e (row-major index in B) reads output
+ *     word e & 3; word x -> u = ((x >> 9) + 0.5) * 2^-23; words (0,1) and (2,3)
+ *     are Box-Muller pairs (sqrt(-2 ln u_a) * {cos, sin}(2 pi u_b)).
+ *     tensor_id = layer * n_targets + slot, slots numbering the adapted
+ *     sections (q, k, v) in ascending order; 0 for ZO_ARCH_LINEAR.
+ *   - Every entry point returns a zo_status; nothing throws, aborts or traps.
+ *     There is no CPU fallback: without a CUDA device the calls fail with
+ *     ZO_ERR_CUDA.
+ */
+#ifndef ZO_H_
+#define ZO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum zo_status {
+  ZO_OK = 0,
+  ZO_ERR_INVALID_ARG = 1, /* null pointer, size out of the configured range, bad enum      */
+  ZO_ERR_UNSUPPORTED = 2, /* shape the kernels do not cover (see zo_init)                   */
+  ZO_ERR_WORKSPACE = 3,   /* workspace too small or misaligned                              */
+  ZO_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (text in zo_last_error)    */
+  ZO_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out; the step's results are void */
+  ZO_ERR_NONFINITE = 6,   /* a loss came out NaN/Inf; B was left untouched                  */
+  ZO_ERR_STATE = 7        /* call order (e.g. zo_losses before any zo_step)                 */
+} zo_status;
+
+enum { ZO_ARCH_LINEAR = 0, ZO_ARCH_OPT = 1, ZO_ARCH_LLAMA = 2 };
+enum { ZO_FP32 = 0, ZO_BF16 = 1 };
+enum { ZO_LOSS_MSE = 0, ZO_LOSS_CE_FULL_VOCAB = 1, ZO_LOSS_CE_LABEL_WORDS = 2 };
+enum { ZO_TARGET_Q = 1, ZO_TARGET_K = 2, ZO_TARGET_V = 4 };
+/* flags: ZO_FLAG_SIMT_GEMM routes every bf16 GEMM (and attention) through the plain
+ * CUDA-core validation kernels instead of the tensor-core ones (cross-checking only). */
+enum { ZO_FLAG_SIMT_GEMM = 1 };
+
+typedef struct zo_ctx zo_ctx; /* opaque; owned by the library; released by zo_free */
+
+/* Model and limits; plain data, versioned by struct_size (= sizeof(zo_config)). */
+typedef struct zo_config {
+  uint32_t struct_size;
+  int32_t arch;      /* ZO_ARCH_*                                                   */
+  int32_t precision; /* ZO_FP32 | ZO_BF16                                           */
+  int32_t loss_kind; /* ZO_LOSS_*; ZO_ARCH_LINEAR requires ZO_LOSS_MSE              */
+  int32_t n_layers;  /* decoder blocks (1 for ZO_ARCH_LINEAR)                       */
+  int32_t d_model;   /* hidden size; ZO_ARCH_LINEAR: k_in                           */
+  int32_t d_out;     /* ZO_ARCH_LINEAR only: k_out                                  */
+  int32_t n_heads;
+  int32_t d_ffn;
+  int32_t vocab;
+  int32_t max_seq;      /* largest S; also rows of the learned position table (OPT) */
+  int32_t lora_rank;    /* r, 1..64                                                  */
+  float lora_scale;     /* multiplies the low-rank term; 1.0 = the layer equation as printed */
+  uint32_t lora_targets; /* ZO_TARGET_* mask over the fused q|k|v projection          */
+  int32_t label_words[2]; /* ZO_LOSS_CE_LABEL_WORDS: the two vocabulary rows          */
+  int32_t max_q;        /* largest q (n = 2q replicas), <= 32                        */
+  int32_t max_E;        /* largest number of sequences in the shared batch           */
+  int32_t max_labelled; /* largest number of labelled positions per sequence         */
+  float norm_eps;
+  float rope_theta;
+  int32_t tie_lm_head; /* 1: LM head = token embedding                               */
+  uint32_t flags;
+} zo_config;
+
+/* Frozen tensors of one decoder block (device pointers; element type per precision).
+ * OPT: LayerNorm gains+biases, biases on every linear, w_fc1 [d_ffn, d], ReLU.
+ * Llama: RMSNorm gains only (bias pointers NULL), w_fc1 [2*d_ffn, d] = gate rows
+ * followed by up rows, SiLU(gate)*up, rotate-half RoPE on q and k. */
+typedef struct zo_layer_weights {
+  const void* norm1_g; const void* norm1_b;
+  const void* w_qkv;   const void* b_qkv;  /* [3d, d], [3d]: q rows, k rows, v rows */
+  const void* w_o;     const void* b_o;    /* [d, d], [d]   */
+  const void* norm2_g; const void* norm2_b;
+  const void* w_fc1;   const void* b_fc1;
+  const void* w_fc2;   const void* b_fc2;  /* [d, d_ffn], [d] */
+} zo_layer_weights;
+
+typedef struct zo_weights {
+  const void* tok_emb;      /* [vocab, d]                                            */
+  const void* pos_emb;      /* [max_seq, d] learned positions (OPT) or NULL          */
+  const void* lm_head;      /* [vocab, d]; ignored when tie_lm_head                  */
+  const void* final_norm_g; const void* final_norm_b;
+  const zo_layer_weights* layers; /* HOST array [n_layers]                           */
+  const void* linear_w;     /* ZO_ARCH_LINEAR: W [d_out, d_model]                    */
+  const void* linear_bias;  /* ZO_ARCH_LINEAR: [d_out] or NULL                       */
+} zo_weights;
+
+/* LoRA tensors: HOST arrays of n_layers device pointers.
+ * A[l]: [n_targets * r, d_model] frozen (LoRA-FA), shared by all replicas.
+ * B[l]: float32 [n_targets, r, k_out]; the master copy, UPDATED IN PLACE by zo_step. */
+typedef struct zo_lora {
+  const void* const* A;
+  float* const* B;
+} zo_lora;
+
+/* Bytes of device workspace zo_init needs for this configuration (0 on a bad config). */
+size_t zo_workspace_bytes(const zo_config* cfg);
+
+/* Validates cfg, partitions the workspace, creates the context.  `cuda_stream` is a
+ * cudaStream_t (NULL = legacy default stream) on which every later call enqueues.
+ * Unsupported (ZO_ERR_UNSUPPORTED): d_model % n_heads != 0; head_dim not in
+ * {16, 32, 64, 128}; max_seq > 512; (r * k_out) % 4 != 0; ZO_BF16 with d_model, d_ffn or
+ * d_out not a multiple of 8 (16-byte row pitch needed by the tensor-memory-accelerator loads). */
+zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
+                  void* cuda_stream, zo_ctx** out);
+
+/* One step of Algorithm 1 on the shared batch.  Asynchronous: enqueues kernels on
+ * the context's stream and returns; never synchronises.
+ *   tokens : int32 [E, S] token ids        (ZO_ARCH_LINEAR: X [E*S, d_model], element type per precision)
+ *   labels : int32 [E, S]; <0 = position not in the loss.  ZO_LOSS_CE_FULL_VOCAB: the
+ *            vocabulary id to predict at that position.  ZO_LOSS_CE_LABEL_WORDS: class id
+ *            0/1 (index into label_words).  At most max_labelled entries >= 0 per sequence.
+ *            (ZO_ARCH_LINEAR: float32 targets [E*S, d_out].)
+ *   seed, q, eps, lr : Algorithm 1's s (s_i = (seed, i)), q, epsilon, eta.
+ *   eps == 0  : losses only; g = 0 and B untouched.
+ *   lr  == 0  : losses and g; B untouched (times the perturbed forward alone).
+ * Errors: ZO_ERR_INVALID_ARG for null pointers, q < 1, q > max_q, E < 1, E > max_E,
+ * S < 1, S > max_seq, eps < 0 or non-finite scalars.  Device-side problems
+ * (ZO_ERR_TIMEOUT, ZO_ERR_NONFINITE, too many labelled positions = ZO_ERR_INVALID_ARG)
+ * are reported by the next zo_losses. */
+zo_status zo_step(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
+                  const void* tokens, const void* labels, int32_t E, int32_t S,
+                  uint64_t seed, int32_t q, float eps, float lr);
+
+/* Same step with tokens and labels in HOST memory (pinned or pageable): they are
+ * copied to the device on the context's stream first.  The host buffers must stay
+ * untouched until the stream has passed the copy (e.g. until zo_losses returns). */
+zo_status zo_step_host(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
+                       const void* host_tokens, const void* host_labels, int32_t E, int32_t S,
+                       uint64_t seed, int32_t q, float eps, float lr);
+
+/* Synchronises the stream and copies out the last step's 2q losses (replica order) and,
+ * if host_g != NULL, its q projected gradients.  Returns the step's deferred status. */
+zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g);
+
+/* Diagnostics: per labelled-row losses of the last step, [2q][rows] with rows in
+ * (sequence, labelled slot) order, max_labelled slots per sequence (unused slots are 0);
+ * *host_n_rows receives rows per replica.  host_rows may be NULL to query the count.
+ * ZO_ARCH_LINEAR: one value per token row (mean over k_out).  Synchronises the stream. */
+zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows);
+
+/* Number of kernels the last zo_step enqueued. */
+int32_t zo_launch_count(const zo_ctx* ctx);
+
+void zo_free(zo_ctx* ctx);
+const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo_init failure */
+
+/* The perturbation stream itself (Algorithm 1: z_i from s_i), for bit-level checks:
+ * writes the first n raw 32-bit words (dev_u32, may be NULL) and normals (dev_z, may be
+ * NULL) of tensor `tensor_id`, query `query`.  Asynchronous on `cuda_stream`. */
+zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, uint32_t query,
+                          int64_t n, uint32_t* dev_u32, float* dev_z);
+
+/* The MP-LoRA linear on its own ("MP-LoRA" paragraph, layer equation):
+ *   Y[n] = X[n or shared] W^T + bias + scale * (X A^T) (B + k_n eps z_{n>>1}),  n < 2q.
+ * x_replicated = 0: X is [T, k_in], the base product is computed once and expanded to the
+ * 2q outputs (first perturbed layer of a model); 1: X is [2q*T, k_in] (every later layer).
+ * Y is [2q, T, k_out].  `precision` selects float32 or bfloat16 for X, W, bias, A and Y.
+ * `scratch` needs zo_mp_lora_scratch_bytes() bytes (256-byte aligned).  bfloat16 requires
+ * k_in % 8 == 0, k_out % 8 == 0 and, for replicated input, T % 128 == 0.
+ * Asynchronous on `cuda_stream`. */
+size_t zo_mp_lora_scratch_bytes(int32_t precision, int32_t T, int32_t k_in, int32_t k_out,
+                                int32_t r, int32_t q, int32_t x_replicated);
+zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X, const void* W,
+                            const void* bias, const void* A, const float* B, void* Y,
+                            int32_t T, int32_t k_in, int32_t k_out, int32_t r, float scale,
+                            uint64_t seed, uint32_t tensor_id, int32_t q, float eps,
+                            int32_t x_replicated, void* scratch, size_t scratch_bytes,
+                            uint32_t flags);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ZO_H_ */
