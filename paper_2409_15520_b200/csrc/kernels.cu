@@ -1,0 +1,697 @@
+// Bandwidth-bound and small kernels of the perturbed forward, the losses and the update.
+#include "common.cuh"
+#include "kernels.h"
+
+namespace zo {
+
+// =========================================================================================
+// Embedding (+ learned positions) on the SHARED token block only: the n replicas of the
+// batch are identical up to the first MP-LoRA layer ("n copies of the input batch"), so
+// this is computed once.  Pad rows (t >= T) are zero-filled.
+// =========================================================================================
+template <typename T>
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ tok_emb,
+                             const T* __restrict__ pos_emb, T* __restrict__ out, int Tn, int S,
+                             int d, int vocab, uint32_t* status) {
+  const int t = blockIdx.x;
+  T* o = out + (size_t)t * d;
+  if (t >= Tn) {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = from_f<T>(0.f);
+    return;
+  }
+  int id = tokens[t];
+  if (id < 0 || id >= vocab) {
+    if (threadIdx.x == 0) atomicOr(status, ST_BAD_TOKEN);
+    id = 0;
+  }
+  const T* e = tok_emb + (size_t)id * d;
+  const T* p = pos_emb ? pos_emb + (size_t)(t % S) * d : nullptr;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float v = to_f(e[c]);
+    if (p) v += to_f(p[c]);
+    o[c] = from_f<T>(v);
+  }
+}
+
+void launch_embed(cudaStream_t st, int bf, const int32_t* tokens, const void* tok_emb,
+                  const void* pos_emb, void* out, int T, int Tp, int S, int d, int vocab,
+                  uint32_t* status) {
+  if (bf)
+    embed_kernel<bf16><<<Tp, 128, 0, st>>>(tokens, (const bf16*)tok_emb, (const bf16*)pos_emb,
+                                           (bf16*)out, T, S, d, vocab, status);
+  else
+    embed_kernel<float><<<Tp, 128, 0, st>>>(tokens, (const float*)tok_emb, (const float*)pos_emb,
+                                            (float*)out, T, S, d, vocab, status);
+}
+
+// =========================================================================================
+// LayerNorm / RMSNorm, one block per row, fp32 statistics (two-pass variance).
+// =========================================================================================
+template <typename T>
+__global__ void norm_kernel(int kind, const T* __restrict__ x, T* __restrict__ out,
+                            const T* __restrict__ g, const T* __restrict__ b, int d, float eps,
+                            const int32_t* __restrict__ lab_idx, int EP, int Tp) {
+  __shared__ float red[32];
+  const int row = blockIdx.x;
+  long long src = row;
+  if (lab_idx) {
+    const int n = row / EP, j = row % EP;
+    const int li = lab_idx[j];
+    src = li < 0 ? -1 : (long long)n * Tp + li;
+  }
+  T* o = out + (size_t)row * d;
+  if (src < 0) {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) o[c] = from_f<T>(0.f);
+    return;
+  }
+  const T* xr = x + (size_t)src * d;
+  float s = 0.f;
+  if (kind == 0) {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) s += to_f(xr[c]);
+    const float mu = block_sum(s, red) / d;
+    float v = 0.f;
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+      const float t = to_f(xr[c]) - mu;
+      v += t * t;
+    }
+    const float rstd = rsqrtf(block_sum(v, red) / d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x)
+      o[c] = from_f<T>((to_f(xr[c]) - mu) * rstd * to_f(g[c]) + (b ? to_f(b[c]) : 0.f));
+  } else {
+    for (int c = threadIdx.x; c < d; c += blockDim.x) {
+      const float t = to_f(xr[c]);
+      s += t * t;
+    }
+    const float rstd = rsqrtf(block_sum(s, red) / d + eps);
+    for (int c = threadIdx.x; c < d; c += blockDim.x)
+      o[c] = from_f<T>(to_f(xr[c]) * rstd * to_f(g[c]));
+  }
+}
+
+void launch_norm(cudaStream_t st, int bf, int kind, const void* x, void* out, const void* g,
+                 const void* b, int rows, int d, float eps, const int32_t* lab_idx, int EP,
+                 int Tp) {
+  if (rows <= 0) return;
+  const int th = d >= 2048 ? 256 : 128;
+  if (bf)
+    norm_kernel<bf16><<<rows, th, 0, st>>>(kind, (const bf16*)x, (bf16*)out, (const bf16*)g,
+                                           (const bf16*)b, d, eps, lab_idx, EP, Tp);
+  else
+    norm_kernel<float><<<rows, th, 0, st>>>(kind, (const float*)x, (float*)out, (const float*)g,
+                                            (const float*)b, d, eps, lab_idx, EP, Tp);
+}
+
+// =========================================================================================
+// LoRA down-projection U = X A^T (A shared by all replicas, frozen): [rows,K] x [J,K]^T.
+// 32 rows per block, K streamed through shared memory in chunks of 32.
+// =========================================================================================
+constexpr int LD_MAXJ = 192;  // 3 targets x rank 64
+template <typename T>
+__global__ void __launch_bounds__(256)
+lora_down_kernel(const T* __restrict__ X, int ldx, const T* __restrict__ A,
+                 float* __restrict__ U, int rows, int K, int J) {
+  extern __shared__ float sm[];
+  float* Xs = sm;              // [32][33]
+  float* As = sm + 32 * 33;    // [J][33]
+  const int tid = threadIdx.x, r = tid >> 3, cg = tid & 7;
+  const int row0 = blockIdx.x * 32;
+  float acc[LD_MAXJ / 8];
+#pragma unroll
+  for (int i = 0; i < LD_MAXJ / 8; ++i) acc[i] = 0.f;
+  for (int k0 = 0; k0 < K; k0 += 32) {
+    for (int i = tid; i < 32 * 32; i += 256) {
+      const int rr = i >> 5, kk = i & 31;
+      const int gr = row0 + rr, gk = k0 + kk;
+      Xs[rr * 33 + kk] = (gr < rows && gk < K) ? to_f(X[(size_t)gr * ldx + gk]) : 0.f;
+    }
+    for (int i = tid; i < J * 32; i += 256) {
+      const int jj = i >> 5, kk = i & 31;
+      const int gk = k0 + kk;
+      As[jj * 33 + kk] = gk < K ? to_f(A[(size_t)jj * K + gk]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int kk = 0; kk < 32; ++kk) {
+      const float xv = Xs[r * 33 + kk];
+#pragma unroll
+      for (int i = 0; i < LD_MAXJ / 8; ++i) {
+        const int j = cg + 8 * i;
+        if (j < J) acc[i] = fmaf(xv, As[j * 33 + kk], acc[i]);
+      }
+    }
+    __syncthreads();
+  }
+  const int gr = row0 + r;
+  if (gr < rows) {
+#pragma unroll
+    for (int i = 0; i < LD_MAXJ / 8; ++i) {
+      const int j = cg + 8 * i;
+      if (j < J) U[(size_t)gr * J + j] = acc[i];
+    }
+  }
+}
+
+void launch_lora_down(cudaStream_t st, int bf, const void* X, int ldx, const void* A, float* U,
+                      int rows, int K, int J) {
+  if (rows <= 0 || J <= 0) return;
+  const size_t smem = (size_t)(32 * 33 + J * 33) * sizeof(float);
+  const int grid = (rows + 31) / 32;
+  if (bf)
+    lora_down_kernel<bf16><<<grid, 256, smem, st>>>((const bf16*)X, ldx, (const bf16*)A, U, rows, K, J);
+  else
+    lora_down_kernel<float><<<grid, 256, smem, st>>>((const float*)X, ldx, (const float*)A, U, rows, K, J);
+}
+
+// =========================================================================================
+// MP-LoRA low-rank term applied to a base product:
+//   out[n, t, c] = base[(shared ? t : n*Tp + t), c]
+//                + s * sum_k U[.., slot*r + k] * (B[slot,k,c'] + k_n eps z)
+// z regenerated from the seed in registers (never stored).  Each thread owns 4 consecutive
+// columns (= one Philox block per rank index) and LA_ROWS rows of one replica.
+// =========================================================================================
+constexpr int LA_ROWS = 8;
+template <typename T>
+__global__ void lora_apply_kernel(const T* __restrict__ base, int ldb, int base_shared,
+                                  T* __restrict__ out, int ldo, int Tn, LoraDesc L, int nsec) {
+  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (c0 >= nsec * L.width) return;
+  const int n = blockIdx.z;
+  const int t0 = blockIdx.y * LA_ROWS;
+  const int sec = c0 / L.width, cc = c0 - sec * L.width;
+  const int slot = L.slot_of_sec[sec];
+  const int Tp = L.rows_per_replica;
+  float acc[LA_ROWS][4];
+#pragma unroll
+  for (int i = 0; i < LA_ROWS; ++i) {
+    const int t = t0 + i;
+    if (t < Tn) {
+      const T* bp = base + (size_t)(base_shared ? t : n * Tp + t) * ldb + c0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = to_f(bp[j]);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+    }
+  }
+  if (slot >= 0) {
+    const float sgn = (n & 1) ? -L.eps : L.eps;
+    const uint32_t query = (uint32_t)(n >> 1);
+    const float* Bs = L.B + (size_t)slot * L.r * L.width;
+    float la[LA_ROWS][4];
+#pragma unroll
+    for (int i = 0; i < LA_ROWS; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) la[i][j] = 0.f;
+    for (int k = 0; k < L.r; ++k) {
+      const size_t e = (size_t)k * L.width + cc;
+      const float4 bm = *reinterpret_cast<const float4*>(Bs + e);
+      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (L.eps != 0.f) z = z_block(L.seed, L.tensor_base + slot, query, (uint32_t)(e >> 2));
+      const float b0 = fmaf(sgn, z.x, bm.x), b1 = fmaf(sgn, z.y, bm.y);
+      const float b2 = fmaf(sgn, z.z, bm.z), b3 = fmaf(sgn, z.w, bm.w);
+#pragma unroll
+      for (int i = 0; i < LA_ROWS; ++i) {
+        const int t = t0 + i;
+        if (t < Tn) {
+          const float u = L.U[(size_t)(base_shared ? t : n * Tp + t) * L.ldu + slot * L.r + k];
+          la[i][0] = fmaf(u, b0, la[i][0]);
+          la[i][1] = fmaf(u, b1, la[i][1]);
+          la[i][2] = fmaf(u, b2, la[i][2]);
+          la[i][3] = fmaf(u, b3, la[i][3]);
+        }
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < LA_ROWS; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(L.scale, la[i][j], acc[i][j]);
+  }
+#pragma unroll
+  for (int i = 0; i < LA_ROWS; ++i) {
+    const int t = t0 + i;
+    if (t < Tn) {
+      T* op = out + (size_t)(n * Tp + t) * ldo + c0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) op[j] = from_f<T>(acc[i][j]);
+    }
+  }
+}
+
+void launch_lora_apply(cudaStream_t st, int bf, const void* base, int ldb, int base_shared,
+                       void* out, int ldo, int n, int T, const LoraDesc& L, int nsec) {
+  if (n <= 0 || T <= 0) return;
+  const int cols4 = nsec * L.width / 4;
+  dim3 grid((cols4 + 127) / 128, (T + LA_ROWS - 1) / LA_ROWS, n);
+  if (bf)
+    lora_apply_kernel<bf16><<<grid, 128, 0, st>>>((const bf16*)base, ldb, base_shared, (bf16*)out, ldo, T, L, nsec);
+  else
+    lora_apply_kernel<float><<<grid, 128, 0, st>>>((const float*)base, ldb, base_shared, (float*)out, ldo, T, L, nsec);
+}
+
+// =========================================================================================
+// RoPE (rotate-half pairing (j, j + dh/2)); table of cos/sin built once in fp64.
+// =========================================================================================
+__global__ void rope_table_kernel(float* tab, int max_seq, int half, double theta) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= max_seq * half) return;
+  const int s = i / half, j = i % half;
+  const double inv = pow(theta, -2.0 * (double)j / (double)(2 * half));
+  const double a = (double)s * inv;
+  tab[2 * i] = (float)cos(a);
+  tab[2 * i + 1] = (float)sin(a);
+}
+void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float theta) {
+  const int n = max_seq * (dh / 2);
+  rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, max_seq, dh / 2, (double)theta);
+}
+
+template <typename T>
+__global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S, int d, int H,
+                            const float* __restrict__ tab) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int half = d / H / 2;
+  const int j = (int)(i % half);
+  long long rest = i / half;
+  const int h = (int)(rest % H);
+  rest /= H;
+  const int which = (int)(rest % 2);  // 0 = q, 1 = k
+  const long long row = rest / 2;
+  const int s = (int)((row % Tp) % S);
+  const float c = tab[2 * (s * half + j)], sn = tab[2 * (s * half + j) + 1];
+  T* p = qkv + (size_t)row * 3 * d + (size_t)which * d + h * 2 * half + j;
+  const float x1 = to_f(p[0]), x2 = to_f(p[half]);
+  p[0] = from_f<T>(x1 * c - x2 * sn);
+  p[half] = from_f<T>(x2 * c + x1 * sn);
+}
+void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, int d, int H,
+                 const float* tab) {
+  const long long total = (long long)rows * 2 * H * (d / H / 2);
+  if (total <= 0) return;
+  const unsigned grid = (unsigned)((total + 255) / 256);
+  if (bf)
+    rope_kernel<bf16><<<grid, 256, 0, st>>>((bf16*)qkv, total, Tp, S, d, H, tab);
+  else
+    rope_kernel<float><<<grid, 256, 0, st>>>((float*)qkv, total, Tp, S, d, H, tab);
+}
+
+// =========================================================================================
+// Causal attention on CUDA cores (validation / fp32 path): one block per
+// (64-query tile, head, sequence).  Scores of the tile against all visible keys are kept in
+// shared memory (S <= 512), then a row softmax, then P V.
+// =========================================================================================
+template <typename T, int DH>
+__global__ void __launch_bounds__(256)
+attention_simt_kernel(const T* __restrict__ qkv, T* __restrict__ ctx, int E, int S, int Tp,
+                      int d) {
+  extern __shared__ float sm[];
+  constexpr int LDQ = DH + 1;
+  const int Sp = (S + 63) & ~63;
+  float* Qs = sm;                 // [64][LDQ]
+  float* Ks = Qs + 64 * LDQ;      // [64][LDQ]  (K tile, later V tile)
+  float* Ss = Ks + 64 * LDQ;      // [64][Sp + 1]
+  const int LDS = Sp + 1;
+  const int q0 = blockIdx.x * 64, h = blockIdx.y, sq = blockIdx.z;
+  const int n = sq / E, b = sq % E;
+  const size_t row_base = (size_t)n * Tp + (size_t)b * S;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const float scale = rsqrtf((float)DH);
+  const int ld = 3 * d;
+
+  for (int i = tid; i < 64 * DH; i += 256) {
+    const int r = i / DH, c = i % DH;
+    const int s = q0 + r;
+    Qs[r * LDQ + c] = s < S ? to_f(qkv[(row_base + s) * ld + h * DH + c]) : 0.f;
+  }
+  const int kend = min(S, q0 + 64);  // keys visible to this query tile
+  for (int k0 = 0; k0 < kend; k0 += 64) {
+    __syncthreads();
+    for (int i = tid; i < 64 * DH; i += 256) {
+      const int r = i / DH, c = i % DH;
+      const int s = k0 + r;
+      Ks[r * LDQ + c] = s < S ? to_f(qkv[(row_base + s) * ld + d + h * DH + c]) : 0.f;
+    }
+    __syncthreads();
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+#pragma unroll 8
+    for (int c = 0; c < DH; ++c) {
+      float qv[4], kv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) qv[i] = Qs[(ty * 4 + i) * LDQ + c];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) kv[j] = Ks[(tx * 4 + j) * LDQ + c];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(qv[i], kv[j], acc[i][j]);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) Ss[(ty * 4 + i) * LDS + k0 + tx * 4 + j] = acc[i][j] * scale;
+  }
+  __syncthreads();
+  // row softmax over keys 0..q (causal), one warp per row
+  const int warp = tid >> 5, lane = tid & 31;
+  for (int r = warp; r < 64; r += 8) {
+    const int s = q0 + r;
+    const int lim = min(s, S - 1) + 1;  // number of visible keys
+    float* p = Ss + r * LDS;
+    float m = -INFINITY;
+    for (int k = lane; k < lim; k += 32) m = fmaxf(m, p[k]);
+    m = warp_max(m);
+    float sum = 0.f;
+    for (int k = lane; k < lim; k += 32) {
+      const float e = expf(p[k] - m);
+      p[k] = e;
+      sum += e;
+    }
+    sum = warp_sum(sum);
+    const float inv = 1.f / sum;
+    for (int k = lane; k < Sp; k += 32) p[k] = k < lim ? p[k] * inv : 0.f;
+  }
+  // O = P V
+  constexpr int NC = DH / 16;
+  float o[4][NC];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < NC; ++j) o[i][j] = 0.f;
+  for (int k0 = 0; k0 < kend; k0 += 64) {
+    __syncthreads();
+    for (int i = tid; i < 64 * DH; i += 256) {
+      const int r = i / DH, c = i % DH;
+      const int s = k0 + r;
+      Ks[r * LDQ + c] = s < S ? to_f(qkv[(row_base + s) * ld + 2 * d + h * DH + c]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll 4
+    for (int k = 0; k < 64; ++k) {
+      float pv[4], vv[NC];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) pv[i] = Ss[(ty * 4 + i) * LDS + k0 + k];
+#pragma unroll
+      for (int j = 0; j < NC; ++j) vv[j] = Ks[k * LDQ + tx + 16 * j];
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < NC; ++j) o[i][j] = fmaf(pv[i], vv[j], o[i][j]);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int s = q0 + ty * 4 + i;
+    if (s < S) {
+#pragma unroll
+      for (int j = 0; j < NC; ++j)
+        ctx[(row_base + s) * d + h * DH + tx + 16 * j] = from_f<T>(o[i][j]);
+    }
+  }
+}
+
+template <typename T, int DH>
+static void attention_simt_launch(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S,
+                                  int Tp, int d, int H) {
+  const int Sp = (S + 63) & ~63;
+  const size_t smem = (size_t)(2 * 64 * (DH + 1) + 64 * (Sp + 1)) * sizeof(float);
+  cudaFuncSetAttribute(attention_simt_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                       (int)smem);
+  dim3 grid((S + 63) / 64, H, n * E);
+  attention_simt_kernel<T, DH><<<grid, 256, smem, st>>>((const T*)qkv, (T*)ctx, E, S, Tp, d);
+}
+
+void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, int E,
+                           int S, int Tp, int d, int H) {
+  const int dh = d / H;
+#define ZO_ATT(DH)                                                             \
+  if (dh == DH) {                                                              \
+    if (bf) attention_simt_launch<bf16, DH>(st, qkv, ctx, n, E, S, Tp, d, H);  \
+    else attention_simt_launch<float, DH>(st, qkv, ctx, n, E, S, Tp, d, H);    \
+    return;                                                                    \
+  }
+  ZO_ATT(16) ZO_ATT(32) ZO_ATT(64) ZO_ATT(128)
+#undef ZO_ATT
+}
+
+// =========================================================================================
+// SwiGLU on an unfused [rows, 2*ffn] gate|up buffer.
+// =========================================================================================
+template <typename T>
+__global__ void swiglu_kernel(const T* __restrict__ gu, T* __restrict__ out, long long total,
+                              int ffn) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const long long row = i / ffn;
+  const int c = (int)(i % ffn);
+  const float g = to_f(gu[row * 2 * ffn + c]), u = to_f(gu[row * 2 * ffn + ffn + c]);
+  out[i] = from_f<T>(g / (1.f + expf(-g)) * u);
+}
+void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows, int ffn) {
+  const long long total = (long long)rows * ffn;
+  if (total <= 0) return;
+  const unsigned grid = (unsigned)((total + 255) / 256);
+  if (bf) swiglu_kernel<bf16><<<grid, 256, 0, st>>>((const bf16*)gu, (bf16*)out, total, ffn);
+  else swiglu_kernel<float><<<grid, 256, 0, st>>>((const float*)gu, (float*)out, total, ffn);
+}
+
+// =========================================================================================
+// Labelled positions of each sequence, in order: lab_idx[b*P + p] = b*S + s (or -1),
+// lab_val = the label there.  One thread per sequence (S is small).
+// =========================================================================================
+__global__ void label_scan_kernel(const int32_t* __restrict__ labels, int E, int S, int P,
+                                  int n_classes, int32_t* lab_idx, int32_t* lab_val,
+                                  int32_t* lab_cnt, uint32_t* status) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= E) return;
+  int cnt = 0;
+  for (int s = 0; s < S; ++s) {
+    const int v = labels[b * S + s];
+    if (v < 0) continue;
+    if (v >= n_classes || cnt >= P) {
+      atomicOr(status, ST_BAD_LABELS);
+      continue;
+    }
+    lab_idx[b * P + cnt] = b * S + s;
+    lab_val[b * P + cnt] = v;
+    ++cnt;
+  }
+  lab_cnt[b] = cnt;
+  for (; cnt < P; ++cnt) {
+    lab_idx[b * P + cnt] = -1;
+    lab_val[b * P + cnt] = -1;
+  }
+}
+void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
+                       int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status) {
+  label_scan_kernel<<<(E + 63) / 64, 64, 0, st>>>(labels, E, S, P, n_classes, lab_idx, lab_val,
+                                                  lab_cnt, status);
+}
+
+// =========================================================================================
+// Fused log-softmax / label pick over the whole vocabulary, one block per labelled row:
+// row_loss = logsumexp(logits) - logits[label].
+// =========================================================================================
+__global__ void ce_rows_kernel(const float* __restrict__ logits, int ldl, int V,
+                               const int32_t* __restrict__ lab_val, int EP,
+                               float* __restrict__ row_loss) {
+  __shared__ float red[32];
+  const int row = blockIdx.x;
+  const int lab = lab_val[row % EP];
+  if (lab < 0) {
+    if (threadIdx.x == 0) row_loss[row] = 0.f;
+    return;
+  }
+  const float* p = logits + (size_t)row * ldl;
+  float m = -INFINITY;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) m = fmaxf(m, p[c]);
+  m = block_max(m, red);
+  float s = 0.f;
+  for (int c = threadIdx.x; c < V; c += blockDim.x) s += expf(p[c] - m);
+  s = block_sum(s, red);
+  if (threadIdx.x == 0) row_loss[row] = (m - p[lab]) + logf(s);
+}
+void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
+                    int EP, int rows, float* row_loss) {
+  if (rows <= 0) return;
+  ce_rows_kernel<<<rows, 256, 0, st>>>(logits, ldl, V, lab_val, EP, row_loss);
+}
+
+// Two-way softmax over the two label-word logits at the labelled (final) position.
+template <typename T>
+__global__ void label_word_rows_kernel(const T* __restrict__ xh, const T* __restrict__ head,
+                                       int d, int w0, int w1, const int32_t* __restrict__ lab_val,
+                                       int EP, float* __restrict__ row_loss) {
+  __shared__ float red[32];
+  const int row = blockIdx.x;
+  const int cls = lab_val[row % EP];
+  if (cls < 0) {
+    if (threadIdx.x == 0) row_loss[row] = 0.f;
+    return;
+  }
+  const T* x = xh + (size_t)row * d;
+  const T* h0 = head + (size_t)w0 * d;
+  const T* h1 = head + (size_t)w1 * d;
+  float a = 0.f, b = 0.f;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    const float xv = to_f(x[c]);
+    a = fmaf(xv, to_f(h0[c]), a);
+    b = fmaf(xv, to_f(h1[c]), b);
+  }
+  a = block_sum(a, red);
+  b = block_sum(b, red);
+  if (threadIdx.x == 0) {
+    const float m = fmaxf(a, b);
+    const float lse = m + logf(expf(a - m) + expf(b - m));
+    row_loss[row] = lse - (cls == 0 ? a : b);
+  }
+}
+void launch_label_word_rows(cudaStream_t st, int bf, const void* xh, const void* head, int d,
+                            int w0, int w1, const int32_t* lab_val, int EP, int rows,
+                            float* row_loss) {
+  if (rows <= 0) return;
+  if (bf)
+    label_word_rows_kernel<bf16><<<rows, 128, 0, st>>>((const bf16*)xh, (const bf16*)head, d, w0, w1, lab_val, EP, row_loss);
+  else
+    label_word_rows_kernel<float><<<rows, 128, 0, st>>>((const float*)xh, (const float*)head, d, w0, w1, lab_val, EP, row_loss);
+}
+
+// Mean squared error of one output row against its target (ZO_ARCH_LINEAR).
+template <typename T>
+__global__ void mse_rows_kernel(const T* __restrict__ Y, const float* __restrict__ target, int Tn,
+                                int Tp, int k_out, float* __restrict__ row_loss) {
+  __shared__ float red[32];
+  const int t = blockIdx.x, n = blockIdx.y;
+  const T* y = Y + ((size_t)n * Tp + t) * k_out;
+  const float* g = target + (size_t)t * k_out;
+  float s = 0.f;
+  for (int c = threadIdx.x; c < k_out; c += blockDim.x) {
+    const float dlt = to_f(y[c]) - g[c];
+    s = fmaf(dlt, dlt, s);
+  }
+  s = block_sum(s, red);
+  if (threadIdx.x == 0) row_loss[(size_t)n * Tn + t] = s / (float)k_out;
+}
+void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target, int n, int T,
+                     int Tp, int k_out, float* row_loss) {
+  if (n <= 0 || T <= 0) return;
+  dim3 grid(T, n);
+  if (bf) mse_rows_kernel<bf16><<<grid, 128, 0, st>>>((const bf16*)Y, target, T, Tp, k_out, row_loss);
+  else mse_rows_kernel<float><<<grid, 128, 0, st>>>((const float*)Y, target, T, Tp, k_out, row_loss);
+}
+
+// =========================================================================================
+// Per-replica mean over its valid rows: fixed order, fp64 accumulation (Algorithm 1: the
+// loss of a path is the mean over the labelled positions of the batch).
+// =========================================================================================
+__global__ void replica_mean_kernel(const float* __restrict__ row_loss,
+                                    const int32_t* __restrict__ lab_val, int rows,
+                                    float* __restrict__ losses, uint32_t* status) {
+  __shared__ double sd[256];
+  __shared__ int sc[256];
+  const int n = blockIdx.x;
+  double s = 0.0;
+  int c = 0;
+  for (int i = threadIdx.x; i < rows; i += 256) {
+    if (!lab_val || lab_val[i] >= 0) {
+      s += (double)row_loss[(size_t)n * rows + i];
+      ++c;
+    }
+  }
+  sd[threadIdx.x] = s;
+  sc[threadIdx.x] = c;
+  __syncthreads();
+  for (int o = 128; o > 0; o >>= 1) {
+    if (threadIdx.x < o) {
+      sd[threadIdx.x] += sd[threadIdx.x + o];
+      sc[threadIdx.x] += sc[threadIdx.x + o];
+    }
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    const float l = sc[0] > 0 ? (float)(sd[0] / (double)sc[0]) : 0.f;
+    losses[n] = l;
+    if (!isfinite(l)) atomicOr(status, ST_NONFINITE);
+  }
+}
+void launch_replica_mean(cudaStream_t st, const float* row_loss, const int32_t* lab_val, int n,
+                         int rows_per_replica, float* losses, uint32_t* status) {
+  if (n <= 0) return;
+  replica_mean_kernel<<<n, 256, 0, st>>>(row_loss, lab_val, rows_per_replica, losses, status);
+}
+
+// =========================================================================================
+// Projected gradients and ZO-SGD update (Algorithm 1): g_i = (l+ - l-) / (2 eps);
+// B <- B - eta (1/q) sum_i g_i z_i with z_i regenerated from the same seed.  Only the
+// master copy is written.  Each thread owns one Philox block (4 consecutive elements).
+// =========================================================================================
+constexpr int UPD_MAXQ = 64;
+__global__ void zo_update_kernel(UpdateDesc D, const float* __restrict__ losses,
+                                 float* __restrict__ g_out, int q, float eps, float lr,
+                                 uint64_t seed, const uint32_t* __restrict__ status, int write_g) {
+  __shared__ float gs[UPD_MAXQ];
+  const bool live = eps > 0.f;
+  for (int i = threadIdx.x; i < q; i += blockDim.x)
+    gs[i] = live ? (losses[2 * i] - losses[2 * i + 1]) / (2.f * eps) : 0.f;
+  __syncthreads();
+  if (write_g && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
+    for (int i = threadIdx.x; i < q; i += blockDim.x) g_out[i] = gs[i];
+  if (!live || lr == 0.f || *status != 0u) return;
+  const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long e = blk * 4;
+  if (e >= D.elems_per_slot) return;
+  const int slot = blockIdx.y, li = blockIdx.z;
+  float* Bp = D.B[li] + (size_t)slot * D.elems_per_slot + e;
+  const uint32_t tensor = D.tensor_base[li] + slot;
+  float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+  for (int i = 0; i < q; ++i) {
+    const float4 z = z_block(seed, tensor, (uint32_t)i, (uint32_t)blk);
+    const float gi = gs[i];
+    a0 = fmaf(gi, z.x, a0);
+    a1 = fmaf(gi, z.y, a1);
+    a2 = fmaf(gi, z.z, a2);
+    a3 = fmaf(gi, z.w, a3);
+  }
+  const float sc = lr / (float)q;
+  const long long left = D.elems_per_slot - e;
+  if (left >= 4) {
+    float4 b = *reinterpret_cast<float4*>(Bp);
+    b.x -= sc * a0; b.y -= sc * a1; b.z -= sc * a2; b.w -= sc * a3;
+    *reinterpret_cast<float4*>(Bp) = b;
+  } else {
+    const float a[4] = {a0, a1, a2, a3};
+    for (int j = 0; j < left; ++j) Bp[j] -= sc * a[j];
+  }
+}
+void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const float* losses, float* g, int q,
+                      float eps, float lr, uint64_t seed, const uint32_t* status, int write_g) {
+  const long long blks = (D.elems_per_slot + 3) / 4;
+  dim3 grid((unsigned)((blks + 127) / 128), D.n_slots, D.count);
+  zo_update_kernel<<<grid, 128, 0, st>>>(D, losses, g, q, eps, lr, seed, status, write_g);
+}
+
+__global__ void perturbation_kernel(uint64_t seed, uint32_t tensor, uint32_t query, long long n,
+                                    uint32_t* u32, float* z) {
+  const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long e = blk * 4;
+  if (e >= n) return;
+  const uint4 w = z_words(seed, tensor, query, (uint32_t)blk);
+  const float4 zn = z_normals(w);
+  const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+  const float zz[4] = {zn.x, zn.y, zn.z, zn.w};
+  for (int j = 0; j < 4 && e + j < n; ++j) {
+    if (u32) u32[e + j] = ww[j];
+    if (z) z[e + j] = zz[j];
+  }
+}
+void launch_perturbation(cudaStream_t st, uint64_t seed, uint32_t tensor, uint32_t query,
+                         long long n, uint32_t* u32, float* z) {
+  if (n <= 0) return;
+  const long long blks = (n + 3) / 4;
+  perturbation_kernel<<<(unsigned)((blks + 127) / 128), 128, 0, st>>>(seed, tensor, query, n, u32, z);
+}
+
+}  // namespace zo

@@ -1,0 +1,91 @@
+// Host-side launchers of the CUDA kernels (internal to the library).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace zo {
+
+// Where the per-replica low-rank term s * U (B + k eps z) comes from.
+struct LoraDesc {
+  const float* U;        // [rows, ldu] fp32 down-projections X A^T, row-indexed like the X operand
+  int ldu;
+  const float* B;        // [n_slots, r, width] fp32 master copy of this layer
+  int r;
+  int width;             // k_out of one section
+  int slot_of_sec[3];    // output columns [j*width, (j+1)*width) -> slot, or -1 (not adapted)
+  float scale, eps;
+  uint64_t seed;
+  uint32_t tensor_base;  // tensor_id of slot 0
+  int rows_per_replica;  // rows of one replica in the (padded) activation layout
+};
+
+enum { ACT_NONE = 0, ACT_RELU = 1 };
+
+struct GemmDesc {
+  const void* A; int lda;       // [M, K] activations
+  const void* W;                // [N, K] weights (K contiguous)
+  int M, N, K;
+  void* out; int ldo;           // [M, N]  (swiglu: [M, N/2])
+  int out_f32;                  // 1: float output regardless of the operand type
+  const void* bias;             // [N] or null
+  const void* res; int ldr;     // residual rows (row % res_mod when res_mod > 0) or null
+  int res_mod;
+  int act;
+  int swiglu;                   // 1: W = [gate rows | up rows] (N = 2 * d_ffn), out = silu(g)*u
+  const LoraDesc* lora;         // null: plain GEMM
+};
+
+// --- elementwise / reduction kernels (bf = 1: bfloat16 tensors, 0: float) -------------------
+void launch_embed(cudaStream_t st, int bf, const int32_t* tokens, const void* tok_emb,
+                  const void* pos_emb, void* out, int T, int Tp, int S, int d, int vocab,
+                  uint32_t* status);
+// Row norm. kind 0 = LayerNorm (gain, bias), 1 = RMSNorm (gain).  When lab_idx != null the
+// source row of output row (n, j) with j < EP is n*Tp + lab_idx[j] (negative: zero row).
+void launch_norm(cudaStream_t st, int bf, int kind, const void* x, void* out, const void* g,
+                 const void* b, int rows, int d, float eps, const int32_t* lab_idx, int EP,
+                 int Tp);
+void launch_lora_down(cudaStream_t st, int bf, const void* X, int ldx, const void* A, float* U,
+                      int rows, int K, int J);
+void launch_lora_apply(cudaStream_t st, int bf, const void* base, int ldb, int base_shared,
+                       void* out, int ldo, int n, int T, const LoraDesc& L, int nsec);
+void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float theta);
+void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, int d, int H,
+                 const float* tab);
+void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, int E,
+                           int S, int Tp, int d, int H);
+void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows, int ffn);
+void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
+                       int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status);
+void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
+                    int EP, int rows, float* row_loss);
+void launch_label_word_rows(cudaStream_t st, int bf, const void* xh, const void* head, int d,
+                            int w0, int w1, const int32_t* lab_val, int EP, int rows,
+                            float* row_loss);
+void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target, int n, int T,
+                     int Tp, int k_out, float* row_loss);
+// losses[n] = mean of the valid rows of replica n (fixed order, fp64 accumulation).
+void launch_replica_mean(cudaStream_t st, const float* row_loss, const int32_t* lab_val, int n,
+                         int rows_per_replica, float* losses, uint32_t* status);
+
+struct UpdateDesc {
+  enum { MAX_T = 96 };
+  float* B[MAX_T];       // tensors updated by this launch (one per layer)
+  uint32_t tensor_base[MAX_T];
+  int count;
+  int n_slots;
+  long long elems_per_slot;  // r * width
+};
+// g_i = (l_{2i} - l_{2i+1}) / (2 eps); B <- B - (lr/q) sum_i g_i z_i  (skipped if *status != 0
+// or lr == 0).  With write_g, block 0 also stores g[0..q).
+void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const float* losses, float* g, int q,
+                      float eps, float lr, uint64_t seed, const uint32_t* status, int write_g);
+void launch_perturbation(cudaStream_t st, uint64_t seed, uint32_t tensor, uint32_t query,
+                         long long n, uint32_t* u32, float* z);
+
+// --- GEMMs ---------------------------------------------------------------------------------
+void launch_gemm_simt(cudaStream_t st, int bf, const GemmDesc& G);
+// bf16 tensor-core GEMM (tcgen05 + TMEM + TMA).  Returns a CUDA error code (0 = ok).
+int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_sms);
+int gemm_tc_init();  // resolves the driver entry point for tensor-map encoding; 0 = ok
+
+}  // namespace zo
