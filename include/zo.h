@@ -42,6 +42,12 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#if defined(__GNUC__)
+#define ZO_API __attribute__((visibility("default")))
+#else
+#define ZO_API
+#endif
+
 #ifdef __cplusplus
 extern "C" {
 #endif
@@ -125,14 +131,14 @@ typedef struct zo_lora {
 } zo_lora;
 
 /* Bytes of device workspace zo_init needs for this configuration (0 on a bad config). */
-size_t zo_workspace_bytes(const zo_config* cfg);
+ZO_API size_t zo_workspace_bytes(const zo_config* cfg);
 
 /* Validates cfg, partitions the workspace, creates the context.  `cuda_stream` is a
  * cudaStream_t (NULL = legacy default stream) on which every later call enqueues.
  * Unsupported (ZO_ERR_UNSUPPORTED): d_model % n_heads != 0; head_dim not in
  * {16, 32, 64, 128}; max_seq > 512; (r * k_out) % 4 != 0; ZO_BF16 with d_model, d_ffn or
  * d_out not a multiple of 8 (16-byte row pitch needed by the tensor-memory-accelerator loads). */
-zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
+ZO_API zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
                   void* cuda_stream, zo_ctx** out);
 
 /* One step of Algorithm 1 on the shared batch.  Asynchronous: enqueues kernels on
@@ -149,37 +155,37 @@ zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
  * S < 1, S > max_seq, eps < 0 or non-finite scalars.  Device-side problems
  * (ZO_ERR_TIMEOUT, ZO_ERR_NONFINITE, too many labelled positions = ZO_ERR_INVALID_ARG)
  * are reported by the next zo_losses. */
-zo_status zo_step(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
+ZO_API zo_status zo_step(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
                   const void* tokens, const void* labels, int32_t E, int32_t S,
                   uint64_t seed, int32_t q, float eps, float lr);
 
 /* Same step with tokens and labels in HOST memory (pinned or pageable): they are
  * copied to the device on the context's stream first.  The host buffers must stay
  * untouched until the stream has passed the copy (e.g. until zo_losses returns). */
-zo_status zo_step_host(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
+ZO_API zo_status zo_step_host(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
                        const void* host_tokens, const void* host_labels, int32_t E, int32_t S,
                        uint64_t seed, int32_t q, float eps, float lr);
 
 /* Synchronises the stream and copies out the last step's 2q losses (replica order) and,
  * if host_g != NULL, its q projected gradients.  Returns the step's deferred status. */
-zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g);
+ZO_API zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g);
 
 /* Diagnostics: per labelled-row losses of the last step, [2q][rows] with rows in
  * (sequence, labelled slot) order, max_labelled slots per sequence (unused slots are 0);
  * *host_n_rows receives rows per replica.  host_rows may be NULL to query the count.
  * ZO_ARCH_LINEAR: one value per token row (mean over k_out).  Synchronises the stream. */
-zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows);
+ZO_API zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows);
 
 /* Number of kernels the last zo_step enqueued. */
-int32_t zo_launch_count(const zo_ctx* ctx);
+ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 
-void zo_free(zo_ctx* ctx);
-const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo_init failure */
+ZO_API void zo_free(zo_ctx* ctx);
+ZO_API const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo_init failure */
 
 /* The perturbation stream itself (Algorithm 1: z_i from s_i), for bit-level checks:
  * writes the first n raw 32-bit words (dev_u32, may be NULL) and normals (dev_z, may be
  * NULL) of tensor `tensor_id`, query `query`.  Asynchronous on `cuda_stream`. */
-zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, uint32_t query,
+ZO_API zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, uint32_t query,
                           int64_t n, uint32_t* dev_u32, float* dev_z);
 
 /* The MP-LoRA linear on its own ("MP-LoRA" paragraph, layer equation):
@@ -190,9 +196,9 @@ zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, 
  * `scratch` needs zo_mp_lora_scratch_bytes() bytes (256-byte aligned).  bfloat16 requires
  * k_in % 8 == 0, k_out % 8 == 0 and, for replicated input, T % 128 == 0.
  * Asynchronous on `cuda_stream`. */
-size_t zo_mp_lora_scratch_bytes(int32_t precision, int32_t T, int32_t k_in, int32_t k_out,
+ZO_API size_t zo_mp_lora_scratch_bytes(int32_t precision, int32_t T, int32_t k_in, int32_t k_out,
                                 int32_t r, int32_t q, int32_t x_replicated);
-zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X, const void* W,
+ZO_API zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X, const void* W,
                             const void* bias, const void* A, const float* B, void* Y,
                             int32_t T, int32_t k_in, int32_t k_out, int32_t r, float scale,
                             uint64_t seed, uint32_t tensor_id, int32_t q, float eps,

@@ -1,0 +1,264 @@
+"""ctypes binding of include/zo.h: structure mirrors and argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libzo_b200.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(
+        f"{_LIB_PATH} is missing: build it with `python -m paper_2409_15520_b200.build` "
+        "(there is no CPU or PyTorch fallback)")
+LIB = C.CDLL(_LIB_PATH)
+
+STATUS_NAMES = ["ZO_OK", "ZO_ERR_INVALID_ARG", "ZO_ERR_UNSUPPORTED", "ZO_ERR_WORKSPACE",
+                "ZO_ERR_CUDA", "ZO_ERR_TIMEOUT", "ZO_ERR_NONFINITE", "ZO_ERR_STATE"]
+ZO_FP32, ZO_BF16 = 0, 1
+ZO_FLAG_SIMT_GEMM = 1
+
+
+class ZoError(RuntimeError):
+    def __init__(self, status, msg=""):
+        self.status = int(status)
+        name = STATUS_NAMES[self.status] if 0 <= self.status < len(STATUS_NAMES) else str(status)
+        super().__init__(f"{name}: {msg}")
+
+
+class ZoConfig(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("arch", C.c_int32), ("precision", C.c_int32),
+                ("loss_kind", C.c_int32), ("n_layers", C.c_int32), ("d_model", C.c_int32),
+                ("d_out", C.c_int32), ("n_heads", C.c_int32), ("d_ffn", C.c_int32),
+                ("vocab", C.c_int32), ("max_seq", C.c_int32), ("lora_rank", C.c_int32),
+                ("lora_scale", C.c_float), ("lora_targets", C.c_uint32),
+                ("label_words", C.c_int32 * 2), ("max_q", C.c_int32), ("max_E", C.c_int32),
+                ("max_labelled", C.c_int32), ("norm_eps", C.c_float), ("rope_theta", C.c_float),
+                ("tie_lm_head", C.c_int32), ("flags", C.c_uint32)]
+
+
+_LAYER_FIELDS = ["norm1_g", "norm1_b", "w_qkv", "b_qkv", "w_o", "b_o", "norm2_g", "norm2_b",
+                 "w_fc1", "b_fc1", "w_fc2", "b_fc2"]
+
+
+class ZoLayerWeights(C.Structure):
+    _fields_ = [(f, C.c_void_p) for f in _LAYER_FIELDS]
+
+
+class ZoWeights(C.Structure):
+    _fields_ = [("tok_emb", C.c_void_p), ("pos_emb", C.c_void_p), ("lm_head", C.c_void_p),
+                ("final_norm_g", C.c_void_p), ("final_norm_b", C.c_void_p),
+                ("layers", C.POINTER(ZoLayerWeights)), ("linear_w", C.c_void_p),
+                ("linear_bias", C.c_void_p)]
+
+
+class ZoLora(C.Structure):
+    _fields_ = [("A", C.POINTER(C.c_void_p)), ("B", C.POINTER(C.c_void_p))]
+
+
+def _sig(name, res, args):
+    f = getattr(LIB, name)
+    f.restype, f.argtypes = res, args
+    return f
+
+
+zo_workspace_bytes = _sig("zo_workspace_bytes", C.c_size_t, [C.POINTER(ZoConfig)])
+zo_init = _sig("zo_init", C.c_int, [C.POINTER(ZoConfig), C.c_void_p, C.c_size_t, C.c_void_p,
+                                    C.POINTER(C.c_void_p)])
+_STEP_ARGS = [C.c_void_p, C.POINTER(ZoWeights), C.POINTER(ZoLora), C.c_void_p, C.c_void_p,
+              C.c_int32, C.c_int32, C.c_uint64, C.c_int32, C.c_float, C.c_float]
+zo_step = _sig("zo_step", C.c_int, _STEP_ARGS)
+zo_step_host = _sig("zo_step_host", C.c_int, _STEP_ARGS)
+zo_losses = _sig("zo_losses", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p])
+zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)])
+zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
+zo_free = _sig("zo_free", None, [C.c_void_p])
+zo_last_error = _sig("zo_last_error", C.c_char_p, [C.c_void_p])
+zo_perturbation = _sig("zo_perturbation", C.c_int, [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
+                                                    C.c_int64, C.c_void_p, C.c_void_p])
+zo_mp_lora_scratch_bytes = _sig("zo_mp_lora_scratch_bytes", C.c_size_t, [C.c_int32] * 7)
+zo_mp_lora_linear = _sig("zo_mp_lora_linear", C.c_int, [
+    C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+    C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_uint64, C.c_uint32, C.c_int32,
+    C.c_float, C.c_int32, C.c_void_p, C.c_size_t, C.c_uint32])
+
+
+def make_config(spec, *, max_q=None, max_E=None, max_seq=None, max_labelled=None, flags=0,
+                precision=None) -> ZoConfig:
+    """zo_config from a shape record with the attribute names of workloads.ModelSpec."""
+    c = ZoConfig()
+    c.struct_size = C.sizeof(ZoConfig)
+    c.arch, c.loss_kind = spec.arch, spec.loss_kind
+    c.precision = (ZO_BF16 if spec.bf16 else ZO_FP32) if precision is None else precision
+    c.n_layers, c.d_model, c.d_out = spec.n_layers, spec.d_model, spec.d_out
+    c.n_heads, c.d_ffn, c.vocab = spec.n_heads, spec.d_ffn, spec.vocab
+    c.max_seq = max_seq or max(spec.max_seq, spec.S)
+    c.lora_rank, c.lora_scale, c.lora_targets = spec.lora_rank, spec.lora_scale, spec.lora_targets
+    c.label_words[0], c.label_words[1] = spec.label_words
+    c.max_q, c.max_E = max_q or spec.q, max_E or spec.E
+    c.max_labelled = max_labelled or spec.n_labelled
+    c.norm_eps, c.rope_theta = spec.norm_eps, spec.rope_theta
+    c.tie_lm_head, c.flags = int(spec.tie_lm_head), flags
+    return c
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(None)
+
+
+class DeviceProblem:
+    """Device copies of a synthetic problem (dict of numpy arrays as produced by the
+    workload generators) plus the zo_weights / zo_lora structures pointing at them."""
+
+    def __init__(self, p: dict, bf16: bool, device="cuda"):
+        self.dtype = torch.bfloat16 if bf16 else torch.float32
+        self.device = device
+        self._keep = []
+        self.weights = ZoWeights()
+        self.lora = ZoLora()
+        if "W" in p:  # single linear
+            self.linear = True
+            self.W, self.bias, self.A = self._up(p["W"]), self._up(p.get("bias")), self._up(p["A"])
+            self.B = [torch.tensor(p["B"], dtype=torch.float32, device=device).contiguous()]
+            self.weights.linear_w, self.weights.linear_bias = _ptr(self.W), _ptr(self.bias)
+            self._A = [self.A]
+            self.tokens = self._up(p["X"])
+            self.labels = torch.tensor(p["target"], dtype=torch.float32, device=device).contiguous()
+            self.host_tokens = self.tokens.cpu().pin_memory()
+            self.host_labels = self.labels.cpu().pin_memory()
+        else:
+            self.linear = False
+            for k in ("tok_emb", "pos_emb", "lm_head", "final_norm_g", "final_norm_b"):
+                t = self._up(p.get(k))
+                setattr(self, k, t)
+                setattr(self.weights, k, _ptr(t))
+            n = len(p["layers"])
+            self._layers = (ZoLayerWeights * n)()
+            self._A, self.B = [], []
+            for l, L in enumerate(p["layers"]):
+                for f in _LAYER_FIELDS:
+                    setattr(self._layers[l], f, _ptr(self._up(L.get(f))))
+                self._A.append(self._up(L["A"]) if L["A"].size else None)
+                self.B.append(torch.tensor(L["B"], dtype=torch.float32, device=device).contiguous()
+                              if L["B"].size else None)
+            self.weights.layers = self._layers
+            self.tokens = torch.tensor(p["tokens"], dtype=torch.int32, device=device).contiguous()
+            self.labels = torch.tensor(p["labels"], dtype=torch.int32, device=device).contiguous()
+            self.host_tokens = torch.tensor(p["tokens"], dtype=torch.int32).pin_memory()
+            self.host_labels = torch.tensor(p["labels"], dtype=torch.int32).pin_memory()
+        n = len(self.B)
+        self._Aarr = (C.c_void_p * n)(*[(t.data_ptr() if t is not None else None) for t in self._A])
+        self._Barr = (C.c_void_p * n)(*[(t.data_ptr() if t is not None else None) for t in self.B])
+        self.lora.A = C.cast(self._Aarr, C.POINTER(C.c_void_p))
+        self.lora.B = C.cast(self._Barr, C.POINTER(C.c_void_p))
+
+    def _up(self, x):
+        if x is None:
+            return None
+        t = torch.tensor(np.asarray(x, np.float32), device=self.device).to(self.dtype).contiguous()
+        self._keep.append(t)
+        return t
+
+    def B_numpy(self):
+        return [b.detach().cpu().numpy().astype(np.float64) if b is not None else None
+                for b in self.B]
+
+
+class Estimator:
+    """zo_init / zo_step / zo_losses with a torch-allocated workspace on the current stream."""
+
+    def __init__(self, cfg: ZoConfig, device="cuda"):
+        self.cfg = cfg
+        nbytes = zo_workspace_bytes(C.byref(cfg))
+        if nbytes == 0:
+            h = C.c_void_p()
+            st = zo_init(C.byref(cfg), None, 0, None, C.byref(h))
+            raise ZoError(st, zo_last_error(None).decode())
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.stream = torch.cuda.current_stream()
+        self._h = C.c_void_p()
+        st = zo_init(C.byref(cfg), C.c_void_p(base), nbytes, C.c_void_p(self.stream.cuda_stream),
+                     C.byref(self._h))
+        if st:
+            raise ZoError(st, zo_last_error(None).decode())
+        self.q = 0
+
+    def _check(self, st):
+        if st:
+            raise ZoError(st, zo_last_error(self._h).decode())
+
+    def step(self, prob: DeviceProblem, E, S, seed, q, eps, lr, tokens=None, labels=None):
+        tok = prob.tokens if tokens is None else tokens
+        lab = prob.labels if labels is None else labels
+        self._check(zo_step(self._h, C.byref(prob.weights), C.byref(prob.lora), _ptr(tok), _ptr(lab),
+                            E, S, seed, q, eps, lr))
+        self.q = q
+
+    def step_host(self, prob: DeviceProblem, E, S, seed, q, eps, lr):
+        self._check(zo_step_host(self._h, C.byref(prob.weights), C.byref(prob.lora),
+                                 C.c_void_p(prob.host_tokens.data_ptr()),
+                                 C.c_void_p(prob.host_labels.data_ptr()), E, S, seed, q, eps, lr))
+        self.q = q
+
+    def losses(self):
+        l = np.zeros(2 * self.q, np.float32)
+        g = np.zeros(self.q, np.float32)
+        self._check(zo_losses(self._h, l.ctypes.data_as(C.c_void_p), g.ctypes.data_as(C.c_void_p)))
+        return l, g
+
+    def row_losses(self):
+        n = C.c_int32()
+        self._check(zo_row_losses(self._h, None, C.byref(n)))
+        out = np.zeros((2 * self.q, n.value), np.float32)
+        self._check(zo_row_losses(self._h, out.ctypes.data_as(C.c_void_p), C.byref(n)))
+        return out
+
+    def launch_count(self):
+        return int(zo_launch_count(self._h))
+
+    def close(self):
+        if self._h:
+            zo_free(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def perturbation(seed, tensor_id, query, n, device="cuda"):
+    """(raw 32-bit words, normals) of the perturbation stream, as numpy arrays."""
+    u = torch.empty(n, dtype=torch.int32, device=device)
+    z = torch.empty(n, dtype=torch.float32, device=device)
+    st = zo_perturbation(C.c_void_p(torch.cuda.current_stream().cuda_stream), seed, tensor_id, query,
+                         n, _ptr(u), _ptr(z))
+    if st:
+        raise ZoError(st)
+    torch.cuda.synchronize()
+    return u.cpu().numpy().view(np.uint32), z.cpu().numpy()
+
+
+def mp_lora_linear(X, W, bias, A, B, T, q, scale, seed, tensor_id, eps, x_replicated, flags=0):
+    """Y [2q, T, k_out] = MP-LoRA linear of torch device tensors (float32 or bfloat16)."""
+    bf = X.dtype == torch.bfloat16
+    k_out, k_in = W.shape
+    r = A.shape[0]
+    Y = torch.empty((2 * q, T, k_out), dtype=X.dtype, device=X.device)
+    nb = zo_mp_lora_scratch_bytes(int(bf), T, k_in, k_out, r, q, int(x_replicated))
+    scratch = torch.empty(nb + 256, dtype=torch.uint8, device=X.device)
+    base = (scratch.data_ptr() + 255) // 256 * 256
+    st = zo_mp_lora_linear(C.c_void_p(torch.cuda.current_stream().cuda_stream), int(bf), _ptr(X),
+                           _ptr(W), _ptr(bias), _ptr(A), _ptr(B), _ptr(Y), T, k_in, k_out, r, scale,
+                           seed, tensor_id, q, eps, int(x_replicated), C.c_void_p(base), nb, flags)
+    if st:
+        raise ZoError(st)
+    torch.cuda.synchronize()
+    status = int(scratch.view(torch.int32)[(base - scratch.data_ptr()) // 4].item())
+    if status:
+        raise ZoError(5, f"device status word {status}")
+    return Y

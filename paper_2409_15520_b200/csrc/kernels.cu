@@ -171,8 +171,8 @@ void launch_lora_down(cudaStream_t st, int bf, const void* X, int ldx, const voi
 // =========================================================================================
 constexpr int LA_ROWS = 8;
 template <typename T>
-__global__ void lora_apply_kernel(const T* __restrict__ base, int ldb, int base_shared,
-                                  T* __restrict__ out, int ldo, int Tn, LoraDesc L, int nsec) {
+__global__ void lora_apply_kernel(const T* base, int ldb, int base_shared,
+                                  T* out, int ldo, int Tn, LoraDesc L, int nsec) {
   const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (c0 >= nsec * L.width) return;
   const int n = blockIdx.z;

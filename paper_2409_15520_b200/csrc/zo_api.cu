@@ -1,0 +1,597 @@
+// C ABI of the library: argument checks, workspace partition and the per-step launch plan.
+#include <math.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "../../include/zo.h"
+#include "common.cuh"
+#include "kernels.h"
+
+using namespace zo;
+
+namespace {
+
+char g_init_error[256] = "";
+
+struct Plan {  // byte offsets into the workspace
+  size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
+      xh, logits, rowloss, losses, g, status, total;
+};
+
+inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline int n_targets(const zo_config& c) {
+  return ((c.lora_targets >> 0) & 1) + ((c.lora_targets >> 1) & 1) + ((c.lora_targets >> 2) & 1);
+}
+inline int row_pad(const zo_config& c) { return c.precision == ZO_BF16 ? 128 : 1; }
+
+// Returns ZO_OK or the reason the configuration cannot be run.
+zo_status check_config(const zo_config* c, char* err, size_t errn) {
+#define BAD(code, ...)                 \
+  do {                                 \
+    snprintf(err, errn, __VA_ARGS__);  \
+    return code;                       \
+  } while (0)
+  if (!c) BAD(ZO_ERR_INVALID_ARG, "config is NULL");
+  if (c->struct_size != sizeof(zo_config))
+    BAD(ZO_ERR_INVALID_ARG, "struct_size %u != %zu", c->struct_size, sizeof(zo_config));
+  if (c->arch < ZO_ARCH_LINEAR || c->arch > ZO_ARCH_LLAMA) BAD(ZO_ERR_INVALID_ARG, "bad arch");
+  if (c->precision != ZO_FP32 && c->precision != ZO_BF16) BAD(ZO_ERR_INVALID_ARG, "bad precision");
+  if (c->loss_kind < ZO_LOSS_MSE || c->loss_kind > ZO_LOSS_CE_LABEL_WORDS)
+    BAD(ZO_ERR_INVALID_ARG, "bad loss_kind");
+  if (c->lora_rank < 1 || c->lora_rank > 64) BAD(ZO_ERR_INVALID_ARG, "lora_rank must be 1..64");
+  if (c->max_q < 1 || c->max_q > 32) BAD(ZO_ERR_INVALID_ARG, "max_q must be 1..32");
+  if (c->max_E < 1 || c->max_seq < 1) BAD(ZO_ERR_INVALID_ARG, "max_E and max_seq must be >= 1");
+  if (c->d_model < 1) BAD(ZO_ERR_INVALID_ARG, "d_model must be >= 1");
+  if (!isfinite(c->lora_scale)) BAD(ZO_ERR_INVALID_ARG, "lora_scale not finite");
+  const bool bf = c->precision == ZO_BF16;
+  if (c->arch == ZO_ARCH_LINEAR) {
+    if (c->loss_kind != ZO_LOSS_MSE) BAD(ZO_ERR_INVALID_ARG, "ZO_ARCH_LINEAR requires ZO_LOSS_MSE");
+    if (c->d_out < 1) BAD(ZO_ERR_INVALID_ARG, "d_out must be >= 1");
+    if (c->d_out % 4) BAD(ZO_ERR_UNSUPPORTED, "d_out must be a multiple of 4");
+    if (bf && (c->d_model % 8 || c->d_out % 8))
+      BAD(ZO_ERR_UNSUPPORTED, "bf16 needs d_model and d_out to be multiples of 8");
+    return ZO_OK;
+  }
+  if (c->loss_kind == ZO_LOSS_MSE) BAD(ZO_ERR_INVALID_ARG, "decoders need a cross-entropy loss");
+  if (c->n_layers < 1 || c->n_heads < 1 || c->d_ffn < 1 || c->vocab < 2 || c->max_labelled < 1)
+    BAD(ZO_ERR_INVALID_ARG, "n_layers, n_heads, d_ffn, vocab, max_labelled must be positive");
+  if (c->lora_targets & ~7u) BAD(ZO_ERR_INVALID_ARG, "unknown lora_targets bits");
+  if (c->d_model % c->n_heads) BAD(ZO_ERR_UNSUPPORTED, "d_model %% n_heads != 0");
+  const int dh = c->d_model / c->n_heads;
+  if (dh != 16 && dh != 32 && dh != 64 && dh != 128)
+    BAD(ZO_ERR_UNSUPPORTED, "head_dim %d not in {16,32,64,128}", dh);
+  if (c->max_seq > 512) BAD(ZO_ERR_UNSUPPORTED, "max_seq > 512");
+  if (c->d_model % 4) BAD(ZO_ERR_UNSUPPORTED, "d_model must be a multiple of 4");
+  if (bf && (c->d_model % 8 || c->d_ffn % 8))
+    BAD(ZO_ERR_UNSUPPORTED, "bf16 needs d_model and d_ffn to be multiples of 8");
+  if (c->loss_kind == ZO_LOSS_CE_LABEL_WORDS)
+    for (int i = 0; i < 2; ++i)
+      if (c->label_words[i] < 0 || c->label_words[i] >= c->vocab)
+        BAD(ZO_ERR_INVALID_ARG, "label word out of the vocabulary");
+  if (!(c->norm_eps > 0.f)) BAD(ZO_ERR_INVALID_ARG, "norm_eps must be > 0");
+  if (c->arch == ZO_ARCH_LLAMA && !(c->rope_theta > 1.f)) BAD(ZO_ERR_INVALID_ARG, "rope_theta must be > 1");
+  return ZO_OK;
+#undef BAD
+}
+
+Plan make_plan(const zo_config& c) {
+  Plan p;
+  memset(&p, 0, sizeof(p));
+  const size_t es = c.precision == ZO_BF16 ? 2 : 4;
+  const size_t n = 2 * (size_t)c.max_q;
+  const size_t Tm = (size_t)c.max_E * c.max_seq;
+  const size_t Tp = up(Tm, row_pad(c));
+  const size_t Mp = n * Tp;
+  size_t off = 0;
+  auto take = [&](size_t bytes) {
+    const size_t o = off;
+    off += up(bytes, 256);
+    return o;
+  };
+  const bool unfused_mlp = c.precision == ZO_FP32 || (c.flags & ZO_FLAG_SIMT_GEMM);
+  if (c.arch == ZO_ARCH_LINEAR) {
+    p.U = take(Tp * c.lora_rank * 4);
+    p.qkv0 = take(Tp * c.d_out * es);                 // base product X W^T
+    p.qkv = take(Mp * c.d_out * es);                  // Y[n]
+    p.tok_stage = take(Tm * c.d_model * es);          // host-variant staging of X
+    p.lab_stage = take(Tm * c.d_out * 4);             // and of the targets
+    p.rowloss = take(n * Tm * 4);
+  } else {
+    const size_t d = c.d_model, f = c.d_ffn, J = (size_t)n_targets(c) * c.lora_rank;
+    const size_t P = c.max_labelled, Mh = n * c.max_E * P;
+    p.h0 = take(Tp * d * es);
+    p.x0 = take(Tp * d * es);
+    p.qkv0 = take(Tp * 3 * d * es);
+    p.h = take(Mp * d * es);
+    p.x = take(Mp * d * es);
+    p.qkv = take(Mp * 3 * d * es);
+    p.a = take(Mp * f * es);
+    if (c.arch == ZO_ARCH_LLAMA && unfused_mlp) p.gu = take(Mp * 2 * f * es);
+    p.U = take(Mp * (J ? J : 1) * 4);
+    if (c.arch == ZO_ARCH_LLAMA) p.rope = take((size_t)c.max_seq * (d / c.n_heads) * 4);
+    p.lab_idx = take(c.max_E * P * 4);
+    p.lab_val = take(c.max_E * P * 4);
+    p.lab_cnt = take(c.max_E * 4);
+    p.tok_stage = take(Tm * 4);
+    p.lab_stage = take(Tm * 4);
+    p.xh = take(Mh * d * es);
+    if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
+    p.rowloss = take(Mh * 4);
+  }
+  p.losses = take(n * 4);
+  p.g = take((size_t)c.max_q * 4);
+  p.status = take(256);
+  p.total = off;
+  return p;
+}
+
+}  // namespace
+
+struct zo_ctx {
+  zo_config cfg;
+  Plan plan;
+  uint8_t* ws;
+  cudaStream_t st;
+  int bf, n_sms, nt;
+  int slot_of_sec[3];
+  int launches;
+  int stepped, last_q, last_E, last_S;
+  char err[256];
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+namespace {
+
+zo_status fail(zo_ctx* c, zo_status s, const char* fmt, const char* a = "") {
+  snprintf(c->err, sizeof(c->err), fmt, a);
+  return s;
+}
+
+// GEMM dispatch: tensor-core kernel for bf16 unless the validation flag asks otherwise.
+zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const GemmDesc& G,
+                   uint32_t* status, int n_sms, int* launches, char* err, size_t errn) {
+  if (bf && !(flags & ZO_FLAG_SIMT_GEMM)) {
+    const int e = launch_gemm_tc(st, G, status, n_sms);
+    if (e) {
+      snprintf(err, errn, "tensor-core GEMM launch failed (code %d: %s)", e,
+               e < 10000 ? cudaGetErrorString((cudaError_t)e) : "tensor-map encode");
+      return ZO_ERR_CUDA;
+    }
+  } else {
+    launch_gemm_simt(st, bf, G);
+  }
+  ++*launches;
+  (void)c;
+  return ZO_OK;
+}
+
+// Can the MP-LoRA term ride in the tensor-core GEMM's epilogue?
+inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
+  return bf && !(flags & ZO_FLAG_SIMT_GEMM) && Tp % 128 == 0 && width % 32 == 0;
+}
+
+zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* X,
+                      const void* target, int T, uint64_t seed, int q, float eps, float lr) {
+  const zo_config& cf = c->cfg;
+  const int bf = c->bf, n = 2 * q, r = cf.lora_rank, ki = cf.d_model, ko = cf.d_out;
+  const int Tp = (int)up(T, row_pad(cf));
+  cudaStream_t st = c->st;
+  uint32_t* status = c->at<uint32_t>(c->plan.status);
+  float* U = c->at<float>(c->plan.U);
+  void* base = c->at<uint8_t>(c->plan.qkv0);
+  void* Y = c->at<uint8_t>(c->plan.qkv);
+  float* rowloss = c->at<float>(c->plan.rowloss);
+  float* losses = c->at<float>(c->plan.losses);
+
+  launch_lora_down(st, bf, X, ki, lora->A[0], U, T, ki, r); ++c->launches;
+  GemmDesc G{};
+  G.A = X; G.lda = ki; G.W = w->linear_w; G.M = T; G.N = ko; G.K = ki;
+  G.out = base; G.ldo = ko; G.bias = w->linear_bias;
+  zo_status s = run_gemm(c, st, bf, cf.flags, G, status, c->n_sms, &c->launches, c->err, sizeof(c->err));
+  if (s) return s;
+  LoraDesc L{};
+  L.U = U; L.ldu = r; L.B = lora->B[0]; L.r = r; L.width = ko;
+  L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
+  L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
+  launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1); ++c->launches;
+  launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss); ++c->launches;
+  launch_replica_mean(st, rowloss, nullptr, n, T, losses, status); ++c->launches;
+  UpdateDesc D{};
+  D.B[0] = lora->B[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
+  D.elems_per_slot = (long long)r * ko;
+  launch_zo_update(st, D, losses, c->at<float>(c->plan.g), q, eps, lr, seed, status, 1); ++c->launches;
+  return ZO_OK;
+}
+
+zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const int32_t* tokens,
+                       const int32_t* labels, int E, int S, uint64_t seed, int q, float eps,
+                       float lr) {
+  const zo_config& cf = c->cfg;
+  const int bf = c->bf, n = 2 * q, r = cf.lora_rank, d = cf.d_model, f = cf.d_ffn, H = cf.n_heads;
+  const int T = E * S, Tp = (int)up(T, row_pad(cf)), M = n * Tp;
+  const int nt = c->nt, J = nt * r;
+  const bool opt = cf.arch == ZO_ARCH_OPT;
+  const int nkind = opt ? 0 : 1;
+  const bool unfused_mlp = !bf || (cf.flags & ZO_FLAG_SIMT_GEMM);
+  cudaStream_t st = c->st;
+  uint32_t* status = c->at<uint32_t>(c->plan.status);
+  void *h0 = c->at<uint8_t>(c->plan.h0), *x0 = c->at<uint8_t>(c->plan.x0);
+  void *qkv0 = c->at<uint8_t>(c->plan.qkv0), *h = c->at<uint8_t>(c->plan.h);
+  void *x = c->at<uint8_t>(c->plan.x), *qkv = c->at<uint8_t>(c->plan.qkv);
+  void *a = c->at<uint8_t>(c->plan.a), *gu = c->at<uint8_t>(c->plan.gu);
+  float* U = c->at<float>(c->plan.U);
+  const float* rope = c->at<float>(c->plan.rope);
+  int32_t *lab_idx = c->at<int32_t>(c->plan.lab_idx), *lab_val = c->at<int32_t>(c->plan.lab_val);
+  int32_t* lab_cnt = c->at<int32_t>(c->plan.lab_cnt);
+  float *rowloss = c->at<float>(c->plan.rowloss), *losses = c->at<float>(c->plan.losses);
+  zo_status s;
+#define GEMM(G)                                                                                  \
+  do {                                                                                           \
+    s = run_gemm(c, st, bf, cf.flags, G, status, c->n_sms, &c->launches, c->err, sizeof(c->err)); \
+    if (s) return s;                                                                             \
+  } while (0)
+
+  // shared prefix: embedding on the T shared tokens, once for all 2q replicas
+  launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, S, d, cf.vocab, status);
+  ++c->launches;
+  const int P = cf.max_labelled, EP = E * P;
+  const int n_classes = cf.loss_kind == ZO_LOSS_CE_LABEL_WORDS ? 2 : cf.vocab;
+  launch_label_scan(st, labels, E, S, P, n_classes, lab_idx, lab_val, lab_cnt, status); ++c->launches;
+
+  for (int l = 0; l < cf.n_layers; ++l) {
+    const zo_layer_weights& W = w->layers[l];
+    const bool first = l == 0;
+    const int rows = first ? Tp : M;           // layer 0 still works on the shared block
+    void* hin = first ? h0 : h;
+    void* xn = first ? x0 : x;
+    launch_norm(st, bf, nkind, hin, xn, W.norm1_g, W.norm1_b, rows, d, cf.norm_eps, nullptr, 0, 0);
+    ++c->launches;
+    LoraDesc L{};
+    L.U = U; L.ldu = J; L.B = J ? lora->B[l] : nullptr; L.r = r; L.width = d;
+    for (int j = 0; j < 3; ++j) L.slot_of_sec[j] = c->slot_of_sec[j];
+    L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = (uint32_t)(l * nt);
+    L.rows_per_replica = Tp;
+    if (J) { launch_lora_down(st, bf, xn, d, lora->A[l], U, rows, d, J); ++c->launches; }
+    GemmDesc G{};
+    G.A = xn; G.lda = d; G.W = W.w_qkv; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
+    if (first) {
+      // first perturbed layer: one base product on the shared block, expanded to 2q outputs
+      G.out = qkv0; G.ldo = 3 * d;
+      GEMM(G);
+      launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3); ++c->launches;
+    } else if (J && fused_lora_ok(bf, cf.flags, Tp, d)) {
+      G.out = qkv; G.ldo = 3 * d; G.lora = &L;
+      GEMM(G);
+    } else {
+      G.out = qkv; G.ldo = 3 * d;
+      GEMM(G);
+      if (J) { launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3); ++c->launches; }
+    }
+    if (!opt) { launch_rope(st, bf, qkv, M, Tp, S, d, H, rope); ++c->launches; }
+    launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H); ++c->launches;
+    GemmDesc O{};
+    O.A = x; O.lda = d; O.W = W.w_o; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
+    O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0;
+    GEMM(O);
+    launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0);
+    ++c->launches;
+    GemmDesc F1{};
+    F1.A = x; F1.lda = d; F1.W = W.w_fc1; F1.M = M; F1.K = d; F1.bias = W.b_fc1;
+    if (opt) {
+      F1.N = f; F1.out = a; F1.ldo = f; F1.act = ACT_RELU;
+      GEMM(F1);
+    } else if (unfused_mlp) {
+      F1.N = 2 * f; F1.out = gu; F1.ldo = 2 * f;
+      GEMM(F1);
+      launch_swiglu(st, bf, gu, a, M, f); ++c->launches;
+    } else {
+      F1.N = 2 * f; F1.out = a; F1.ldo = f; F1.swiglu = 1;
+      GEMM(F1);
+    }
+    GemmDesc F2{};
+    F2.A = a; F2.lda = f; F2.W = W.w_fc2; F2.M = M; F2.N = d; F2.K = f; F2.out = h; F2.ldo = d;
+    F2.bias = W.b_fc2; F2.res = h; F2.ldr = d;
+    GEMM(F2);
+  }
+
+  // per-replica loss on the labelled rows only
+  const int Mh = n * EP;
+  void* xh = c->at<uint8_t>(c->plan.xh);
+  launch_norm(st, bf, nkind, h, xh, w->final_norm_g, w->final_norm_b, Mh, d, cf.norm_eps, lab_idx, EP, Tp);
+  ++c->launches;
+  const void* head = cf.tie_lm_head ? w->tok_emb : w->lm_head;
+  if (cf.loss_kind == ZO_LOSS_CE_FULL_VOCAB) {
+    float* logits = c->at<float>(c->plan.logits);
+    GemmDesc Hd{};
+    Hd.A = xh; Hd.lda = d; Hd.W = head; Hd.M = Mh; Hd.N = cf.vocab; Hd.K = d;
+    Hd.out = logits; Hd.ldo = cf.vocab; Hd.out_f32 = 1;
+    GEMM(Hd);
+    launch_ce_rows(st, logits, cf.vocab, cf.vocab, lab_val, EP, Mh, rowloss); ++c->launches;
+  } else {
+    launch_label_word_rows(st, bf, xh, head, d, cf.label_words[0], cf.label_words[1], lab_val, EP, Mh, rowloss);
+    ++c->launches;
+  }
+  launch_replica_mean(st, rowloss, lab_val, n, EP, losses, status); ++c->launches;
+
+  // projected gradients and ZO-SGD update of every B tensor
+  float* g = c->at<float>(c->plan.g);
+  if (J == 0) {
+    UpdateDesc D{};
+    D.count = 0; D.n_slots = 0; D.elems_per_slot = 0;
+    launch_zo_update(st, D, losses, g, q, eps, 0.f, seed, status, 1); ++c->launches;
+  }
+  for (int l0 = 0; l0 < cf.n_layers && J; l0 += UpdateDesc::MAX_T) {
+    UpdateDesc D{};
+    D.count = cf.n_layers - l0 < UpdateDesc::MAX_T ? cf.n_layers - l0 : UpdateDesc::MAX_T;
+    D.n_slots = nt;
+    D.elems_per_slot = (long long)r * d;
+    for (int i = 0; i < D.count; ++i) {
+      D.B[i] = lora->B[l0 + i];
+      D.tensor_base[i] = (uint32_t)((l0 + i) * nt);
+    }
+    launch_zo_update(st, D, losses, g, q, eps, lr, seed, status, l0 == 0); ++c->launches;
+  }
+#undef GEMM
+  return ZO_OK;
+}
+
+zo_status check_step_args(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* tokens,
+                          const void* labels, int E, int S, int q, float eps, float lr) {
+  if (!c) return ZO_ERR_INVALID_ARG;
+  const zo_config& cf = c->cfg;
+  if (!w || !lora || !tokens || !labels) return fail(c, ZO_ERR_INVALID_ARG, "null argument");
+  if (q < 1 || q > cf.max_q) return fail(c, ZO_ERR_INVALID_ARG, "q outside 1..max_q");
+  if (E < 1 || E > cf.max_E) return fail(c, ZO_ERR_INVALID_ARG, "E outside 1..max_E");
+  if (S < 1 || S > cf.max_seq) return fail(c, ZO_ERR_INVALID_ARG, "S outside 1..max_seq");
+  if (!(eps >= 0.f) || !isfinite(eps)) return fail(c, ZO_ERR_INVALID_ARG, "eps must be finite and >= 0");
+  if (!isfinite(lr)) return fail(c, ZO_ERR_INVALID_ARG, "lr must be finite");
+  if (!lora->A || !lora->B) return fail(c, ZO_ERR_INVALID_ARG, "lora pointer arrays are NULL");
+  if (cf.arch == ZO_ARCH_LINEAR) {
+    if (!w->linear_w || !lora->A[0] || !lora->B[0]) return fail(c, ZO_ERR_INVALID_ARG, "null linear tensor");
+    return ZO_OK;
+  }
+  if (!w->tok_emb || !w->final_norm_g || !w->layers) return fail(c, ZO_ERR_INVALID_ARG, "null model tensor");
+  if (cf.arch == ZO_ARCH_OPT && (!w->pos_emb || !w->final_norm_b))
+    return fail(c, ZO_ERR_INVALID_ARG, "OPT needs pos_emb and final_norm_b");
+  if (!cf.tie_lm_head && !w->lm_head) return fail(c, ZO_ERR_INVALID_ARG, "lm_head is NULL");
+  for (int l = 0; l < cf.n_layers; ++l) {
+    const zo_layer_weights& W = w->layers[l];
+    if (!W.norm1_g || !W.w_qkv || !W.w_o || !W.norm2_g || !W.w_fc1 || !W.w_fc2)
+      return fail(c, ZO_ERR_INVALID_ARG, "null layer tensor");
+    if (cf.arch == ZO_ARCH_OPT && (!W.norm1_b || !W.b_qkv || !W.b_o || !W.norm2_b || !W.b_fc1 || !W.b_fc2))
+      return fail(c, ZO_ERR_INVALID_ARG, "OPT layers need every bias");
+    if (c->nt && (!lora->A[l] || !lora->B[l])) return fail(c, ZO_ERR_INVALID_ARG, "null LoRA tensor");
+  }
+  return ZO_OK;
+}
+
+zo_status do_step(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* tokens,
+                  const void* labels, int E, int S, uint64_t seed, int q, float eps, float lr) {
+  c->launches = 0;
+  cudaError_t e = cudaMemsetAsync(c->at<uint32_t>(c->plan.status), 0, 4, c->st);
+  if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  zo_status s;
+  if (c->cfg.arch == ZO_ARCH_LINEAR)
+    s = step_linear(c, w, lora, tokens, labels, E * S, seed, q, eps, lr);
+  else
+    s = step_decoder(c, w, lora, (const int32_t*)tokens, (const int32_t*)labels, E, S, seed, q, eps, lr);
+  if (s) return s;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  c->stepped = 1; c->last_q = q; c->last_E = E; c->last_S = S;
+  return ZO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t zo_workspace_bytes(const zo_config* cfg) {
+  char err[256];
+  if (check_config(cfg, err, sizeof(err)) != ZO_OK) return 0;
+  return make_plan(*cfg).total;
+}
+
+zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes, void* cuda_stream,
+                  zo_ctx** out) {
+  if (!out) { snprintf(g_init_error, sizeof(g_init_error), "out is NULL"); return ZO_ERR_INVALID_ARG; }
+  *out = nullptr;
+  zo_status s = check_config(cfg, g_init_error, sizeof(g_init_error));
+  if (s) return s;
+  const Plan plan = make_plan(*cfg);
+  if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < plan.total) {
+    snprintf(g_init_error, sizeof(g_init_error), "workspace NULL, misaligned or smaller than %zu bytes", plan.total);
+    return ZO_ERR_WORKSPACE;
+  }
+  int dev = 0, sms = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  int major = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+  if (e != cudaSuccess) {
+    snprintf(g_init_error, sizeof(g_init_error), "no usable CUDA device: %s", cudaGetErrorString(e));
+    return ZO_ERR_CUDA;
+  }
+  if (major != 10) {
+    snprintf(g_init_error, sizeof(g_init_error), "device compute capability %d.x: built for sm_100a only", major);
+    return ZO_ERR_UNSUPPORTED;
+  }
+  if (cfg->precision == ZO_BF16 && !(cfg->flags & ZO_FLAG_SIMT_GEMM)) {
+    const int ge = gemm_tc_init();
+    if (ge) {
+      snprintf(g_init_error, sizeof(g_init_error), "tensor-core GEMM set-up failed (%d)", ge);
+      return ZO_ERR_CUDA;
+    }
+  }
+  zo_ctx* c = new (std::nothrow) zo_ctx;
+  if (!c) { snprintf(g_init_error, sizeof(g_init_error), "out of host memory"); return ZO_ERR_CUDA; }
+  memset(c, 0, sizeof(*c));
+  c->cfg = *cfg; c->plan = plan; c->ws = (uint8_t*)workspace; c->st = (cudaStream_t)cuda_stream;
+  c->bf = cfg->precision == ZO_BF16; c->n_sms = sms;
+  c->nt = cfg->arch == ZO_ARCH_LINEAR ? 1 : n_targets(*cfg);
+  int slot = 0;
+  for (int j = 0; j < 3; ++j) c->slot_of_sec[j] = ((cfg->lora_targets >> j) & 1) ? slot++ : -1;
+  // a defined (finite) start for pad rows, which kernels carry along but never mix into real rows
+  e = cudaMemsetAsync(workspace, 0, plan.total, c->st);
+  if (e == cudaSuccess && cfg->arch == ZO_ARCH_LLAMA) {
+    launch_rope_table(c->st, c->at<float>(plan.rope), cfg->max_seq, cfg->d_model / cfg->n_heads, cfg->rope_theta);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) {
+    snprintf(g_init_error, sizeof(g_init_error), "workspace set-up: %s", cudaGetErrorString(e));
+    delete c;
+    return ZO_ERR_CUDA;
+  }
+  *out = c;
+  return ZO_OK;
+}
+
+zo_status zo_step(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora, const void* tokens,
+                  const void* labels, int32_t E, int32_t S, uint64_t seed, int32_t q, float eps,
+                  float lr) {
+  zo_status s = check_step_args(ctx, weights, lora, tokens, labels, E, S, q, eps, lr);
+  if (s) return s;
+  return do_step(ctx, weights, lora, tokens, labels, E, S, seed, q, eps, lr);
+}
+
+zo_status zo_step_host(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
+                       const void* host_tokens, const void* host_labels, int32_t E, int32_t S,
+                       uint64_t seed, int32_t q, float eps, float lr) {
+  zo_status s = check_step_args(ctx, weights, lora, host_tokens, host_labels, E, S, q, eps, lr);
+  if (s) return s;
+  const zo_config& cf = ctx->cfg;
+  const size_t T = (size_t)E * S;
+  size_t tb, lb;
+  if (cf.arch == ZO_ARCH_LINEAR) {
+    tb = T * cf.d_model * (ctx->bf ? 2 : 4);
+    lb = T * cf.d_out * 4;
+  } else {
+    tb = lb = T * 4;
+  }
+  void* dt = ctx->at<uint8_t>(ctx->plan.tok_stage);
+  void* dl = ctx->at<uint8_t>(ctx->plan.lab_stage);
+  cudaError_t e = cudaMemcpyAsync(dt, host_tokens, tb, cudaMemcpyHostToDevice, ctx->st);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(dl, host_labels, lb, cudaMemcpyHostToDevice, ctx->st);
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "host-to-device copy: %s", cudaGetErrorString(e));
+  return do_step(ctx, weights, lora, dt, dl, E, S, seed, q, eps, lr);
+}
+
+zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (!host_losses) return fail(ctx, ZO_ERR_INVALID_ARG, "host_losses is NULL");
+  if (!ctx->stepped) return fail(ctx, ZO_ERR_STATE, "zo_losses before any zo_step");
+  uint32_t st = 0;
+  cudaError_t e = cudaMemcpyAsync(host_losses, ctx->at<float>(ctx->plan.losses), (size_t)2 * ctx->last_q * 4,
+                                  cudaMemcpyDeviceToHost, ctx->st);
+  if (e == cudaSuccess && host_g)
+    e = cudaMemcpyAsync(host_g, ctx->at<float>(ctx->plan.g), (size_t)ctx->last_q * 4, cudaMemcpyDeviceToHost, ctx->st);
+  if (e == cudaSuccess)
+    e = cudaMemcpyAsync(&st, ctx->at<uint32_t>(ctx->plan.status), 4, cudaMemcpyDeviceToHost, ctx->st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->st);
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "zo_losses: %s", cudaGetErrorString(e));
+  if (st & ST_TIMEOUT) return fail(ctx, ZO_ERR_TIMEOUT, "a bounded device-side wait ran out");
+  if (st & (ST_BAD_LABELS | ST_BAD_TOKEN))
+    return fail(ctx, ZO_ERR_INVALID_ARG, "token id or label out of range, or too many labelled positions");
+  if (st & ST_NONFINITE) return fail(ctx, ZO_ERR_NONFINITE, "a replica loss is not finite; B left untouched");
+  return ZO_OK;
+}
+
+zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (!host_n_rows) return fail(ctx, ZO_ERR_INVALID_ARG, "host_n_rows is NULL");
+  if (!ctx->stepped) return fail(ctx, ZO_ERR_STATE, "zo_row_losses before any zo_step");
+  const int rows = ctx->cfg.arch == ZO_ARCH_LINEAR ? ctx->last_E * ctx->last_S
+                                                   : ctx->last_E * ctx->cfg.max_labelled;
+  *host_n_rows = rows;
+  if (!host_rows) return ZO_OK;
+  cudaError_t e = cudaMemcpyAsync(host_rows, ctx->at<float>(ctx->plan.rowloss),
+                                  (size_t)2 * ctx->last_q * rows * 4, cudaMemcpyDeviceToHost, ctx->st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->st);
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "zo_row_losses: %s", cudaGetErrorString(e));
+  return ZO_OK;
+}
+
+int32_t zo_launch_count(const zo_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+void zo_free(zo_ctx* ctx) { delete ctx; }
+
+const char* zo_last_error(const zo_ctx* ctx) { return ctx ? ctx->err : g_init_error; }
+
+zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, uint32_t query,
+                          int64_t n, uint32_t* dev_u32, float* dev_z) {
+  if (n < 0 || (n > 0 && !dev_u32 && !dev_z)) return ZO_ERR_INVALID_ARG;
+  if (n > ((int64_t)1 << 34)) return ZO_ERR_INVALID_ARG;   // block index must fit 32 bits
+  launch_perturbation((cudaStream_t)cuda_stream, seed, tensor_id, query, n, dev_u32, dev_z);
+  return cudaGetLastError() == cudaSuccess ? ZO_OK : ZO_ERR_CUDA;
+}
+
+size_t zo_mp_lora_scratch_bytes(int32_t precision, int32_t T, int32_t k_in, int32_t k_out, int32_t r,
+                                int32_t q, int32_t x_replicated) {
+  if (T < 1 || k_in < 1 || k_out < 1 || r < 1 || q < 1) return 0;
+  const size_t es = precision == ZO_BF16 ? 2 : 4;
+  const size_t rows = x_replicated ? (size_t)2 * q * T : (size_t)T;
+  size_t b = 256 + up(rows * r * 4, 256);
+  if (!x_replicated) b += up((size_t)T * k_out * es, 256);
+  return b;
+}
+
+zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X, const void* W,
+                            const void* bias, const void* A, const float* B, void* Y, int32_t T,
+                            int32_t k_in, int32_t k_out, int32_t r, float scale, uint64_t seed,
+                            uint32_t tensor_id, int32_t q, float eps, int32_t x_replicated,
+                            void* scratch, size_t scratch_bytes, uint32_t flags) {
+  if (!X || !W || !A || !B || !Y || !scratch) return ZO_ERR_INVALID_ARG;
+  if (precision != ZO_FP32 && precision != ZO_BF16) return ZO_ERR_INVALID_ARG;
+  if (T < 1 || k_in < 1 || k_out < 1 || r < 1 || r > 64 || q < 1 || q > 32 || !(eps >= 0.f))
+    return ZO_ERR_INVALID_ARG;
+  const int bf = precision == ZO_BF16;
+  if (k_out % 4) return ZO_ERR_UNSUPPORTED;
+  if (bf && (k_in % 8 || k_out % 8)) return ZO_ERR_UNSUPPORTED;
+  if (bf && x_replicated && T % 128) return ZO_ERR_UNSUPPORTED;
+  const size_t need = zo_mp_lora_scratch_bytes(precision, T, k_in, k_out, r, q, x_replicated);
+  if (((uintptr_t)scratch & 255) || scratch_bytes < need) return ZO_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return ZO_ERR_CUDA;
+  const int n = 2 * q;
+  const size_t rows = x_replicated ? (size_t)n * T : (size_t)T;
+  uint8_t* sp = (uint8_t*)scratch;
+  uint32_t* status = (uint32_t*)sp;
+  float* U = (float*)(sp + 256);
+  void* base = sp + 256 + up(rows * r * 4, 256);
+  if (cudaMemsetAsync(status, 0, 4, st) != cudaSuccess) return ZO_ERR_CUDA;
+  launch_lora_down(st, bf, X, k_in, A, U, (int)rows, k_in, r);
+  LoraDesc L{};
+  L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
+  L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
+  L.scale = scale; L.eps = eps; L.seed = seed; L.tensor_base = tensor_id; L.rows_per_replica = T;
+  GemmDesc G{};
+  G.A = X; G.lda = k_in; G.W = W; G.M = (int)rows; G.N = k_out; G.K = k_in; G.bias = bias;
+  G.ldo = k_out;
+  int launches = 0;
+  char err[128];
+  zo_status s;
+  if (!x_replicated) {
+    G.out = base;
+    s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
+    if (s) return s;
+    launch_lora_apply(st, bf, base, k_out, 1, Y, k_out, n, T, L, 1);
+  } else if (fused_lora_ok(bf, flags, T, k_out)) {
+    G.out = Y; G.lora = &L;
+    s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
+    if (s) return s;
+  } else {
+    G.out = Y;
+    s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
+    if (s) return s;
+    launch_lora_apply(st, bf, Y, k_out, 0, Y, k_out, n, T, L, 1);
+  }
+  return cudaGetLastError() == cudaSuccess ? ZO_OK : ZO_ERR_CUDA;
+}
+
+}  // extern "C"

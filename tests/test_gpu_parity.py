@@ -1,0 +1,204 @@
+"""GPU parity: the CUDA library through its C ABI against the CPU oracle, element by element,
+on the same seeded inputs.  Tolerances: perturbation words bit-exact; fp32 mode losses 1e-4
+relative, projected gradients 1e-2 relative, updated B 1e-3 relative to the update; bf16 mode
+losses 2e-2 relative."""
+import numpy as np
+import pytest
+
+import oracle
+from oracle.philox import perturbation, perturbation_u32
+from workloads import ModelSpec, config
+from workloads.spec import (ARCH_LLAMA, ARCH_OPT, LOSS_CE_FULL, LOSS_CE_LABEL_WORDS, TARGET_K,
+                            TARGET_Q, TARGET_V)
+
+from gpu_util import make_problem, old_B, run_gpu, run_oracle, update_rel_err
+
+pytestmark = pytest.mark.gpu
+
+SIMT = 1  # ZO_FLAG_SIMT_GEMM
+
+
+def test_perturbation_words_bit_exact_and_normals_close():
+    import paper_2409_15520_b200 as zo
+    for seed, tensor, query, n in [(1, 0, 0, 4096), (0xDEADBEEFCAFEF00D, 63, 15, 1003), (7, 5, 2, 1)]:
+        u, z = zo.perturbation(seed, tensor, query, n)
+        assert np.array_equal(u, perturbation_u32(seed, tensor, query, n))
+        ref = perturbation(seed, tensor, query, (n,))
+        assert np.max(np.abs(z - ref)) <= 4e-7 * max(1.0, np.max(np.abs(ref)))
+
+
+def _check_fp32(spec, seed, b_std, q=None, eps=None, lr=None, tol_g=1e-2, **kw):
+    p, tok, lab = make_problem(spec, b_std=b_std)
+    ref = run_oracle(spec, p, tok, lab, seed, q, eps, lr)
+    got = run_gpu(spec, p, seed, q, eps, lr, **kw)
+    assert np.allclose(got["losses"], ref["losses"], rtol=1e-4, atol=0), (got["losses"], ref["losses"])
+    scale = np.max(np.abs(ref["g"]))
+    assert np.all(np.abs(got["g"] - ref["g"]) <= tol_g * scale), (got["g"], ref["g"])
+    assert update_rel_err(spec, p, got["B"], ref["B"]) < max(1e-3, tol_g / 10 * 1.5)
+    return got, ref
+
+
+def test_linear_fp32_config():
+    """The single MP-LoRA linear + MSE configuration, B = 0 and mid-training B."""
+    spec = config("linear_fp32")
+    got, ref = _check_fp32(spec, seed=1, b_std=0.0)
+    assert update_rel_err(spec, *[make_problem(spec)[0]], got["B"], ref["B"]) < 1e-3
+    _check_fp32(spec, seed=2, b_std=0.02)
+    _check_fp32(spec, seed=3, b_std=0.02, host=True)
+
+
+def test_linear_fp32_ragged_shapes_and_scale():
+    spec = config("linear_fp32", d_model=40, d_out=20, lora_rank=3, E=1, S=37, q=5, lora_scale=2.0)
+    _check_fp32(spec, seed=5, b_std=0.05)
+    spec = config("linear_fp32", d_model=8, d_out=4, lora_rank=1, E=1, S=1, q=1)
+    _check_fp32(spec, seed=6, b_std=0.05)
+
+
+TINY = dict(n_layers=2, d_model=64, n_heads=4, d_ffn=96, vocab=131, max_seq=24, lora_rank=4,
+            E=3, S=24, q=3, n_labelled=5, eps=1e-2, lr=1e-2)
+
+
+@pytest.mark.parametrize("arch,targets,loss", [
+    (ARCH_OPT, TARGET_Q | TARGET_V, LOSS_CE_FULL),
+    (ARCH_LLAMA, TARGET_Q | TARGET_V, LOSS_CE_FULL),
+    (ARCH_LLAMA, TARGET_Q | TARGET_K | TARGET_V, LOSS_CE_FULL),
+    (ARCH_OPT, TARGET_V, LOSS_CE_LABEL_WORDS),
+])
+def test_decoder_fp32(arch, targets, loss):
+    spec = ModelSpec(arch=arch, lora_targets=targets, loss_kind=loss, label_words=(7, 90),
+                     tie_lm_head=(arch == ARCH_OPT), bf16=False, lora_scale=2.0,
+                     **{**TINY, "n_labelled": 1 if loss == LOSS_CE_LABEL_WORDS else 5})
+    got, ref = _check_fp32(spec, seed=11, b_std=0.05)
+    # per labelled-row losses as well
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    z = [oracle.zo.draw_z(spec, p, 11, i) for i in range(spec.q)]
+    Bn = [np.stack([np.asarray(L["B"], np.float64) + (1 if n % 2 == 0 else -1) * spec.eps * z[n // 2][l]
+                    for n in range(2 * spec.q)]) for l, L in enumerate(p["layers"])]
+    _, rows = oracle.replica_losses(spec, p, Bn, tok, lab, return_rows=True)
+    assert np.allclose(got["rows"].reshape(rows.shape), rows, rtol=2e-4)
+
+
+def test_decoder_fp32_head_dims_and_ragged_sequence():
+    for dh, S, E in [(32, 7, 2), (64, 70, 1), (128, 65, 1)]:
+        spec = ModelSpec(arch=ARCH_LLAMA, bf16=False, **{**TINY, "d_model": 2 * dh, "n_heads": 2,
+                                                         "S": S, "E": E, "max_seq": S,
+                                                         "n_layers": 1, "q": 2})
+        _check_fp32(spec, seed=4, b_std=0.05)
+
+
+@pytest.mark.parametrize("flags", [SIMT, 0])
+@pytest.mark.parametrize("arch", [ARCH_OPT, ARCH_LLAMA])
+def test_decoder_bf16(arch, flags):
+    """bf16 storage; flags=SIMT runs the validation GEMM, 0 the tensor-core path.
+    T = 3*40 = 120 (< one 128-row tile) and d = 64 (< one 256-column tile)."""
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
+                     **{**TINY, "S": 40, "max_seq": 40})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 21)
+    got = run_gpu(spec, p, 21, flags=flags)
+    assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
+
+
+@pytest.mark.parametrize("arch", [ARCH_OPT, ARCH_LLAMA])
+def test_decoder_bf16_tensor_core_multi_tile(arch):
+    """Several row tiles per replica and several column tiles with ragged tails:
+    T = 2*160 = 320 -> padded 384 rows per replica, d = 320, ffn = 328, vocab = 1003."""
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
+                     **{**TINY, "d_model": 320, "n_heads": 5, "d_ffn": 328, "vocab": 1003,
+                        "S": 160, "E": 2, "max_seq": 160, "q": 2, "lora_rank": 8, "n_labelled": 7})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 31)
+    got = run_gpu(spec, p, 31)
+    simt = run_gpu(spec, p, 31, flags=SIMT)
+    assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
+    # the two bf16 GEMM implementations agree far more closely with each other
+    assert np.allclose(got["losses"], simt["losses"], rtol=2e-3, atol=0), (got["losses"], simt["losses"])
+    assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
+
+
+@pytest.mark.parametrize("x_replicated", [0, 1])
+@pytest.mark.parametrize("r", [8, 16, 64])
+def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
+    """The MP-LoRA layer equation on its own, both input modes, against the oracle's layer."""
+    import torch
+    import paper_2409_15520_b200 as zo
+    from workloads import bf16_round
+    rng = np.random.default_rng(r + x_replicated)
+    T, ki, ko, q, eps, scale, seed, tid = 256, 328, 544, 2, 1e-2, 2.0, 77, 3
+    n = 2 * q
+    X = bf16_round(rng.standard_normal((n if x_replicated else 1, T, ki)).astype(np.float32))
+    W = bf16_round(0.05 * rng.standard_normal((ko, ki)).astype(np.float32))
+    bias = bf16_round(0.05 * rng.standard_normal(ko).astype(np.float32))
+    A = bf16_round(0.05 * rng.standard_normal((r, ki)).astype(np.float32))
+    B = (0.05 * rng.standard_normal((r, ko))).astype(np.float32)
+    Bn = np.stack([B.astype(np.float64) + (1 if i % 2 == 0 else -1) * eps * perturbation(seed, tid, i // 2, (r, ko))
+                   for i in range(n)])
+    Xn = np.broadcast_to(X, (n, T, ki)).astype(np.float64)
+    ref = oracle.mp_lora_linear(Xn, W, bias, A, Bn, scale)
+    dev = lambda a: torch.tensor(a, device="cuda").to(torch.bfloat16).contiguous()
+    Bd = torch.tensor(B, device="cuda")
+    outs = {}
+    for flags in (0, SIMT):
+        Y = zo.mp_lora_linear(dev(X.reshape(-1, ki)), dev(W), dev(bias), dev(A), Bd, T, q, scale, seed,
+                              tid, eps, x_replicated, flags=flags)
+        outs[flags] = Y.float().cpu().numpy().astype(np.float64)
+        err = np.max(np.abs(outs[flags] - ref))
+        assert err < 2e-2 * np.max(np.abs(ref)), (flags, err, np.max(np.abs(ref)))
+    # the perturbation must be visible in the outputs: replicas 0 and 1 differ as the oracle's do
+    d_gpu, d_ref = outs[0][0] - outs[0][1], ref[0] - ref[1]
+    assert np.max(np.abs(d_ref)) > 0
+    assert np.max(np.abs(d_gpu - d_ref)) < 0.1 * np.max(np.abs(d_ref)) + 2 * 2.0 ** -8 * np.max(np.abs(ref))
+
+
+def test_degenerate_steps():
+    spec = ModelSpec(arch=ARCH_OPT, tie_lm_head=True, bf16=False, **TINY)
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    got = run_gpu(spec, p, 3, eps=0.0)                     # eps = 0: identical replicas, no update
+    assert np.all(got["losses"] == got["losses"][0]) and np.all(got["g"] == 0)
+    assert all(np.array_equal(a, b) for a, b in zip(got["B"], [b.astype(np.float32) for b in old_B(spec, p)]))
+    ref = run_oracle(spec, p, tok, lab, 3, eps=0.0)
+    assert np.allclose(got["losses"], ref["losses"], rtol=1e-4)
+    got = run_gpu(spec, p, 3, lr=0.0)                      # lr = 0: g but no update
+    assert np.any(got["g"] != 0)
+    assert all(np.array_equal(a, b) for a, b in zip(got["B"], [b.astype(np.float32) for b in old_B(spec, p)]))
+    p0, _, _ = make_problem(spec, b_std=0.0)               # B = 0: first step of a fine-tuning run
+    ref = run_oracle(spec, p0, tok, lab, 3)
+    got = run_gpu(spec, p0, 3)
+    assert np.allclose(got["losses"], ref["losses"], rtol=1e-4)
+    assert update_rel_err(spec, p0, got["B"], ref["B"]) < 2e-3
+
+
+def test_argument_errors_are_reported_not_faulted():
+    import ctypes as C
+    import paper_2409_15520_b200 as zo
+    from paper_2409_15520_b200 import binding as b
+    spec = ModelSpec(arch=ARCH_OPT, tie_lm_head=True, bf16=False, **TINY)
+    p, tok, lab = make_problem(spec)
+    cfg = zo.make_config(spec)
+    est = zo.Estimator(cfg)
+    prob = zo.DeviceProblem(p, False)
+    for kw, code in [(dict(q=0), 1), (dict(q=spec.q + 1), 1), (dict(E=spec.E + 1), 1),
+                     (dict(S=spec.max_seq + 1), 1), (dict(eps=-1.0), 1), (dict(eps=float("nan")), 1)]:
+        a = dict(E=spec.E, S=spec.S, seed=1, q=spec.q, eps=1e-3, lr=1e-3)
+        a.update(kw)
+        with pytest.raises(zo.ZoError) as ei:
+            est.step(prob, **a)
+        assert ei.value.status == code
+    with pytest.raises(zo.ZoError) as ei:
+        est.losses()
+    assert ei.value.status == 7                             # ZO_ERR_STATE: no step yet
+    # too many labelled positions for max_labelled -> deferred ZO_ERR_INVALID_ARG, B untouched
+    import torch
+    bad = torch.zeros_like(prob.labels)
+    est.step(prob, spec.E, spec.S, 1, spec.q, 1e-3, 1e-3, labels=bad)
+    with pytest.raises(zo.ZoError) as ei:
+        est.losses()
+    assert ei.value.status == 1
+    assert all(np.array_equal(a, c.astype(np.float32)) for a, c in zip(prob.B_numpy(), old_B(spec, p)))
+    est.step(prob, spec.E, spec.S, 1, spec.q, 1e-3, 1e-3)  # the context is still usable
+    est.losses()
+    bad_cfg = zo.make_config(spec.with_(n_heads=5))
+    assert b.zo_workspace_bytes(C.byref(bad_cfg)) == 0
+    with pytest.raises(zo.ZoError) as ei:
+        zo.Estimator(bad_cfg)
+    assert ei.value.status == 2
