@@ -497,12 +497,12 @@ void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int
 // =========================================================================================
 __global__ void ce_rows_kernel(const float* __restrict__ logits, int ldl, int V,
                                const int32_t* __restrict__ lab_val, int EP,
-                               float* __restrict__ row_loss) {
+                               double* __restrict__ row_loss) {
   __shared__ float red[32];
   const int row = blockIdx.x;
   const int lab = lab_val[row % EP];
   if (lab < 0) {
-    if (threadIdx.x == 0) row_loss[row] = 0.f;
+    if (threadIdx.x == 0) row_loss[row] = 0.0;
     return;
   }
   const float* p = logits + (size_t)row * ldl;
@@ -512,10 +512,10 @@ __global__ void ce_rows_kernel(const float* __restrict__ logits, int ldl, int V,
   float s = 0.f;
   for (int c = threadIdx.x; c < V; c += blockDim.x) s += expf(p[c] - m);
   s = block_sum(s, red);
-  if (threadIdx.x == 0) row_loss[row] = (m - p[lab]) + logf(s);
+  if (threadIdx.x == 0) row_loss[row] = ((double)m - (double)p[lab]) + log((double)s);
 }
 void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
-                    int EP, int rows, float* row_loss) {
+                    int EP, int rows, double* row_loss) {
   if (rows <= 0) return;
   ce_rows_kernel<<<rows, 256, 0, st>>>(logits, ldl, V, lab_val, EP, row_loss);
 }
@@ -524,12 +524,12 @@ void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const 
 template <typename T>
 __global__ void label_word_rows_kernel(const T* __restrict__ xh, const T* __restrict__ head,
                                        int d, int w0, int w1, const int32_t* __restrict__ lab_val,
-                                       int EP, float* __restrict__ row_loss) {
+                                       int EP, double* __restrict__ row_loss) {
   __shared__ float red[32];
   const int row = blockIdx.x;
   const int cls = lab_val[row % EP];
   if (cls < 0) {
-    if (threadIdx.x == 0) row_loss[row] = 0.f;
+    if (threadIdx.x == 0) row_loss[row] = 0.0;
     return;
   }
   const T* x = xh + (size_t)row * d;
@@ -544,14 +544,14 @@ __global__ void label_word_rows_kernel(const T* __restrict__ xh, const T* __rest
   a = block_sum(a, red);
   b = block_sum(b, red);
   if (threadIdx.x == 0) {
-    const float m = fmaxf(a, b);
-    const float lse = m + logf(expf(a - m) + expf(b - m));
-    row_loss[row] = lse - (cls == 0 ? a : b);
+    const double da = a, db = b, m = fmax(da, db);
+    const double lse = m + log(exp(da - m) + exp(db - m));
+    row_loss[row] = lse - (cls == 0 ? da : db);
   }
 }
 void launch_label_word_rows(cudaStream_t st, int bf, const void* xh, const void* head, int d,
                             int w0, int w1, const int32_t* lab_val, int EP, int rows,
-                            float* row_loss) {
+                            double* row_loss) {
   if (rows <= 0) return;
   if (bf)
     label_word_rows_kernel<bf16><<<rows, 128, 0, st>>>((const bf16*)xh, (const bf16*)head, d, w0, w1, lab_val, EP, row_loss);
@@ -562,21 +562,21 @@ void launch_label_word_rows(cudaStream_t st, int bf, const void* xh, const void*
 // Mean squared error of one output row against its target (ZO_ARCH_LINEAR).
 template <typename T>
 __global__ void mse_rows_kernel(const T* __restrict__ Y, const float* __restrict__ target, int Tn,
-                                int Tp, int k_out, float* __restrict__ row_loss) {
-  __shared__ float red[32];
+                                int Tp, int k_out, double* __restrict__ row_loss) {
+  __shared__ double red[32];
   const int t = blockIdx.x, n = blockIdx.y;
   const T* y = Y + ((size_t)n * Tp + t) * k_out;
   const float* g = target + (size_t)t * k_out;
-  float s = 0.f;
+  double s = 0.0;
   for (int c = threadIdx.x; c < k_out; c += blockDim.x) {
-    const float dlt = to_f(y[c]) - g[c];
-    s = fmaf(dlt, dlt, s);
+    const double dlt = (double)to_f(y[c]) - (double)g[c];
+    s = fma(dlt, dlt, s);
   }
-  s = block_sum(s, red);
-  if (threadIdx.x == 0) row_loss[(size_t)n * Tn + t] = s / (float)k_out;
+  s = block_sum_d(s, red);
+  if (threadIdx.x == 0) row_loss[(size_t)n * Tn + t] = s / (double)k_out;
 }
 void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target, int n, int T,
-                     int Tp, int k_out, float* row_loss) {
+                     int Tp, int k_out, double* row_loss) {
   if (n <= 0 || T <= 0) return;
   dim3 grid(T, n);
   if (bf) mse_rows_kernel<bf16><<<grid, 128, 0, st>>>((const bf16*)Y, target, T, Tp, k_out, row_loss);
@@ -587,9 +587,10 @@ void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target
 // Per-replica mean over its valid rows: fixed order, fp64 accumulation (Algorithm 1: the
 // loss of a path is the mean over the labelled positions of the batch).
 // =========================================================================================
-__global__ void replica_mean_kernel(const float* __restrict__ row_loss,
+__global__ void replica_mean_kernel(const double* __restrict__ row_loss,
                                     const int32_t* __restrict__ lab_val, int rows,
-                                    float* __restrict__ losses, uint32_t* status) {
+                                    float* __restrict__ losses, double* __restrict__ losses_d,
+                                    uint32_t* status) {
   __shared__ double sd[256];
   __shared__ int sc[256];
   const int n = blockIdx.x;
@@ -597,7 +598,7 @@ __global__ void replica_mean_kernel(const float* __restrict__ row_loss,
   int c = 0;
   for (int i = threadIdx.x; i < rows; i += 256) {
     if (!lab_val || lab_val[i] >= 0) {
-      s += (double)row_loss[(size_t)n * rows + i];
+      s += row_loss[(size_t)n * rows + i];
       ++c;
     }
   }
@@ -612,15 +613,17 @@ __global__ void replica_mean_kernel(const float* __restrict__ row_loss,
     __syncthreads();
   }
   if (threadIdx.x == 0) {
-    const float l = sc[0] > 0 ? (float)(sd[0] / (double)sc[0]) : 0.f;
+    const double ld = sc[0] > 0 ? sd[0] / (double)sc[0] : 0.0;
+    const float l = (float)ld;
     losses[n] = l;
+    losses_d[n] = ld;
     if (!isfinite(l)) atomicOr(status, ST_NONFINITE);
   }
 }
-void launch_replica_mean(cudaStream_t st, const float* row_loss, const int32_t* lab_val, int n,
-                         int rows_per_replica, float* losses, uint32_t* status) {
+void launch_replica_mean(cudaStream_t st, const double* row_loss, const int32_t* lab_val, int n,
+                         int rows_per_replica, float* losses, double* losses_d, uint32_t* status) {
   if (n <= 0) return;
-  replica_mean_kernel<<<n, 256, 0, st>>>(row_loss, lab_val, rows_per_replica, losses, status);
+  replica_mean_kernel<<<n, 256, 0, st>>>(row_loss, lab_val, rows_per_replica, losses, losses_d, status);
 }
 
 // =========================================================================================
@@ -629,13 +632,13 @@ void launch_replica_mean(cudaStream_t st, const float* row_loss, const int32_t* 
 // master copy is written.  Each thread owns one Philox block (4 consecutive elements).
 // =========================================================================================
 constexpr int UPD_MAXQ = 64;
-__global__ void zo_update_kernel(UpdateDesc D, const float* __restrict__ losses,
+__global__ void zo_update_kernel(UpdateDesc D, const double* __restrict__ losses,
                                  float* __restrict__ g_out, int q, float eps, float lr,
                                  uint64_t seed, const uint32_t* __restrict__ status, int write_g) {
   __shared__ float gs[UPD_MAXQ];
   const bool live = eps > 0.f;
   for (int i = threadIdx.x; i < q; i += blockDim.x)
-    gs[i] = live ? (losses[2 * i] - losses[2 * i + 1]) / (2.f * eps) : 0.f;
+    gs[i] = live ? (float)((losses[2 * i] - losses[2 * i + 1]) / (2.0 * (double)eps)) : 0.f;
   __syncthreads();
   if (write_g && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
     for (int i = threadIdx.x; i < q; i += blockDim.x) g_out[i] = gs[i];
@@ -666,7 +669,7 @@ __global__ void zo_update_kernel(UpdateDesc D, const float* __restrict__ losses,
     for (int j = 0; j < left; ++j) Bp[j] -= sc * a[j];
   }
 }
-void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const float* losses, float* g, int q,
+void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g) {
   const long long blks = (D.elems_per_slot + 3) / 4;
   dim3 grid((unsigned)((blks + 127) / 128), D.n_slots, D.count);

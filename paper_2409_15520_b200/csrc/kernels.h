@@ -57,15 +57,16 @@ void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows,
 void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
                        int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status);
 void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
-                    int EP, int rows, float* row_loss);
+                    int EP, int rows, double* row_loss);
 void launch_label_word_rows(cudaStream_t st, int bf, const void* xh, const void* head, int d,
                             int w0, int w1, const int32_t* lab_val, int EP, int rows,
-                            float* row_loss);
+                            double* row_loss);
 void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target, int n, int T,
-                     int Tp, int k_out, float* row_loss);
-// losses[n] = mean of the valid rows of replica n (fixed order, fp64 accumulation).
-void launch_replica_mean(cudaStream_t st, const float* row_loss, const int32_t* lab_val, int n,
-                         int rows_per_replica, float* losses, uint32_t* status);
+                     int Tp, int k_out, double* row_loss);
+// losses[n] = mean of the valid rows of replica n (fixed order, fp64 accumulation); the fp64
+// copy feeds the projected gradients, whose loss difference would drown in fp32 rounding.
+void launch_replica_mean(cudaStream_t st, const double* row_loss, const int32_t* lab_val, int n,
+                         int rows_per_replica, float* losses, double* losses_d, uint32_t* status);
 
 struct UpdateDesc {
   enum { MAX_T = 96 };
@@ -77,7 +78,7 @@ struct UpdateDesc {
 };
 // g_i = (l_{2i} - l_{2i+1}) / (2 eps); B <- B - (lr/q) sum_i g_i z_i  (skipped if *status != 0
 // or lr == 0).  With write_g, block 0 also stores g[0..q).
-void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const float* losses, float* g, int q,
+void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g);
 void launch_perturbation(cudaStream_t st, uint64_t seed, uint32_t tensor, uint32_t query,
                          long long n, uint32_t* u32, float* z);

@@ -17,7 +17,7 @@ char g_init_error[256] = "";
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
-      xh, logits, rowloss, losses, g, status, total;
+      xh, logits, rowloss, losses, losses_d, g, status, total;
 };
 
 inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -98,7 +98,7 @@ Plan make_plan(const zo_config& c) {
     p.qkv = take(Mp * c.d_out * es);                  // Y[n]
     p.tok_stage = take(Tm * c.d_model * es);          // host-variant staging of X
     p.lab_stage = take(Tm * c.d_out * 4);             // and of the targets
-    p.rowloss = take(n * Tm * 4);
+    p.rowloss = take(n * Tm * 8);
   } else {
     const size_t d = c.d_model, f = c.d_ffn, J = (size_t)n_targets(c) * c.lora_rank;
     const size_t P = c.max_labelled, Mh = n * c.max_E * P;
@@ -119,9 +119,10 @@ Plan make_plan(const zo_config& c) {
     p.lab_stage = take(Tm * 4);
     p.xh = take(Mh * d * es);
     if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
-    p.rowloss = take(Mh * 4);
+    p.rowloss = take(Mh * 8);
   }
   p.losses = take(n * 4);
+  p.losses_d = take(n * 8);
   p.g = take((size_t)c.max_q * 4);
   p.status = take(256);
   p.total = off;
@@ -183,8 +184,9 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   float* U = c->at<float>(c->plan.U);
   void* base = c->at<uint8_t>(c->plan.qkv0);
   void* Y = c->at<uint8_t>(c->plan.qkv);
-  float* rowloss = c->at<float>(c->plan.rowloss);
+  double* rowloss = c->at<double>(c->plan.rowloss);
   float* losses = c->at<float>(c->plan.losses);
+  double* losses_d = c->at<double>(c->plan.losses_d);
 
   launch_lora_down(st, bf, X, ki, lora->A[0], U, T, ki, r); ++c->launches;
   GemmDesc G{};
@@ -198,11 +200,11 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
   launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1); ++c->launches;
   launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss); ++c->launches;
-  launch_replica_mean(st, rowloss, nullptr, n, T, losses, status); ++c->launches;
+  launch_replica_mean(st, rowloss, nullptr, n, T, losses, losses_d, status); ++c->launches;
   UpdateDesc D{};
   D.B[0] = lora->B[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
   D.elems_per_slot = (long long)r * ko;
-  launch_zo_update(st, D, losses, c->at<float>(c->plan.g), q, eps, lr, seed, status, 1); ++c->launches;
+  launch_zo_update(st, D, losses_d, c->at<float>(c->plan.g), q, eps, lr, seed, status, 1); ++c->launches;
   return ZO_OK;
 }
 
@@ -226,7 +228,9 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   const float* rope = c->at<float>(c->plan.rope);
   int32_t *lab_idx = c->at<int32_t>(c->plan.lab_idx), *lab_val = c->at<int32_t>(c->plan.lab_val);
   int32_t* lab_cnt = c->at<int32_t>(c->plan.lab_cnt);
-  float *rowloss = c->at<float>(c->plan.rowloss), *losses = c->at<float>(c->plan.losses);
+  double* rowloss = c->at<double>(c->plan.rowloss);
+  float* losses = c->at<float>(c->plan.losses);
+  double* losses_d = c->at<double>(c->plan.losses_d);
   zo_status s;
 #define GEMM(G)                                                                                  \
   do {                                                                                           \
@@ -314,14 +318,14 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     launch_label_word_rows(st, bf, xh, head, d, cf.label_words[0], cf.label_words[1], lab_val, EP, Mh, rowloss);
     ++c->launches;
   }
-  launch_replica_mean(st, rowloss, lab_val, n, EP, losses, status); ++c->launches;
+  launch_replica_mean(st, rowloss, lab_val, n, EP, losses, losses_d, status); ++c->launches;
 
   // projected gradients and ZO-SGD update of every B tensor
   float* g = c->at<float>(c->plan.g);
   if (J == 0) {
     UpdateDesc D{};
     D.count = 0; D.n_slots = 0; D.elems_per_slot = 0;
-    launch_zo_update(st, D, losses, g, q, eps, 0.f, seed, status, 1); ++c->launches;
+    launch_zo_update(st, D, losses_d, g, q, eps, 0.f, seed, status, 1); ++c->launches;
   }
   for (int l0 = 0; l0 < cf.n_layers && J; l0 += UpdateDesc::MAX_T) {
     UpdateDesc D{};
@@ -332,7 +336,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       D.B[i] = lora->B[l0 + i];
       D.tensor_base[i] = (uint32_t)((l0 + i) * nt);
     }
-    launch_zo_update(st, D, losses, g, q, eps, lr, seed, status, l0 == 0); ++c->launches;
+    launch_zo_update(st, D, losses_d, g, q, eps, lr, seed, status, l0 == 0); ++c->launches;
   }
 #undef GEMM
   return ZO_OK;
@@ -507,9 +511,14 @@ zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows) {
                                                    : ctx->last_E * ctx->cfg.max_labelled;
   *host_n_rows = rows;
   if (!host_rows) return ZO_OK;
-  cudaError_t e = cudaMemcpyAsync(host_rows, ctx->at<float>(ctx->plan.rowloss),
-                                  (size_t)2 * ctx->last_q * rows * 4, cudaMemcpyDeviceToHost, ctx->st);
+  const size_t cnt = (size_t)2 * ctx->last_q * rows;
+  double* tmp = new (std::nothrow) double[cnt];
+  if (!tmp) return fail(ctx, ZO_ERR_CUDA, "out of host memory");
+  cudaError_t e = cudaMemcpyAsync(tmp, ctx->at<double>(ctx->plan.rowloss), cnt * 8, cudaMemcpyDeviceToHost, ctx->st);
   if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->st);
+  if (e == cudaSuccess)
+    for (size_t i = 0; i < cnt; ++i) host_rows[i] = (float)tmp[i];
+  delete[] tmp;
   if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "zo_row_losses: %s", cudaGetErrorString(e));
   return ZO_OK;
 }

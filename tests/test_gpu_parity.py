@@ -34,15 +34,14 @@ def _check_fp32(spec, seed, b_std, q=None, eps=None, lr=None, tol_g=1e-2, **kw):
     assert np.allclose(got["losses"], ref["losses"], rtol=1e-4, atol=0), (got["losses"], ref["losses"])
     scale = np.max(np.abs(ref["g"]))
     assert np.all(np.abs(got["g"] - ref["g"]) <= tol_g * scale), (got["g"], ref["g"])
-    assert update_rel_err(spec, p, got["B"], ref["B"]) < max(1e-3, tol_g / 10 * 1.5)
+    assert update_rel_err(spec, p, got["B"], ref["B"]) < 1e-3
     return got, ref
 
 
 def test_linear_fp32_config():
     """The single MP-LoRA linear + MSE configuration, B = 0 and mid-training B."""
     spec = config("linear_fp32")
-    got, ref = _check_fp32(spec, seed=1, b_std=0.0)
-    assert update_rel_err(spec, *[make_problem(spec)[0]], got["B"], ref["B"]) < 1e-3
+    _check_fp32(spec, seed=1, b_std=0.0)
     _check_fp32(spec, seed=2, b_std=0.02)
     _check_fp32(spec, seed=3, b_std=0.02, host=True)
 

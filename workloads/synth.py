@@ -60,15 +60,9 @@ def make_linear_problem(spec: ModelSpec, seed: int = 1234, b_std: float = 0.0):
     return p
 
 
-def make_decoder_problem(spec: ModelSpec, seed: int = 1234, b_std: float = 0.0,
-                         layers=None):
-    """Random-init decoder of the given family.  Per layer: norm1, fused
-    q|k|v projection [3d,d], output projection, norm2, MLP (OPT: fc1 [ffn,d],
-    fc2 [d,ffn]; Llama: fc1 = gate rows then up rows [2ffn,d], fc2 [d,ffn]),
-    LoRA A [n_targets*r, d] and B [n_targets, r, d].  ``layers`` restricts
-    generation to a subset of layer indices (others are left out)."""
-    assert spec.arch in (ARCH_OPT, ARCH_LLAMA)
-    d, f, V, r, nt = spec.d_model, spec.d_ffn, spec.vocab, spec.lora_rank, spec.n_targets
+def make_decoder_globals(spec: ModelSpec, seed: int = 1234):
+    """Embeddings, final norm, LM head, tokens and labels of a random-init decoder."""
+    d, V = spec.d_model, spec.vocab
     h = spec.bf16
     opt = spec.arch == ARCH_OPT
     p = {"tok_emb": _normal(_rng(seed, 10), (V, d), 0.02, h),
@@ -78,35 +72,52 @@ def make_decoder_problem(spec: ModelSpec, seed: int = 1234, b_std: float = 0.0,
         p["final_norm_b"] = _normal(_rng(seed, 13), (d,), 0.02, h)
     if not spec.tie_lm_head:
         p["lm_head"] = _normal(_rng(seed, 14), (V, d), 0.02, h)
-    p["layers"] = []
-    for l in (range(spec.n_layers) if layers is None else layers):
-        f1 = f if opt else 2 * f
-        L = {
-            "norm1_g": _normal(_rng(seed, 100, l, 0), (d,), 0.02, h, mean=1.0),
-            "w_qkv": _normal(_rng(seed, 100, l, 2), (3 * d, d), 0.02, h),
-            "w_o": _normal(_rng(seed, 100, l, 4), (d, d), 0.02, h),
-            "norm2_g": _normal(_rng(seed, 100, l, 6), (d,), 0.02, h, mean=1.0),
-            "w_fc1": _normal(_rng(seed, 100, l, 8), (f1, d), 0.02, h),
-            "w_fc2": _normal(_rng(seed, 100, l, 10), (d, f), 0.02, h),
-            "A": _normal(_rng(seed, 100, l, 12), (nt * r, d), 0.02, h),
-            "B": (_normal(_rng(seed, 100, l, 13), (nt, r, d), b_std, False) if b_std > 0
-                  else np.zeros((nt, r, d), np.float32)),
-        }
-        if opt:
-            L.update({
-                "norm1_b": _normal(_rng(seed, 100, l, 1), (d,), 0.02, h),
-                "b_qkv": _normal(_rng(seed, 100, l, 3), (3 * d,), 0.02, h),
-                "b_o": _normal(_rng(seed, 100, l, 5), (d,), 0.02, h),
-                "norm2_b": _normal(_rng(seed, 100, l, 7), (d,), 0.02, h),
-                "b_fc1": _normal(_rng(seed, 100, l, 9), (f1,), 0.02, h),
-                "b_fc2": _normal(_rng(seed, 100, l, 11), (d,), 0.02, h),
-            })
-        p["layers"].append(L)
     p["tokens"] = _rng(seed, 20).integers(0, V, size=(spec.E, spec.S), dtype=np.int32)
     if spec.loss_kind == LOSS_CE_LABEL_WORDS:
         p["labels"] = label_word_labels(spec, seed)
     else:
         p["labels"] = next_token_labels(p["tokens"], spec.n_labelled)
+    return p
+
+
+def make_decoder_layer(spec: ModelSpec, seed: int, l: int, b_std: float = 0.0):
+    """Frozen tensors and LoRA A/B of decoder block ``l``: norm1, fused q|k|v projection
+    [3d,d], output projection, norm2, MLP (OPT: fc1 [ffn,d], fc2 [d,ffn]; Llama: fc1 = gate
+    rows then up rows [2ffn,d], fc2 [d,ffn]), LoRA A [n_targets*r, d], B [n_targets, r, d]."""
+    d, f, r, nt = spec.d_model, spec.d_ffn, spec.lora_rank, spec.n_targets
+    h = spec.bf16
+    opt = spec.arch == ARCH_OPT
+    f1 = f if opt else 2 * f
+    L = {
+        "norm1_g": _normal(_rng(seed, 100, l, 0), (d,), 0.02, h, mean=1.0),
+        "w_qkv": _normal(_rng(seed, 100, l, 2), (3 * d, d), 0.02, h),
+        "w_o": _normal(_rng(seed, 100, l, 4), (d, d), 0.02, h),
+        "norm2_g": _normal(_rng(seed, 100, l, 6), (d,), 0.02, h, mean=1.0),
+        "w_fc1": _normal(_rng(seed, 100, l, 8), (f1, d), 0.02, h),
+        "w_fc2": _normal(_rng(seed, 100, l, 10), (d, f), 0.02, h),
+        "A": _normal(_rng(seed, 100, l, 12), (nt * r, d), 0.02, h),
+        "B": (_normal(_rng(seed, 100, l, 13), (nt, r, d), b_std, False) if b_std > 0
+              else np.zeros((nt, r, d), np.float32)),
+    }
+    if opt:
+        L.update({
+            "norm1_b": _normal(_rng(seed, 100, l, 1), (d,), 0.02, h),
+            "b_qkv": _normal(_rng(seed, 100, l, 3), (3 * d,), 0.02, h),
+            "b_o": _normal(_rng(seed, 100, l, 5), (d,), 0.02, h),
+            "norm2_b": _normal(_rng(seed, 100, l, 7), (d,), 0.02, h),
+            "b_fc1": _normal(_rng(seed, 100, l, 9), (f1,), 0.02, h),
+            "b_fc2": _normal(_rng(seed, 100, l, 11), (d,), 0.02, h),
+        })
+    return L
+
+
+def make_decoder_problem(spec: ModelSpec, seed: int = 1234, b_std: float = 0.0, layers=None):
+    """Random-init decoder of the given family (globals + every block, or the blocks whose
+    indices are listed in ``layers``)."""
+    assert spec.arch in (ARCH_OPT, ARCH_LLAMA)
+    p = make_decoder_globals(spec, seed)
+    p["layers"] = [make_decoder_layer(spec, seed, l, b_std)
+                   for l in (range(spec.n_layers) if layers is None else layers)]
     return p
 
 
