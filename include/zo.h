@@ -179,6 +179,17 @@ ZO_API zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_ro
 /* Number of kernels the last zo_step enqueued. */
 ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 
+/* Profiling aid.  While enabled, every kernel launch of zo_step is bracketed by CUDA events
+ * on the context's stream.  zo_profile_read synchronises the stream and returns, per kernel
+ * class, the summed device time in ms, the summed algorithmic flops 2*M*N*K (GEMM classes
+ * only) and the number of launches since the previous read.  Arrays of ZO_PROFILE_CLASSES. */
+enum { ZO_PROF_GEMM_TC = 0, ZO_PROF_GEMM_SIMT, ZO_PROF_ATTENTION, ZO_PROF_NORM, ZO_PROF_LORA_DOWN,
+       ZO_PROF_LORA_APPLY, ZO_PROF_ROPE, ZO_PROF_SWIGLU, ZO_PROF_LOSS, ZO_PROF_UPDATE,
+       ZO_PROF_MISC, ZO_PROFILE_CLASSES };
+ZO_API zo_status zo_profile_enable(zo_ctx* ctx, int32_t on);
+ZO_API zo_status zo_profile_read(zo_ctx* ctx, double* host_ms, double* host_flops,
+                                 int32_t* host_launches);
+
 ZO_API void zo_free(zo_ctx* ctx);
 ZO_API const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo_init failure */
 

@@ -75,6 +75,10 @@ zo_losses = _sig("zo_losses", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p])
 zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)])
 zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
 zo_free = _sig("zo_free", None, [C.c_void_p])
+zo_profile_enable = _sig("zo_profile_enable", C.c_int, [C.c_void_p, C.c_int32])
+zo_profile_read = _sig("zo_profile_read", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p])
+PROFILE_CLASSES = ["gemm_tc", "gemm_simt", "attention", "norm", "lora_down", "lora_apply", "rope",
+                   "swiglu", "loss", "update", "misc"]
 zo_last_error = _sig("zo_last_error", C.c_char_p, [C.c_void_p])
 zo_perturbation = _sig("zo_perturbation", C.c_int, [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
                                                     C.c_int64, C.c_void_p, C.c_void_p])
@@ -112,7 +116,7 @@ class DeviceProblem:
     """Device copies of a synthetic problem (dict of numpy arrays as produced by the
     workload generators) plus the zo_weights / zo_lora structures pointing at them."""
 
-    def __init__(self, p: dict, bf16: bool, device="cuda"):
+    def __init__(self, p: dict, bf16: bool, device="cuda", n_layers=None):
         self.dtype = torch.bfloat16 if bf16 else torch.float32
         self.device = device
         self._keep = []
@@ -134,7 +138,8 @@ class DeviceProblem:
                 t = self._up(p.get(k))
                 setattr(self, k, t)
                 setattr(self.weights, k, _ptr(t))
-            n = len(p["layers"])
+            # p["layers"] may be a generator (one block in host memory at a time)
+            n = len(p["layers"]) if n_layers is None else n_layers
             self._layers = (ZoLayerWeights * n)()
             self._A, self.B = [], []
             for l, L in enumerate(p["layers"]):
@@ -215,6 +220,17 @@ class Estimator:
         out = np.zeros((2 * self.q, n.value), np.float32)
         self._check(zo_row_losses(self._h, out.ctypes.data_as(C.c_void_p), C.byref(n)))
         return out
+
+    def profile_enable(self, on=True):
+        self._check(zo_profile_enable(self._h, int(on)))
+
+    def profile_read(self):
+        """{class: (ms, flops, launches)} since the previous read; synchronises the stream."""
+        n = len(PROFILE_CLASSES)
+        ms, fl, cnt = np.zeros(n), np.zeros(n), np.zeros(n, np.int32)
+        self._check(zo_profile_read(self._h, ms.ctypes.data_as(C.c_void_p),
+                                    fl.ctypes.data_as(C.c_void_p), cnt.ctypes.data_as(C.c_void_p)))
+        return {k: (float(ms[i]), float(fl[i]), int(cnt[i])) for i, k in enumerate(PROFILE_CLASSES)}
 
     def launch_count(self):
         return int(zo_launch_count(self._h))

@@ -291,6 +291,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ epilogue warps
     const int wq = warp & 3;                       // tensor-memory lane quarter of this warp
     const int et = threadIdx.x - 64;               // 0..127
+    const bool out_vec_ok = ((uintptr_t)P.out & 15) == 0 && (P.ldo % (P.out_f32 ? 4 : 8)) == 0;
+    const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
     uint32_t titer = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++titer) {
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -384,9 +386,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (!row_ok) continue;
         const bool full_chunk = col0 + 32 <= P.N;
+        // 16-byte vector accesses need the row pitch (and base) to keep rows 16-byte aligned
+        const bool vec_out = full_chunk && out_vec_ok;
         if (P.res) {
           const bf16* rp = P.res + (size_t)rrow * P.ldr + col0;
-          if (full_chunk) {
+          if (full_chunk && res_vec_ok) {
 #pragma unroll
             for (int j8 = 0; j8 < 4; ++j8) {
               float t[8];
@@ -402,7 +406,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (P.out_f32) {
           float* op = (float*)P.out + (size_t)row * P.ldo + col0;
-          if (full_chunk) {
+          if (vec_out) {
 #pragma unroll
             for (int j4 = 0; j4 < 8; ++j4)
               *reinterpret_cast<float4*>(op + 4 * j4) =
@@ -414,7 +418,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         } else {
           bf16* op = (bf16*)P.out + (size_t)row * P.ldo + col0;
-          if (full_chunk) {
+          if (vec_out) {
 #pragma unroll
             for (int j8 = 0; j8 < 4; ++j8)
               *reinterpret_cast<uint4*>(op + 8 * j8) =

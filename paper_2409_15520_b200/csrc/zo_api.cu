@@ -4,6 +4,7 @@
 #include <string.h>
 
 #include <new>
+#include <vector>
 
 #include "../../include/zo.h"
 #include "common.cuh"
@@ -131,7 +132,16 @@ Plan make_plan(const zo_config& c) {
 
 }  // namespace
 
+enum { PC_GEMM_TC = 0, PC_GEMM_SIMT, PC_ATTN, PC_NORM, PC_LORA_DOWN, PC_LORA_APPLY, PC_ROPE,
+       PC_SWIGLU, PC_LOSS, PC_UPDATE, PC_MISC, PC_COUNT };
+static_assert(PC_COUNT == ZO_PROFILE_CLASSES, "profile classes out of sync with zo.h");
+
+struct ProfRec { int cat; double flops; cudaEvent_t e0, e1; };
+
 struct zo_ctx {
+  int prof_on;
+  std::vector<ProfRec>* prof;      // records of the launches since the last read
+  std::vector<cudaEvent_t>* evpool; // events free for reuse
   zo_config cfg;
   Plan plan;
   uint8_t* ws;
@@ -146,6 +156,33 @@ struct zo_ctx {
 
 namespace {
 
+// Brackets one launch with CUDA events on the context's stream when profiling is on.
+struct ProfScope {
+  zo_ctx* c;
+  ProfRec r;
+  bool live;
+  ProfScope(zo_ctx* ctx, int cat, double flops) : c(ctx), live(false) {
+    if (!c || !c->prof_on) return;
+    r.cat = cat; r.flops = flops; r.e0 = r.e1 = nullptr;
+    for (cudaEvent_t* e : {&r.e0, &r.e1}) {
+      if (!c->evpool->empty()) { *e = c->evpool->back(); c->evpool->pop_back(); }
+      else if (cudaEventCreate(e) != cudaSuccess) { *e = nullptr; }
+    }
+    if (!r.e0 || !r.e1) return;
+    live = cudaEventRecord(r.e0, c->st) == cudaSuccess;
+  }
+  ~ProfScope() {
+    if (!live) return;
+    if (cudaEventRecord(r.e1, c->st) == cudaSuccess) c->prof->push_back(r);
+  }
+};
+#define PROF(cat, flops, call)      \
+  do {                              \
+    ProfScope ps_(c, cat, flops);   \
+    call;                           \
+    ++c->launches;                  \
+  } while (0)
+
 zo_status fail(zo_ctx* c, zo_status s, const char* fmt, const char* a = "") {
   snprintf(c->err, sizeof(c->err), fmt, a);
   return s;
@@ -154,7 +191,9 @@ zo_status fail(zo_ctx* c, zo_status s, const char* fmt, const char* a = "") {
 // GEMM dispatch: tensor-core kernel for bf16 unless the validation flag asks otherwise.
 zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const GemmDesc& G,
                    uint32_t* status, int n_sms, int* launches, char* err, size_t errn) {
-  if (bf && !(flags & ZO_FLAG_SIMT_GEMM)) {
+  const bool tcore = bf && !(flags & ZO_FLAG_SIMT_GEMM);
+  ProfScope ps(c, tcore ? PC_GEMM_TC : PC_GEMM_SIMT, 2.0 * G.M * (double)G.N * G.K);
+  if (tcore) {
     const int e = launch_gemm_tc(st, G, status, n_sms);
     if (e) {
       snprintf(err, errn, "tensor-core GEMM launch failed (code %d: %s)", e,
@@ -165,7 +204,6 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
     launch_gemm_simt(st, bf, G);
   }
   ++*launches;
-  (void)c;
   return ZO_OK;
 }
 
@@ -188,7 +226,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   float* losses = c->at<float>(c->plan.losses);
   double* losses_d = c->at<double>(c->plan.losses_d);
 
-  launch_lora_down(st, bf, X, ki, lora->A[0], U, T, ki, r); ++c->launches;
+  PROF(PC_LORA_DOWN, 0.0, launch_lora_down(st, bf, X, ki, lora->A[0], U, T, ki, r));
   GemmDesc G{};
   G.A = X; G.lda = ki; G.W = w->linear_w; G.M = T; G.N = ko; G.K = ki;
   G.out = base; G.ldo = ko; G.bias = w->linear_bias;
@@ -198,13 +236,13 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   L.U = U; L.ldu = r; L.B = lora->B[0]; L.r = r; L.width = ko;
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
-  launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1); ++c->launches;
-  launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss); ++c->launches;
-  launch_replica_mean(st, rowloss, nullptr, n, T, losses, losses_d, status); ++c->launches;
+  PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
+  PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss));
+  PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss, nullptr, n, T, losses, losses_d, status));
   UpdateDesc D{};
   D.B[0] = lora->B[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
   D.elems_per_slot = (long long)r * ko;
-  launch_zo_update(st, D, losses_d, c->at<float>(c->plan.g), q, eps, lr, seed, status, 1); ++c->launches;
+  PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, c->at<float>(c->plan.g), q, eps, lr, seed, status, 1));
   return ZO_OK;
 }
 
@@ -239,11 +277,10 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   } while (0)
 
   // shared prefix: embedding on the T shared tokens, once for all 2q replicas
-  launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, S, d, cf.vocab, status);
-  ++c->launches;
+  PROF(PC_MISC, 0.0, launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, S, d, cf.vocab, status));
   const int P = cf.max_labelled, EP = E * P;
   const int n_classes = cf.loss_kind == ZO_LOSS_CE_LABEL_WORDS ? 2 : cf.vocab;
-  launch_label_scan(st, labels, E, S, P, n_classes, lab_idx, lab_val, lab_cnt, status); ++c->launches;
+  PROF(PC_MISC, 0.0, launch_label_scan(st, labels, E, S, P, n_classes, lab_idx, lab_val, lab_cnt, status));
 
   for (int l = 0; l < cf.n_layers; ++l) {
     const zo_layer_weights& W = w->layers[l];
@@ -251,37 +288,35 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     const int rows = first ? Tp : M;           // layer 0 still works on the shared block
     void* hin = first ? h0 : h;
     void* xn = first ? x0 : x;
-    launch_norm(st, bf, nkind, hin, xn, W.norm1_g, W.norm1_b, rows, d, cf.norm_eps, nullptr, 0, 0);
-    ++c->launches;
+    PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, hin, xn, W.norm1_g, W.norm1_b, rows, d, cf.norm_eps, nullptr, 0, 0));
     LoraDesc L{};
     L.U = U; L.ldu = J; L.B = J ? lora->B[l] : nullptr; L.r = r; L.width = d;
     for (int j = 0; j < 3; ++j) L.slot_of_sec[j] = c->slot_of_sec[j];
     L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = (uint32_t)(l * nt);
     L.rows_per_replica = Tp;
-    if (J) { launch_lora_down(st, bf, xn, d, lora->A[l], U, rows, d, J); ++c->launches; }
+    if (J) { PROF(PC_LORA_DOWN, 0.0, launch_lora_down(st, bf, xn, d, lora->A[l], U, rows, d, J)); }
     GemmDesc G{};
     G.A = xn; G.lda = d; G.W = W.w_qkv; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
     if (first) {
       // first perturbed layer: one base product on the shared block, expanded to 2q outputs
       G.out = qkv0; G.ldo = 3 * d;
       GEMM(G);
-      launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3); ++c->launches;
+      PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
     } else if (J && fused_lora_ok(bf, cf.flags, Tp, d)) {
       G.out = qkv; G.ldo = 3 * d; G.lora = &L;
       GEMM(G);
     } else {
       G.out = qkv; G.ldo = 3 * d;
       GEMM(G);
-      if (J) { launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3); ++c->launches; }
+      if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
-    if (!opt) { launch_rope(st, bf, qkv, M, Tp, S, d, H, rope); ++c->launches; }
-    launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H); ++c->launches;
+    if (!opt) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
+    PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H));
     GemmDesc O{};
     O.A = x; O.lda = d; O.W = W.w_o; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
     O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0;
     GEMM(O);
-    launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0);
-    ++c->launches;
+    PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0));
     GemmDesc F1{};
     F1.A = x; F1.lda = d; F1.W = W.w_fc1; F1.M = M; F1.K = d; F1.bias = W.b_fc1;
     if (opt) {
@@ -290,7 +325,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     } else if (unfused_mlp) {
       F1.N = 2 * f; F1.out = gu; F1.ldo = 2 * f;
       GEMM(F1);
-      launch_swiglu(st, bf, gu, a, M, f); ++c->launches;
+      PROF(PC_SWIGLU, 0.0, launch_swiglu(st, bf, gu, a, M, f));
     } else {
       F1.N = 2 * f; F1.out = a; F1.ldo = f; F1.swiglu = 1;
       GEMM(F1);
@@ -304,8 +339,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   // per-replica loss on the labelled rows only
   const int Mh = n * EP;
   void* xh = c->at<uint8_t>(c->plan.xh);
-  launch_norm(st, bf, nkind, h, xh, w->final_norm_g, w->final_norm_b, Mh, d, cf.norm_eps, lab_idx, EP, Tp);
-  ++c->launches;
+  PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, xh, w->final_norm_g, w->final_norm_b, Mh, d, cf.norm_eps, lab_idx, EP, Tp));
   const void* head = cf.tie_lm_head ? w->tok_emb : w->lm_head;
   if (cf.loss_kind == ZO_LOSS_CE_FULL_VOCAB) {
     float* logits = c->at<float>(c->plan.logits);
@@ -313,19 +347,18 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     Hd.A = xh; Hd.lda = d; Hd.W = head; Hd.M = Mh; Hd.N = cf.vocab; Hd.K = d;
     Hd.out = logits; Hd.ldo = cf.vocab; Hd.out_f32 = 1;
     GEMM(Hd);
-    launch_ce_rows(st, logits, cf.vocab, cf.vocab, lab_val, EP, Mh, rowloss); ++c->launches;
+    PROF(PC_LOSS, 0.0, launch_ce_rows(st, logits, cf.vocab, cf.vocab, lab_val, EP, Mh, rowloss));
   } else {
-    launch_label_word_rows(st, bf, xh, head, d, cf.label_words[0], cf.label_words[1], lab_val, EP, Mh, rowloss);
-    ++c->launches;
+    PROF(PC_LOSS, 0.0, launch_label_word_rows(st, bf, xh, head, d, cf.label_words[0], cf.label_words[1], lab_val, EP, Mh, rowloss));
   }
-  launch_replica_mean(st, rowloss, lab_val, n, EP, losses, losses_d, status); ++c->launches;
+  PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss, lab_val, n, EP, losses, losses_d, status));
 
   // projected gradients and ZO-SGD update of every B tensor
   float* g = c->at<float>(c->plan.g);
   if (J == 0) {
     UpdateDesc D{};
     D.count = 0; D.n_slots = 0; D.elems_per_slot = 0;
-    launch_zo_update(st, D, losses_d, g, q, eps, 0.f, seed, status, 1); ++c->launches;
+    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, 0.f, seed, status, 1));
   }
   for (int l0 = 0; l0 < cf.n_layers && J; l0 += UpdateDesc::MAX_T) {
     UpdateDesc D{};
@@ -336,7 +369,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       D.B[i] = lora->B[l0 + i];
       D.tensor_base[i] = (uint32_t)((l0 + i) * nt);
     }
-    launch_zo_update(st, D, losses_d, g, q, eps, lr, seed, status, l0 == 0); ++c->launches;
+    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, lr, seed, status, l0 == 0));
   }
 #undef GEMM
   return ZO_OK;
@@ -433,6 +466,8 @@ zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
   zo_ctx* c = new (std::nothrow) zo_ctx;
   if (!c) { snprintf(g_init_error, sizeof(g_init_error), "out of host memory"); return ZO_ERR_CUDA; }
   memset(c, 0, sizeof(*c));
+  c->prof = new (std::nothrow) std::vector<ProfRec>();
+  c->evpool = new (std::nothrow) std::vector<cudaEvent_t>();
   c->cfg = *cfg; c->plan = plan; c->ws = (uint8_t*)workspace; c->st = (cudaStream_t)cuda_stream;
   c->bf = cfg->precision == ZO_BF16; c->n_sms = sms;
   c->nt = cfg->arch == ZO_ARCH_LINEAR ? 1 : n_targets(*cfg);
@@ -525,7 +560,41 @@ zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows) {
 
 int32_t zo_launch_count(const zo_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
-void zo_free(zo_ctx* ctx) { delete ctx; }
+void zo_free(zo_ctx* ctx) {
+  if (!ctx) return;
+  if (ctx->prof) {
+    for (ProfRec& r : *ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    delete ctx->prof;
+  }
+  if (ctx->evpool) {
+    for (cudaEvent_t e : *ctx->evpool) cudaEventDestroy(e);
+    delete ctx->evpool;
+  }
+  delete ctx;
+}
+
+zo_status zo_profile_enable(zo_ctx* ctx, int32_t on) {
+  if (!ctx || !ctx->prof || !ctx->evpool) return ZO_ERR_INVALID_ARG;
+  ctx->prof_on = on ? 1 : 0;
+  return ZO_OK;
+}
+
+zo_status zo_profile_read(zo_ctx* ctx, double* host_ms, double* host_flops, int32_t* host_launches) {
+  if (!ctx || !host_ms || !host_flops || !host_launches) return ZO_ERR_INVALID_ARG;
+  for (int i = 0; i < PC_COUNT; ++i) { host_ms[i] = 0.0; host_flops[i] = 0.0; host_launches[i] = 0; }
+  cudaError_t e = cudaStreamSynchronize(ctx->st);
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "zo_profile_read: %s", cudaGetErrorString(e));
+  for (ProfRec& r : *ctx->prof) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess) {
+      host_ms[r.cat] += ms; host_flops[r.cat] += r.flops; ++host_launches[r.cat];
+    }
+    ctx->evpool->push_back(r.e0);
+    ctx->evpool->push_back(r.e1);
+  }
+  ctx->prof->clear();
+  return ZO_OK;
+}
 
 const char* zo_last_error(const zo_ctx* ctx) { return ctx ? ctx->err : g_init_error; }
 
