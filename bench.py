@@ -1,0 +1,274 @@
+#!/usr/bin/env python
+"""Benchmark of the parallelised ZO estimator step (one zo_step = one pass of the whole hot path:
+shared prefix, 2q-replica MP-LoRA forward, 2q losses, q projected gradients, ZO-SGD update).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama7b] [--impl ours|reference]
+
+Prints one JSON line.  `value` = perturbed-forward tokens/s = 2q*E*S*steps / device time, inputs
+resident in HBM; `e2e` = the same through zo_step_host (tokens/labels copied from pinned host memory,
+losses read back every step).  N > 1 runs N independent replicas of the job (the path is not sharded).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import config, make_decoder_globals, make_decoder_layer, make_linear_problem  # noqa: E402
+from workloads.spec import ARCH_LINEAR, ARCH_OPT  # noqa: E402
+
+METRIC, UNIT = "perturbed_fwd_tokens_per_s", "tokens/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tflops=p["bf16_tflops"], tflops_sustained=p["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "200"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=lambda: self.lines.extend(self.proc.stdout), daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def load_problem(spec, seed=1234, b_std=0.01):
+    """Synthetic weights on the device, one decoder block in host memory at a time."""
+    import paper_2409_15520_b200 as zo
+    if spec.arch == ARCH_LINEAR:
+        return zo.DeviceProblem(make_linear_problem(spec, seed=seed, b_std=b_std), spec.bf16)
+    p = make_decoder_globals(spec, seed)
+    p["layers"] = (make_decoder_layer(spec, seed, l, b_std) for l in range(spec.n_layers))
+    return zo.DeviceProblem(p, spec.bf16, n_layers=spec.n_layers)
+
+
+def algorithmic_flops_per_step(spec):
+    """GEMM flops the method must do per step (nothing saved by sharing is counted as done):
+    per replica row and layer 2*(4 d^2 + c d ffn), LM head on labelled rows, LoRA terms."""
+    n, T = 2 * spec.q, spec.E * spec.S
+    if spec.arch == ARCH_LINEAR:
+        return 2.0 * T * spec.d_model * spec.d_out
+    d, f = spec.d_model, spec.d_ffn
+    c = 2 if spec.arch == ARCH_OPT else 3
+    per_row = 2.0 * (4 * d * d + c * d * f)
+    return per_row * spec.n_layers * n * T + 2.0 * n * spec.E * spec.n_labelled * d * spec.vocab
+
+
+def oracle_sample(spec, seed=1234):
+    """Bounded CPU sample of the same workload: the oracle's zo_step with q = 1 (one +/- pair) on ONE
+    sequence of the batch through a 2-block copy of the model.  Returns (seconds, token-forwards done,
+    scale to full depth)."""
+    import oracle
+    if spec.arch == ARCH_LINEAR:
+        small = spec.with_(q=1)
+        p = make_linear_problem(small, seed=seed, b_std=0.01)
+        t0 = time.perf_counter()
+        oracle.zo_step(small, p, p["X"], p["target"], 1, 1, spec.eps, spec.lr)
+        return time.perf_counter() - t0, 2 * small.E * small.S, 1.0, "q=1 on the full token block"
+    L = min(2, spec.n_layers)
+    small = spec.with_(n_layers=L, E=1, q=1)
+    p = make_decoder_globals(small, seed)
+    p["layers"] = [make_decoder_layer(small, seed, l, 0.01) for l in range(L)]
+    t0 = time.perf_counter()
+    oracle.zo_step(small, p, p["tokens"], p["labels"], 1, 1, spec.eps, spec.lr)
+    dt = time.perf_counter() - t0
+    return dt, 2 * small.S, spec.n_layers / L, f"q=1, 1 sequence of {small.S} tokens, {L} of {spec.n_layers} blocks (time scaled by depth)"
+
+
+def run_reference(args, spec):
+    """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+    cores = torch.get_num_threads()
+    for _ in range(args.warmup if args.warmup < 2 else 1):
+        oracle_sample(spec)
+    times = []
+    for _ in range(args.steps):
+        dt, toks, scale, what = oracle_sample(spec)
+        times.append(dt * scale)
+    sec = float(np.sum(times))
+    value = toks * args.steps / sec
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sec / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": what},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llama7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override the depth (profiling captures of a small case)")
+    ap.add_argument("--q", type=int, default=0, help="override q (profiling captures of a small case)")
+    args = ap.parse_args()
+    spec = config(args.workload)
+    if args.layers:
+        spec = spec.with_(n_layers=args.layers)
+    if args.q:
+        spec = spec.with_(q=args.q)
+    if args.impl == "reference":
+        return run_reference(args, spec)
+
+    import torch
+    import torch.distributed as dist
+    import paper_2409_15520_b200 as zo
+
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    prob = load_problem(spec)
+    est = zo.Estimator(zo.make_config(spec))
+    E, S, q, eps, lr = spec.E, spec.S, spec.q, spec.eps, spec.lr
+    tokens_per_step = 2 * q * E * S
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        est.step(prob, E, S, 100 + i, q, eps, lr)
+    est.losses()
+    sampler = ClockSampler(local)
+    est.profile_enable(True)
+    est.profile_read()
+    barrier()
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for i in range(args.steps):
+        est.step(prob, E, S, 1000 + i, q, eps, lr)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = ev0.elapsed_time(ev1)
+    prof = est.profile_read()
+    est.profile_enable(False)
+    losses, g = est.losses()
+    launches = est.launch_count() * args.steps
+
+    # end to end: host tokens/labels in, losses out, every step
+    barrier()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        est.step_host(prob, E, S, 2000 + i, q, eps, lr)
+        est.losses()
+    e1.record()
+    barrier()
+    ms_e2e = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
+    h2d = prob.host_tokens.numel() * prob.host_tokens.element_size() + \
+        prob.host_labels.numel() * prob.host_labels.element_size()
+    d2h = (2 * q + q) * 4 + 4
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = _peaks()
+    gms, gfl, gcnt = prof["gemm_tc"]
+    gemm_tflops = gfl / (gms * 1e-3) / 1e12 if gms > 0 else 0.0
+    inside_long_step = ms / args.steps > 200.0
+    peak = peaks["tflops_sustained"] if inside_long_step else peaks["tflops"]
+    total_prof = sum(v[0] for v in prof.values())
+    line = {
+        "metric": METRIC, "value": world * tokens_per_step * args.steps / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if spec.bf16 else "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "arch": {0: "linear", 1: "opt", 2: "llama"}[spec.arch],
+                   "n_layers": spec.n_layers, "d_model": spec.d_model, "d_ffn": spec.d_ffn, "vocab": spec.vocab,
+                   "lora_rank": spec.lora_rank, "q": q, "E": E, "S": S, "replicas": 2 * q,
+                   "token_rows_per_step": tokens_per_step, "eps": eps, "lr": lr,
+                   "l2": "inputs larger than L2 (weights and activations of several GB stream every step)",
+                   "parallelism": "replicas only" if world > 1 else "1 gpu"},
+        "zo_steps_per_s": world * args.steps / (ms * 1e-3),
+        "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,
+        "clocks": clocks,
+        "e2e": {"value": world * tokens_per_step * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches,
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tflops, "peak": peak,
+                     "unit": "TFLOP/s", "frac": gemm_tflops / peak if peak else None,
+                     "peak_source": f"{peaks['source']} ({'sustained' if inside_long_step else 'burst'} bf16)",
+                     "launches": gcnt, "avg_launch_ms": gms / gcnt if gcnt else None, "traffic": None},
+        "kernel_time_share": {k: round(v[0] / total_prof, 4) for k, v in prof.items() if v[2]},
+        "kernel_ms_per_step": {k: round(v[0] / args.steps, 3) for k, v in prof.items() if v[2]},
+        "loss_mean": float(np.mean(losses)),
+    }
+    if not args.no_cpu_baseline and world == 1:
+        import torch as _t
+        dt, toks, scale, what = oracle_sample(spec)
+        line["cpu_baseline"] = {"value": toks / (dt * scale), "unit": UNIT, "cores": _t.get_num_threads(),
+                                "kind": "oracle", "sample": what, "seconds": dt}
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
