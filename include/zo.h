@@ -216,6 +216,32 @@ ZO_API zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const v
                             int32_t x_replicated, void* scratch, size_t scratch_bytes,
                             uint32_t flags);
 
+/* zo_mp_lora_linear without any caller-provided scratch (the paper has no counterpart: this is
+ * a packaging variant of the entry point above, same arithmetic, same results).
+ *
+ * For callers that cannot allocate device memory where they need the layer: code hosted inside
+ * a framework whose allocator owns the device budget, plug-ins that receive only their input and
+ * output buffers, and loops where an allocation would stall the device.  The scratch lives in a
+ * fixed array of ZO_STATIC_SCRATCH_BYTES inside the library's device image; every GPU that loads
+ * the library holds those bytes until the process exits.  The call allocates nothing (no
+ * cudaMalloc, cudaFree or allocating library routine); X, W, bias, A, B and Y are still the
+ * caller's buffers.
+ *   - Problems whose zo_mp_lora_scratch_bytes() exceeds ZO_STATIC_SCRATCH_BYTES are rejected
+ *     with ZO_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device looks up the array's device address (a host-side step);
+ *     make that first call before starting any stream capture on that device.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; what
+ *     must start at zero is cleared by every call.  Two calls that overlap on the GPU (different
+ *     streams, no ordering between them) race on it: order them, or use zo_mp_lora_linear with
+ *     separate scratch buffers. */
+#define ZO_STATIC_SCRATCH_BYTES (16u << 20)
+ZO_API zo_status zo_mp_lora_linear_static(void* cuda_stream, int32_t precision, const void* X,
+                                          const void* W, const void* bias, const void* A,
+                                          const float* B, void* Y, int32_t T, int32_t k_in,
+                                          int32_t k_out, int32_t r, float scale, uint64_t seed,
+                                          uint32_t tensor_id, int32_t q, float eps,
+                                          int32_t x_replicated, uint32_t flags);
+
 #ifdef __cplusplus
 }
 #endif

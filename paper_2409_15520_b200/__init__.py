@@ -7,5 +7,5 @@ has not been built (``python -m paper_2409_15520_b200.build``).
 """
 from .binding import (  # noqa: F401
     LIB, ZoConfig, ZoError, Estimator, DeviceProblem, make_config, perturbation,
-    mp_lora_linear, STATUS_NAMES,
+    mp_lora_linear, mp_lora_linear_static, STATUS_NAMES,
 )

@@ -89,6 +89,13 @@ zo_mp_lora_linear = _sig("zo_mp_lora_linear", C.c_int, [
     C.c_float, C.c_int32, C.c_void_p, C.c_size_t, C.c_uint32])
 
 
+zo_mp_lora_linear_static = _sig("zo_mp_lora_linear_static", C.c_int, [
+    C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+    C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_uint64, C.c_uint32, C.c_int32,
+    C.c_float, C.c_int32, C.c_uint32])
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
 def make_config(spec, *, max_q=None, max_E=None, max_seq=None, max_labelled=None, flags=0,
                 precision=None) -> ZoConfig:
     """zo_config from a shape record with the attribute names of workloads.ModelSpec."""
@@ -277,4 +284,18 @@ def mp_lora_linear(X, W, bias, A, B, T, q, scale, seed, tensor_id, eps, x_replic
     status = int(scratch.view(torch.int32)[(base - scratch.data_ptr()) // 4].item())
     if status:
         raise ZoError(5, f"device status word {status}")
+    return Y
+
+
+def mp_lora_linear_static(X, W, bias, A, B, Y, T, q, scale, seed, tensor_id, eps, x_replicated, flags=0):
+    """The MP-LoRA linear through the entry point that allocates nothing: the caller passes the
+    output tensor Y [2q, T, k_out] as well, and the library's built-in scratch is used.  Raises
+    ZoError(ZO_ERR_WORKSPACE) when the problem does not fit STATIC_SCRATCH_BYTES."""
+    bf = X.dtype == torch.bfloat16
+    k_out, k_in = W.shape
+    st = zo_mp_lora_linear_static(C.c_void_p(torch.cuda.current_stream().cuda_stream), int(bf), _ptr(X),
+                                  _ptr(W), _ptr(bias), _ptr(A), _ptr(B), _ptr(Y), T, k_in, k_out,
+                                  A.shape[0], scale, seed, tensor_id, q, eps, int(x_replicated), flags)
+    if st:
+        raise ZoError(st, "zo_mp_lora_linear_static")
     return Y
