@@ -88,17 +88,116 @@ __global__ void norm_kernel(int kind, const T* __restrict__ x, T* __restrict__ o
   }
 }
 
+// Vectorised variant: 16-byte accesses, the row is read once and kept in registers.
+// Requires d % VEC == 0 and d <= blockDim.x * VEC * NV.
+template <typename T, int NV>
+__global__ void __launch_bounds__(256)
+norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
+                const T* __restrict__ b, int d, float eps, const int32_t* __restrict__ lab_idx,
+                int EP, int Tp) {
+  constexpr int VEC = 16 / sizeof(T);
+  __shared__ float red[32];
+  const int row = blockIdx.x;
+  long long src = row;
+  if (lab_idx) {
+    const int n = row / EP, j = row % EP;
+    const int li = lab_idx[j];
+    src = li < 0 ? -1 : (long long)n * Tp + li;
+  }
+  T* o = out + (size_t)row * d;
+  const int nvec = d / VEC;
+  if (src < 0) {
+    for (int v = threadIdx.x; v < nvec; v += blockDim.x)
+      *reinterpret_cast<uint4*>(o + v * VEC) = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  const T* xr = x + (size_t)src * d;
+  float val[NV][VEC];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int v = threadIdx.x + i * blockDim.x;
+    if (v < nvec) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(xr + v * VEC);
+      const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        val[i][j] = to_f(e[j]);
+        s += kind == 0 ? val[i][j] : val[i][j] * val[i][j];
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) val[i][j] = 0.f;
+    }
+  }
+  float mu = 0.f, rstd;
+  if (kind == 0) {
+    mu = block_sum(s, red) / d;
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const int v = threadIdx.x + i * blockDim.x;
+      if (v < nvec) {
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+          const float t = val[i][j] - mu;
+          q += t * t;
+        }
+      }
+    }
+    rstd = rsqrtf(block_sum(q, red) / d + eps);
+  } else {
+    rstd = rsqrtf(block_sum(s, red) / d + eps);
+  }
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int v = threadIdx.x + i * blockDim.x;
+    if (v < nvec) {
+      const uint4 graw = *reinterpret_cast<const uint4*>(g + v * VEC);
+      const T* ge = reinterpret_cast<const T*>(&graw);
+      uint4 braw = make_uint4(0, 0, 0, 0);
+      if (kind == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
+      const T* be = reinterpret_cast<const T*>(&braw);
+      uint4 oraw;
+      T* oe = reinterpret_cast<T*>(&oraw);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j) {
+        const float y = (val[i][j] - mu) * rstd * to_f(ge[j]) + ((kind == 0 && b) ? to_f(be[j]) : 0.f);
+        oe[j] = from_f<T>(y);
+      }
+      *reinterpret_cast<uint4*>(o + v * VEC) = oraw;
+    }
+  }
+}
+
+template <typename T>
+static void norm_dispatch(cudaStream_t st, int kind, const void* x, void* out, const void* g,
+                          const void* b, int rows, int d, float eps, const int32_t* lab_idx, int EP,
+                          int Tp) {
+  constexpr int VEC = 16 / sizeof(T);
+  const bool aligned = (((uintptr_t)x | (uintptr_t)out | (uintptr_t)g | (uintptr_t)b) & 15) == 0;
+  if (aligned && d % VEC == 0 && d <= 256 * VEC * 4) {
+    const int nvec = d / VEC;
+    int th = nvec < 256 ? ((nvec + 31) / 32) * 32 : 256;
+    const int nv = (nvec + th - 1) / th;
+    if (nv <= 1)
+      norm_vec_kernel<T, 1><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
+    else if (nv == 2)
+      norm_vec_kernel<T, 2><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
+    else
+      norm_vec_kernel<T, 4><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
+    return;
+  }
+  const int th = d >= 2048 ? 256 : 128;
+  norm_kernel<T><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
+}
+
 void launch_norm(cudaStream_t st, int bf, int kind, const void* x, void* out, const void* g,
                  const void* b, int rows, int d, float eps, const int32_t* lab_idx, int EP,
                  int Tp) {
   if (rows <= 0) return;
-  const int th = d >= 2048 ? 256 : 128;
-  if (bf)
-    norm_kernel<bf16><<<rows, th, 0, st>>>(kind, (const bf16*)x, (bf16*)out, (const bf16*)g,
-                                           (const bf16*)b, d, eps, lab_idx, EP, Tp);
-  else
-    norm_kernel<float><<<rows, th, 0, st>>>(kind, (const float*)x, (float*)out, (const float*)g,
-                                            (const float*)b, d, eps, lab_idx, EP, Tp);
+  if (bf) norm_dispatch<bf16>(st, kind, x, out, g, b, rows, d, eps, lab_idx, EP, Tp);
+  else norm_dispatch<float>(st, kind, x, out, g, b, rows, d, eps, lab_idx, EP, Tp);
 }
 
 // =========================================================================================
@@ -257,8 +356,8 @@ __global__ void rope_table_kernel(float* tab, int max_seq, int half, double thet
   const int s = i / half, j = i % half;
   const double inv = pow(theta, -2.0 * (double)j / (double)(2 * half));
   const double a = (double)s * inv;
-  tab[2 * i] = (float)cos(a);
-  tab[2 * i + 1] = (float)sin(a);
+  tab[(size_t)s * 2 * half + j] = (float)cos(a);          // row s: cos[0..half) then sin[0..half)
+  tab[(size_t)s * 2 * half + half + j] = (float)sin(a);
 }
 void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float theta) {
   const int n = max_seq * (dh / 2);
@@ -278,7 +377,7 @@ __global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S,
   const int which = (int)(rest % 2);  // 0 = q, 1 = k
   const long long row = rest / 2;
   const int s = (int)((row % Tp) % S);
-  const float c = tab[2 * (s * half + j)], sn = tab[2 * (s * half + j) + 1];
+  const float c = tab[(size_t)s * 2 * half + j], sn = tab[(size_t)s * 2 * half + half + j];
   T* p = qkv + (size_t)row * 3 * d + (size_t)which * d + h * 2 * half + j;
   const float x1 = to_f(p[0]), x2 = to_f(p[half]);
   p[0] = from_f<T>(x1 * c - x2 * sn);

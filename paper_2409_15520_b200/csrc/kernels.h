@@ -53,6 +53,11 @@ void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, in
                  const float* tab);
 void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, int E,
                            int S, int Tp, int d, int H);
+// Tensor-core causal attention for bf16 with head_dim 64 or 128; applies the rotary embedding to
+// q and k on the fly when rope != null (table rows: cos[0..dh/2) | sin[0..dh/2)).
+bool attention_mma_supported(int dh);
+void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp,
+                          int d, int H, const float* rope);
 void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows, int ffn);
 void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
                        int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status);

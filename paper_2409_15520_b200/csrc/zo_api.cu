@@ -207,6 +207,28 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
   return ZO_OK;
 }
 
+// Down-projection U = X A^T (fp32 out): on the tensor cores for bf16 operands (it only has to
+// read X once; the MMA work is small), on CUDA cores otherwise.
+zo_status run_lora_down(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const void* X, int ldx,
+                        const void* A, float* U, int rows, int K, int J, uint32_t* status, int n_sms,
+                        int* launches, char* err, size_t errn) {
+  if (bf && !(flags & ZO_FLAG_SIMT_GEMM) && K % 8 == 0 && ldx % 8 == 0) {
+    GemmDesc G{};
+    G.A = X; G.lda = ldx; G.W = A; G.M = rows; G.N = J; G.K = K; G.out = U; G.ldo = J; G.out_f32 = 1;
+    ProfScope ps(c, PC_LORA_DOWN, 2.0 * rows * (double)J * K);
+    const int e = launch_gemm_tc(st, G, status, n_sms);
+    if (e) {
+      snprintf(err, errn, "tensor-core down-projection launch failed (code %d)", e);
+      return ZO_ERR_CUDA;
+    }
+  } else {
+    ProfScope ps(c, PC_LORA_DOWN, 2.0 * rows * (double)J * K);
+    launch_lora_down(st, bf, X, ldx, A, U, rows, K, J);
+  }
+  ++*launches;
+  return ZO_OK;
+}
+
 // Can the MP-LoRA term ride in the tensor-core GEMM's epilogue?
 inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
   return bf && !(flags & ZO_FLAG_SIMT_GEMM) && Tp % 128 == 0 && width % 32 == 0;
@@ -226,11 +248,13 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   float* losses = c->at<float>(c->plan.losses);
   double* losses_d = c->at<double>(c->plan.losses_d);
 
-  PROF(PC_LORA_DOWN, 0.0, launch_lora_down(st, bf, X, ki, lora->A[0], U, T, ki, r));
+  zo_status s = run_lora_down(c, st, bf, cf.flags, X, ki, lora->A[0], U, T, ki, r, status, c->n_sms,
+                              &c->launches, c->err, sizeof(c->err));
+  if (s) return s;
   GemmDesc G{};
   G.A = X; G.lda = ki; G.W = w->linear_w; G.M = T; G.N = ko; G.K = ki;
   G.out = base; G.ldo = ko; G.bias = w->linear_bias;
-  zo_status s = run_gemm(c, st, bf, cf.flags, G, status, c->n_sms, &c->launches, c->err, sizeof(c->err));
+  s = run_gemm(c, st, bf, cf.flags, G, status, c->n_sms, &c->launches, c->err, sizeof(c->err));
   if (s) return s;
   LoraDesc L{};
   L.U = U; L.ldu = r; L.B = lora->B[0]; L.r = r; L.width = ko;
@@ -294,7 +318,11 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     for (int j = 0; j < 3; ++j) L.slot_of_sec[j] = c->slot_of_sec[j];
     L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = (uint32_t)(l * nt);
     L.rows_per_replica = Tp;
-    if (J) { PROF(PC_LORA_DOWN, 0.0, launch_lora_down(st, bf, xn, d, lora->A[l], U, rows, d, J)); }
+    if (J) {
+      s = run_lora_down(c, st, bf, cf.flags, xn, d, lora->A[l], U, rows, d, J, status, c->n_sms,
+                        &c->launches, c->err, sizeof(c->err));
+      if (s) return s;
+    }
     GemmDesc G{};
     G.A = xn; G.lda = d; G.W = W.w_qkv; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
     if (first) {
@@ -310,8 +338,12 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(G);
       if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
-    if (!opt) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
-    PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H));
+    if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
+      PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, E, S, Tp, d, H, opt ? nullptr : rope));
+    } else {
+      if (!opt) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
+      PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H));
+    }
     GemmDesc O{};
     O.A = x; O.lda = d; O.W = W.w_o; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
     O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0;
@@ -643,7 +675,11 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   float* U = (float*)(sp + 256);
   void* base = sp + 256 + up(rows * r * 4, 256);
   if (cudaMemsetAsync(status, 0, 4, st) != cudaSuccess) return ZO_ERR_CUDA;
-  launch_lora_down(st, bf, X, k_in, A, U, (int)rows, k_in, r);
+  int launches = 0;
+  char err[128];
+  zo_status s = run_lora_down(nullptr, st, bf, flags, X, k_in, A, U, (int)rows, k_in, r, status, sms,
+                              &launches, err, sizeof(err));
+  if (s) return s;
   LoraDesc L{};
   L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
@@ -651,9 +687,6 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   GemmDesc G{};
   G.A = X; G.lda = k_in; G.W = W; G.M = (int)rows; G.N = k_out; G.K = k_in; G.bias = bias;
   G.ldo = k_out;
-  int launches = 0;
-  char err[128];
-  zo_status s;
   if (!x_replicated) {
     G.out = base;
     s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));

@@ -115,6 +115,25 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
     assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
 
 
+@pytest.mark.parametrize("arch,S", [(ARCH_LLAMA, 100), (ARCH_OPT, 64), (ARCH_LLAMA, 1)])
+def test_decoder_bf16_head_dim_128(arch, S):
+    """Tensor-core attention with head_dim 128 (rotary embedding applied while staging), ragged
+    and single-token sequences; compared with the oracle and with the CUDA-core attention."""
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
+                     **{**TINY, "d_model": 256, "n_heads": 2, "d_ffn": 264, "vocab": 517, "S": S,
+                        "E": 2, "max_seq": max(S, 2), "q": 2, "n_layers": 2,
+                        "n_labelled": 1 if S == 1 else 5})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    if S == 1:                       # a one-token sequence has no next token: label the token itself
+        lab = tok.copy()
+        p["labels"] = lab
+    ref = run_oracle(spec, p, tok, lab, 41)
+    got = run_gpu(spec, p, 41)
+    simt = run_gpu(spec, p, 41, flags=SIMT)
+    assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
+    assert np.allclose(got["losses"], simt["losses"], rtol=2e-3, atol=0), (got["losses"], simt["losses"])
+
+
 @pytest.mark.parametrize("x_replicated", [0, 1])
 @pytest.mark.parametrize("r", [8, 16, 64])
 def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
