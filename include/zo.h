@@ -69,7 +69,10 @@ enum { ZO_LOSS_MSE = 0, ZO_LOSS_CE_FULL_VOCAB = 1, ZO_LOSS_CE_LABEL_WORDS = 2 };
 enum { ZO_TARGET_Q = 1, ZO_TARGET_K = 2, ZO_TARGET_V = 4 };
 /* flags: ZO_FLAG_SIMT_GEMM routes every bf16 GEMM (and attention) through the plain
  * CUDA-core validation kernels instead of the tensor-core ones (cross-checking only). */
-enum { ZO_FLAG_SIMT_GEMM = 1 };
+enum { ZO_FLAG_SIMT_GEMM = 1,
+       /* ZO_FLAG_GEMM_1CTA: tensor-core GEMMs run one CTA per 128-row tile instead of the default
+        * CTA pairs on 256-row tiles (diagnostic A/B switch; same results up to rounding order). */
+       ZO_FLAG_GEMM_1CTA = 2 };
 
 typedef struct zo_ctx zo_ctx; /* opaque; owned by the library; released by zo_free */
 

@@ -10,6 +10,11 @@
 //     with z_i regenerated from the Philox seed inside the epilogue (never in HBM).  Every
 //     128-row tile lies inside one replica, so the perturbed B columns of the tile are built
 //     once in shared memory and reused by its 128 rows.
+//   * PAIR variant (default): two CTAs of a cluster work on one 256 x 256 tile with
+//     tcgen05.mma.cta_group::2 - each CTA stages its own 128 rows of A and its 128-row half of
+//     the weight tile, so the shared-memory traffic per SM drops by a third; 6 stages.  The
+//     leader CTA issues the MMAs and releases stages/accumulators in both CTAs with multicast
+//     commits; the peer's TMA completes on the leader's barrier.
 //   * every mbarrier wait is bounded; on expiry the kernel raises ST_TIMEOUT in the status
 //     word, drains its copies and MMAs, frees its tensor memory and returns.
 #include <cuda.h>
@@ -21,10 +26,17 @@ namespace zo {
 
 namespace tc {
 
-constexpr int BM = 128, BN = 256, BK = 64, STAGES = 4;
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int MAX_STAGES = 6;
 constexpr uint32_t A_BYTES = BM * BK * 2;       // 16 KiB
-constexpr uint32_t B_BYTES = BN * BK * 2;       // 32 KiB (two 128-row boxes)
-constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t BOX_BYTES = 128 * BK * 2;    // one 128-row box of the weight tile, 16 KiB
+template <bool PAIR> struct Cfg {
+  static constexpr int STAGES = PAIR ? 6 : 4;
+  static constexpr uint32_t B_BYTES = PAIR ? BOX_BYTES : 2 * BOX_BYTES;   // per CTA
+  static constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr uint32_t TX_BYTES = PAIR ? 2 * STAGE_BYTES : STAGE_BYTES;  // per full barrier
+};
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;     // clears the CTA-rank bit of a shared::cluster address
 constexpr int LORA_MAXR = 64;
 constexpr uint32_t LORA_BUF_FLOATS = LORA_MAXR * 32;  // one 32-column chunk of s*(B + k eps z)
 constexpr uint32_t TMEM_COLS = 512;
@@ -32,12 +44,12 @@ constexpr int THREADS = 192;                    // warp 0: TMA, warp 1: MMA, war
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct Ctrl {
-  unsigned long long full[STAGES], empty[STAGES], tfull[2], tempty[2], drain;
+  unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2], drain;
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
 };
-constexpr size_t SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + 2 * LORA_BUF_FLOATS * 4 + sizeof(Ctrl);
+constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + 2 * LORA_BUF_FLOATS * 4 + sizeof(Ctrl);  // both variants: 192 KiB of stages
 
 struct Params {
   int M, N, K;              // N: accumulator columns (swiglu: d_ffn, the number of OUTPUT columns)
@@ -88,6 +100,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctrl* c
     if (mbar_try(bar, parity)) return true;
     if ((it & 63u) == 0u) {
       if (c->abort) return false;
+      if (*reinterpret_cast<volatile uint32_t*>(status) & ST_TIMEOUT) { c->abort = 1u; return false; }
       if (gtimer() - t0 > WAIT_LIMIT_NS) {
         c->abort = 1u;
         atomicOr(status, ST_TIMEOUT);
@@ -110,6 +123,28 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
+// Pair variant: data lands in this CTA's shared memory, completion is signalled on the barrier
+// at the same offset in the leader (even-ranked) CTA.  No multicast.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                 uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar & PEER_MASK)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK)
+               : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -119,6 +154,22 @@ __device__ __forceinline__ void tc_fence_after() {
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
                : "memory");
+}
+// Arrives on the barrier at this offset in BOTH CTAs of the pair once the MMAs issued so far retire.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+      "h"((unsigned short)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                            uint32_t idesc, uint32_t accumulate) {
+  const uint32_t z = 0u;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(z)
+      : "memory");
 }
 __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
                                        uint32_t idesc, uint32_t accumulate) {
@@ -160,6 +211,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                            ((uint32_t)(BM >> 4) << 24);
+// The pair instruction spans both CTAs: M = 256.
+constexpr uint32_t IDESC_PAIR = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
+                                ((uint32_t)((2 * BM) >> 4) << 24);
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
   __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -176,8 +230,8 @@ __device__ __forceinline__ void unpack8(const uint4 v, float* f) {
 
 // Tile raster: groups of GROUP_M row tiles sweep all column tiles, so a wave of CTAs shares
 // both a few weight panels and a bounded set of activation panels in L2.
-constexpr int GROUP_M = 32;
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int GROUP_M, int& tm,
+                                            int& tn) {
   const int per_group = GROUP_M * tiles_n;
   const int g = tile / per_group, r = tile - g * per_group;
   const int gm0 = g * GROUP_M;
@@ -186,17 +240,25 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
   tm = gm0 + (r - tn * gsz);
 }
 
+template <bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const Params P) {
+  constexpr int STAGES = Cfg<PAIR>::STAGES;
+  constexpr uint32_t STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
+  constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
+  constexpr int GROUP_M = PAIR ? 8 : 16;             // 16 row tiles of 128 per raster group
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   float* lbuf = (float*)(smem + STAGES * STAGE_BYTES);
   Ctrl* ctrl = (Ctrl*)(smem + STAGES * STAGE_BYTES + 2 * LORA_BUF_FLOATS * 4);
   const uint32_t tiles_base = smem_u32(smem);
+  const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
+  const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int n_units = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tiles_m = (P.M + BM - 1) / BM;
+  const int tiles_m = (P.M + TILE_M - 1) / TILE_M;
   const int ncol_tile = P.swiglu ? 128 : BN;          // output columns covered by one tile
   const int tiles_n = (P.N + ncol_tile - 1) / ncol_tile;
   const int num_tiles = tiles_m * tiles_n;
@@ -209,7 +271,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctrl->tfull[a]), 1);
-      mbar_init(smem_u32(&ctrl->tempty[a]), 4);
+      mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 8 : 4);
     }
     mbar_init(smem_u32(&ctrl->drain), 1);
     ctrl->abort = 0u;
@@ -218,14 +280,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
-                     smem_u32(&ctrl->tmem_base)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (PAIR) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                       smem_u32(&ctrl->tmem_base)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
+                       smem_u32(&ctrl->tmem_base)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync();                            // the peer's barriers are initialised too
   tc_fence_after();
   const uint32_t tmem_base = ctrl->tmem_base;
 
@@ -234,10 +305,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       uint32_t issued = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = unit; tile < num_tiles && ok; tile += n_units) {
         int tm, tn;
-        tile_coords(tile, tiles_m, tiles_n, tm, tn);
-        const int m0 = tm * BM;
+        tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+        const int m0 = tm * TILE_M + (int)rank * BM;
         const int brow0 = tn * ncol_tile;
         const int brow1 = P.swiglu ? P.N + brow0 : brow0 + 128;
         for (int kb = 0; kb < num_kb; ++kb, ++issued) {
@@ -245,13 +316,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
           const uint32_t sa = tiles_base + s * STAGE_BYTES;
-          mbar_expect_tx(bar, STAGE_BYTES);
-          tma_load_2d(sa, &tmA, kb * BK, m0, bar);
-          tma_load_2d(sa + A_BYTES, &tmB, kb * BK, brow0, bar);
-          tma_load_2d(sa + A_BYTES + B_BYTES / 2, &tmB, kb * BK, brow1, bar);
+          if (PAIR) {
+            // the leader's barrier collects the bytes of both CTAs
+            if (rank == 0) mbar_expect_tx(bar, Cfg<PAIR>::TX_BYTES);
+            tma_load_2d_pair(sa, &tmA, kb * BK, m0, bar);
+            tma_load_2d_pair(sa + A_BYTES, &tmB, kb * BK, rank == 0 ? brow0 : brow1, bar);
+          } else {
+            mbar_expect_tx(bar, Cfg<PAIR>::TX_BYTES);
+            tma_load_2d(sa, &tmA, kb * BK, m0, bar);
+            tma_load_2d(sa + A_BYTES, &tmB, kb * BK, brow0, bar);
+            tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
+          }
         }
       }
-      if (!ok) {
+      if (!ok && (!PAIR || rank == 0)) {
         // abort: let the copies already issued land before the CTA goes away
         const uint32_t lo = issued > STAGES ? issued - STAGES : 0u;
         for (uint32_t i = lo; i < issued; ++i)
@@ -260,10 +338,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && rank == 0) {
       uint32_t consumed = 0, titer = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++titer) {
+      for (int tile = unit; tile < num_tiles && ok; tile += n_units, ++titer) {
         const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
         if (!mbar_wait(smem_u32(&ctrl->tempty[a]), aph ^ 1u, ctrl, P.status)) { ok = false; break; }
         tc_fence_after();
@@ -275,12 +353,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t sa = tiles_base + s * STAGE_BYTES;
           const uint64_t ad = smem_desc(sa), bd = smem_desc(sa + A_BYTES);
 #pragma unroll
-          for (int k = 0; k < BK / 16; ++k)
-            tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC,
-                   (uint32_t)((kb | k) != 0));
-          tc_commit(smem_u32(&ctrl->empty[s]));   // frees the stage once these MMAs retire
+          for (int k = 0; k < BK / 16; ++k) {
+            if (PAIR)
+              tc_mma_pair(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC_PAIR,
+                          (uint32_t)((kb | k) != 0));
+            else
+              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC,
+                     (uint32_t)((kb | k) != 0));
+          }
+          // frees the stage (in both CTAs of a pair) once these MMAs retire
+          if (PAIR) tc_commit_pair(smem_u32(&ctrl->empty[s]));
+          else tc_commit(smem_u32(&ctrl->empty[s]));
         }
-        if (ok) tc_commit(smem_u32(&ctrl->tfull[a]));
+        if (ok) {
+          if (PAIR) tc_commit_pair(smem_u32(&ctrl->tfull[a]));
+          else tc_commit(smem_u32(&ctrl->tfull[a]));
+        }
       }
       if (!ok) {
         tc_commit(smem_u32(&ctrl->drain));        // wait for the MMAs already issued
@@ -294,7 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool out_vec_ok = ((uintptr_t)P.out & 15) == 0 && (P.ldo % (P.out_f32 ? 4 : 8)) == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
     uint32_t titer = 0;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++titer) {
+    for (int tile = unit; tile < num_tiles; tile += n_units, ++titer) {
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
       if (et == 0) ctrl->ep_go = mbar_wait(smem_u32(&ctrl->tfull[a]), aph, ctrl, P.status) ? 1u : 0u;
       ep_bar();
@@ -303,8 +391,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!go) break;
       tc_fence_after();
       int tm, tn;
-      tile_coords(tile, tiles_m, tiles_n, tm, tn);
-      const int m0 = tm * BM, n0 = tn * ncol_tile;
+      tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+      const int m0 = tm * TILE_M + (int)rank * BM, n0 = tn * ncol_tile;
       const int row = m0 + wq * 32 + lane;
       const bool row_ok = row < P.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + a * BN;
@@ -434,19 +522,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // accumulator buffer drained: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[a]));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_leader(smem_u32(&ctrl->tempty[a]));   // the leader waits for both CTAs
+        else mbar_arrive(smem_u32(&ctrl->tempty[a]));
+      }
     }
   }
 
   // ------------------------------------------------------------------ teardown
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync();      // neither CTA leaves while the other may still signal or write into it
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"(TMEM_COLS)
-                 : "memory");
+    if (PAIR)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(TMEM_COLS)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                   "r"(TMEM_COLS)
+                   : "memory");
   }
 }
 
@@ -466,8 +563,11 @@ int gemm_tc_init() {
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return e ? (int)e : 999;
   g_encode = (EncodeTiledFn)fn;
-  e = cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
   return (int)e;
 }
 
@@ -505,11 +605,34 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.has_lora = G.lora ? 1 : 0;
   if (G.lora) P.L = *G.lora; else P.L = LoraDesc{};
   P.status = status;
-  const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
+  if (!G.single_cta && P.M > tc::BM) {
+    // pairs of CTAs (clusters of 2) on 256-row tiles
+    static int max_clusters = 0;                       // co-resident pairs on this device
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(tc::THREADS); cfg.dynamicSmemBytes = tc::SMEM_BYTES; cfg.stream = st;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (max_clusters == 0) {
+      cfg.gridDim = dim3(2 * (n_sms / 2));
+      int mc = 0;
+      if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true>, &cfg) != cudaSuccess || mc < 1) {
+        cudaGetLastError();
+        mc = n_sms / 2;
+      }
+      max_clusters = mc < n_sms / 2 ? mc : n_sms / 2;
+    }
+    const long long tiles = (long long)((P.M + 2 * tc::BM - 1) / (2 * tc::BM)) * tiles_n;
+    const int pairs = (int)(tiles < max_clusters ? tiles : max_clusters);
+    cfg.gridDim = dim3(2 * pairs);
+    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true>, tmA, tmB, P);
+  }
+  const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
   const long long tiles = (long long)tiles_m * tiles_n;
   const int grid = (int)(tiles < n_sms ? tiles : n_sms);
-  tc::gemm_tc_kernel<<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, P);
+  tc::gemm_tc_kernel<false><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, P);
   return (int)cudaGetLastError();
 }
 

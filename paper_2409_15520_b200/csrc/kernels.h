@@ -33,6 +33,7 @@ struct GemmDesc {
   int act;
   int swiglu;                   // 1: W = [gate rows | up rows] (N = 2 * d_ffn), out = silu(g)*u
   const LoraDesc* lora;         // null: plain GEMM
+  int single_cta;               // 1: one CTA per 128-row tile instead of CTA pairs on 256-row tiles
 };
 
 // --- elementwise / reduction kernels (bf = 1: bfloat16 tensors, 0: float) -------------------
