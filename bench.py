@@ -153,6 +153,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override the depth (profiling captures of a small case)")
     ap.add_argument("--q", type=int, default=0, help="override q (profiling captures of a small case)")
+    ap.add_argument("--flags", type=int, default=0, help="zo_config.flags (diagnostic kernel switches)")
     args = ap.parse_args()
     spec = config(args.workload)
     if args.layers:
@@ -175,7 +176,7 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     prob = load_problem(spec)
-    est = zo.Estimator(zo.make_config(spec))
+    est = zo.Estimator(zo.make_config(spec, flags=args.flags))
     E, S, q, eps, lr = spec.E, spec.S, spec.q, spec.eps, spec.lr
     tokens_per_step = 2 * q * E * S
 
@@ -230,7 +231,8 @@ def main():
         return
 
     peaks = _peaks()
-    gms, gfl, gcnt = prof["gemm_tc"]
+    gemm_classes = [k for k in prof if k.startswith("gemm_") and k != "gemm_simt"]
+    gms, gfl, gcnt = (sum(prof[k][i] for k in gemm_classes) for i in range(3))
     gemm_tflops = gfl / (gms * 1e-3) / 1e12 if gms > 0 else 0.0
     inside_long_step = ms / args.steps > 200.0
     peak = peaks["tflops_sustained"] if inside_long_step else peaks["tflops"]
@@ -256,6 +258,8 @@ def main():
                      "unit": "TFLOP/s", "frac": gemm_tflops / peak if peak else None,
                      "peak_source": f"{peaks['source']} ({'sustained' if inside_long_step else 'burst'} bf16)",
                      "launches": gcnt, "avg_launch_ms": gms / gcnt if gcnt else None, "traffic": None},
+        "gemm_tflops_by_class": {k: round(prof[k][1] / (prof[k][0] * 1e-3) / 1e12, 1)
+                                 for k in gemm_classes if prof[k][0] > 0},
         "kernel_time_share": {k: round(v[0] / total_prof, 4) for k, v in prof.items() if v[2]},
         "kernel_ms_per_step": {k: round(v[0] / args.steps, 3) for k, v in prof.items() if v[2]},
         "loss_mean": float(np.mean(losses)),

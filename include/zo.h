@@ -185,10 +185,13 @@ ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 /* Profiling aid.  While enabled, every kernel launch of zo_step is bracketed by CUDA events
  * on the context's stream.  zo_profile_read synchronises the stream and returns, per kernel
  * class, the summed device time in ms, the summed algorithmic flops 2*M*N*K (GEMM classes
- * only) and the number of launches since the previous read.  Arrays of ZO_PROFILE_CLASSES. */
+ * only) and the number of launches since the previous read.  Arrays of ZO_PROFILE_CLASSES.
+ * Decoder GEMMs are booked under their own classes (QKV, O, FC1, FC2, HEAD); ZO_PROF_GEMM_TC
+ * holds the tensor-core GEMMs of ZO_ARCH_LINEAR. */
 enum { ZO_PROF_GEMM_TC = 0, ZO_PROF_GEMM_SIMT, ZO_PROF_ATTENTION, ZO_PROF_NORM, ZO_PROF_LORA_DOWN,
        ZO_PROF_LORA_APPLY, ZO_PROF_ROPE, ZO_PROF_SWIGLU, ZO_PROF_LOSS, ZO_PROF_UPDATE,
-       ZO_PROF_MISC, ZO_PROFILE_CLASSES };
+       ZO_PROF_MISC, ZO_PROF_GEMM_QKV, ZO_PROF_GEMM_O, ZO_PROF_GEMM_FC1, ZO_PROF_GEMM_FC2,
+       ZO_PROF_GEMM_HEAD, ZO_PROFILE_CLASSES };
 ZO_API zo_status zo_profile_enable(zo_ctx* ctx, int32_t on);
 ZO_API zo_status zo_profile_read(zo_ctx* ctx, double* host_ms, double* host_flops,
                                  int32_t* host_launches);

@@ -78,7 +78,8 @@ zo_free = _sig("zo_free", None, [C.c_void_p])
 zo_profile_enable = _sig("zo_profile_enable", C.c_int, [C.c_void_p, C.c_int32])
 zo_profile_read = _sig("zo_profile_read", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p])
 PROFILE_CLASSES = ["gemm_tc", "gemm_simt", "attention", "norm", "lora_down", "lora_apply", "rope",
-                   "swiglu", "loss", "update", "misc"]
+                   "swiglu", "loss", "update", "misc", "gemm_qkv", "gemm_o", "gemm_fc1", "gemm_fc2",
+                   "gemm_head"]
 zo_last_error = _sig("zo_last_error", C.c_char_p, [C.c_void_p])
 zo_perturbation = _sig("zo_perturbation", C.c_int, [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
                                                     C.c_int64, C.c_void_p, C.c_void_p])

@@ -1,10 +1,10 @@
 // Causal attention for the bf16 path: softmax(Q K^T / sqrt(dh) + causal) V over the n*E
-// sequences of the replicated batch, with the rotary embedding of q and k applied while the
-// tiles are staged in shared memory (no separate pass over the activations).
+// sequences of the replicated batch (q and k already carry their rotary embedding).
 //
 // One CTA (4 warps) per (64-query tile, head, sequence); each warp owns 16 query rows.
-// K/V tiles of 64 keys; scores and P V on warp-level tensor-core MMAs (m16n8k16, bf16 in,
-// fp32 accumulate) with an online softmax; fully masked key tiles are skipped.  Attention is
+// K/V tiles of 64 keys stream through a double-buffered cp.async pipeline; scores and P V on
+// warp-level tensor-core MMAs (m16n8k16, bf16 in, fp32 accumulate) with an online softmax;
+// fully masked key tiles are skipped.  Attention is
 // ~1 % of the step's flops, so this kernel only has to stay off the critical path.
 #include "common.cuh"
 #include "kernels.h"
@@ -48,59 +48,35 @@ __device__ __forceinline__ uint4 pack8f(const float* f) {
   return make_uint4(pack2(f[0], f[1]), pack2(f[2], f[3]), pack2(f[4], f[5]), pack2(f[6], f[7]));
 }
 
-// Stage a [64][DH] tile (rows s0.., columns col0.. of qkv) into shared memory, rotating the
-// pairs (j, j + DH/2) by the position's angle when ROT is set.  Rows >= S are zero-filled.
-template <int DH, bool ROT>
-__device__ __forceinline__ void stage_tile(bf16* dst, const bf16* __restrict__ qkv, size_t row_base,
-                                           int ld, int col0, int s0, int S,
-                                           const float* __restrict__ rope) {
+// Asynchronously stage a [64][DH] tile (rows s0.., columns col0.. of qkv) into shared memory.
+// Rows >= S are zero-filled (zero-size source).
+template <int DH>
+__device__ __forceinline__ void stage_tile_async(bf16* dst, const bf16* __restrict__ qkv,
+                                                 size_t row_base, int ld, int col0, int s0, int S) {
   constexpr int LDS = DH + 8;
-  constexpr int HALF = DH / 2;
-  if (ROT) {
-    constexpr int VPR = HALF / 8;                     // 16-byte vectors per half row
-    for (int i = threadIdx.x; i < 64 * VPR; i += 128) {
-      const int r = i / VPR, j0 = (i % VPR) * 8;
-      const int s = s0 + r;
-      uint4 lo = make_uint4(0, 0, 0, 0), hi = lo;
-      if (s < S) {
-        const bf16* p = qkv + (row_base + s) * (size_t)ld + col0 + j0;
-        float x1[8], x2[8], y1[8], y2[8];
-        unpack8f(*reinterpret_cast<const uint4*>(p), x1);
-        unpack8f(*reinterpret_cast<const uint4*>(p + HALF), x2);
-        const float* cs = rope + (size_t)s * DH + j0;  // [s][cos 0..HALF) | sin 0..HALF)]
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float c = cs[j], sn = cs[HALF + j];
-          y1[j] = x1[j] * c - x2[j] * sn;
-          y2[j] = x2[j] * c + x1[j] * sn;
-        }
-        lo = pack8f(y1);
-        hi = pack8f(y2);
-      }
-      *reinterpret_cast<uint4*>(dst + r * LDS + j0) = lo;
-      *reinterpret_cast<uint4*>(dst + r * LDS + HALF + j0) = hi;
-    }
-  } else {
-    constexpr int VPR = DH / 8;
-    for (int i = threadIdx.x; i < 64 * VPR; i += 128) {
-      const int r = i / VPR, j0 = (i % VPR) * 8;
-      const int s = s0 + r;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (s < S) v = *reinterpret_cast<const uint4*>(qkv + (row_base + s) * (size_t)ld + col0 + j0);
-      *reinterpret_cast<uint4*>(dst + r * LDS + j0) = v;
-    }
+  constexpr int VPR = DH / 8;                          // 16-byte vectors per row
+  for (int i = threadIdx.x; i < 64 * VPR; i += 128) {
+    const int r = i / VPR, j0 = (i % VPR) * 8;
+    const int s = s0 + r;
+    const bf16* src = qkv + (row_base + min(s, S - 1)) * (size_t)ld + col0 + j0;
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + r * LDS + j0);
+    const int bytes = s < S ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
   }
 }
+__device__ __forceinline__ void cp_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
 
-template <int DH, bool ROPE>
+template <int DH>
 __global__ void __launch_bounds__(128)
 attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E, int S, int Tp,
-                     int d, const float* __restrict__ rope) {
+                     int d) {
   extern __shared__ __align__(16) uint8_t sm_raw[];
   constexpr int LDS = DH + 8;
   bf16* Qs = reinterpret_cast<bf16*>(sm_raw);
-  bf16* Ks = Qs + 64 * LDS;
-  bf16* Vs = Ks + 64 * LDS;
+  bf16* KVs = Qs + 64 * LDS;                           // [2 buffers][K tile | V tile]
   const int qt = gridDim.x - 1 - blockIdx.x;          // longest tiles first
   const int q0 = qt * 64, h = blockIdx.y, sq = blockIdx.z;
   const int n = sq / E, b = sq % E;
@@ -109,7 +85,13 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
 
-  stage_tile<DH, ROPE>(Qs, qkv, row_base, ld, h * DH, q0, S, rope);
+  const int kend = min(S, q0 + 64);
+  const int n_kt = (kend + 63) / 64;
+  stage_tile_async<DH>(Qs, qkv, row_base, ld, h * DH, q0, S);
+  stage_tile_async<DH>(KVs, qkv, row_base, ld, d + h * DH, 0, S);
+  stage_tile_async<DH>(KVs + 64 * LDS, qkv, row_base, ld, 2 * d + h * DH, 0, S);
+  cp_commit();
+  cp_wait<0>();
   __syncthreads();
   // Q fragments of this warp's 16 rows stay in registers for the whole kernel
   uint32_t qf[DH / 16][4];
@@ -130,12 +112,16 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
   const float sl2 = rsqrtf((float)DH) * 1.4426950408889634f;   // 1/sqrt(dh) * log2(e)
   const int qrow0 = q0 + warp * 16 + g;                         // this thread's rows: qrow0, qrow0+8
 
-  const int kend = min(S, q0 + 64);
-  for (int k0 = 0; k0 < kend; k0 += 64) {
-    __syncthreads();                                            // previous tile fully consumed
-    stage_tile<DH, ROPE>(Ks, qkv, row_base, ld, d + h * DH, k0, S, rope);
-    stage_tile<DH, false>(Vs, qkv, row_base, ld, 2 * d + h * DH, k0, S, rope);
-    __syncthreads();
+  for (int kt = 0; kt < n_kt; ++kt) {
+    const int k0 = kt * 64;
+    const bf16* Ks = KVs + (kt & 1) * 2 * 64 * LDS;
+    const bf16* Vs = Ks + 64 * LDS;
+    if (kt + 1 < n_kt) {                                        // prefetch the next K/V tile
+      bf16* nb = KVs + ((kt + 1) & 1) * 2 * 64 * LDS;
+      stage_tile_async<DH>(nb, qkv, row_base, ld, d + h * DH, k0 + 64, S);
+      stage_tile_async<DH>(nb + 64 * LDS, qkv, row_base, ld, 2 * d + h * DH, k0 + 64, S);
+      cp_commit();
+    }
     // scores S = Q K^T for 16 rows x 64 keys
     float sc[8][4];
 #pragma unroll
@@ -214,6 +200,8 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
         mma_bf16(o[2 * jp + 1], pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], b2, b3);
       }
     }
+    cp_wait<0>();                                               // next tile has landed ...
+    __syncthreads();                                            // ... and this one is fully consumed
   }
   // normalise and store
 #pragma unroll
@@ -233,14 +221,12 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
   }
 }
 
-template <int DH, bool ROPE>
-void launch_t(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp, int d, int H,
-              const float* rope) {
-  const size_t smem = (size_t)3 * 64 * (DH + 8) * sizeof(bf16);
-  cudaFuncSetAttribute(attention_mma_kernel<DH, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                       (int)smem);
+template <int DH>
+void launch_t(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp, int d, int H) {
+  const size_t smem = (size_t)5 * 64 * (DH + 8) * sizeof(bf16);
+  cudaFuncSetAttribute(attention_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid((S + 63) / 64, H, n * E);
-  attention_mma_kernel<DH, ROPE><<<grid, 128, smem, st>>>((const bf16*)qkv, (bf16*)ctx, E, S, Tp, d, rope);
+  attention_mma_kernel<DH><<<grid, 128, smem, st>>>((const bf16*)qkv, (bf16*)ctx, E, S, Tp, d);
 }
 
 }  // namespace
@@ -248,15 +234,10 @@ void launch_t(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, 
 bool attention_mma_supported(int dh) { return dh == 64 || dh == 128; }
 
 void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp,
-                          int d, int H, const float* rope) {
+                          int d, int H) {
   const int dh = d / H;
-  if (dh == 64) {
-    if (rope) launch_t<64, true>(st, qkv, ctx, n, E, S, Tp, d, H, rope);
-    else launch_t<64, false>(st, qkv, ctx, n, E, S, Tp, d, H, rope);
-  } else if (dh == 128) {
-    if (rope) launch_t<128, true>(st, qkv, ctx, n, E, S, Tp, d, H, rope);
-    else launch_t<128, false>(st, qkv, ctx, n, E, S, Tp, d, H, rope);
-  }
+  if (dh == 64) launch_t<64>(st, qkv, ctx, n, E, S, Tp, d, H);
+  else if (dh == 128) launch_t<128>(st, qkv, ctx, n, E, S, Tp, d, H);
 }
 
 }  // namespace zo

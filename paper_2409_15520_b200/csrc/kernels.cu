@@ -364,9 +364,42 @@ void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float t
   rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(tab, max_seq, dh / 2, (double)theta);
 }
 
+// In place on the q and k sections of the fused [rows, 3d] buffer.  Each thread rotates VEC
+// consecutive pairs (16-byte accesses).
 template <typename T>
 __global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S, int d, int H,
                             const float* __restrict__ tab) {
+  constexpr int VEC = 16 / sizeof(T);
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total) return;
+  const int half = d / H / 2;
+  const int vph = half / VEC;                         // vectors per half head
+  const int j = (int)(i % vph) * VEC;
+  long long rest = i / vph;
+  const int h = (int)(rest % H);
+  rest /= H;
+  const int which = (int)(rest % 2);                  // 0 = q, 1 = k
+  const long long row = rest / 2;
+  const int s = (int)((row % Tp) % S);
+  const float* cs = tab + (size_t)s * 2 * half + j;   // row s: cos[0..half) then sin[0..half)
+  T* p = qkv + (size_t)row * 3 * d + (size_t)which * d + h * 2 * half + j;
+  uint4 lo = *reinterpret_cast<const uint4*>(p), hi = *reinterpret_cast<const uint4*>(p + half);
+  T* e1 = reinterpret_cast<T*>(&lo);
+  T* e2 = reinterpret_cast<T*>(&hi);
+#pragma unroll
+  for (int k = 0; k < VEC; ++k) {
+    const float c = cs[k], sn = cs[half + k];
+    const float x1 = to_f(e1[k]), x2 = to_f(e2[k]);
+    e1[k] = from_f<T>(x1 * c - x2 * sn);
+    e2[k] = from_f<T>(x2 * c + x1 * sn);
+  }
+  *reinterpret_cast<uint4*>(p) = lo;
+  *reinterpret_cast<uint4*>(p + half) = hi;
+}
+// Scalar variant for head dimensions whose half is not a multiple of the vector width.
+template <typename T>
+__global__ void rope_scalar_kernel(T* __restrict__ qkv, long long total, int Tp, int S, int d, int H,
+                                   const float* __restrict__ tab) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
   const int half = d / H / 2;
@@ -374,7 +407,7 @@ __global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S,
   long long rest = i / half;
   const int h = (int)(rest % H);
   rest /= H;
-  const int which = (int)(rest % 2);  // 0 = q, 1 = k
+  const int which = (int)(rest % 2);
   const long long row = rest / 2;
   const int s = (int)((row % Tp) % S);
   const float c = tab[(size_t)s * 2 * half + j], sn = tab[(size_t)s * 2 * half + half + j];
@@ -383,15 +416,25 @@ __global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S,
   p[0] = from_f<T>(x1 * c - x2 * sn);
   p[half] = from_f<T>(x2 * c + x1 * sn);
 }
+template <typename T>
+static void rope_dispatch(cudaStream_t st, void* qkv, int rows, int Tp, int S, int d, int H,
+                          const float* tab) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int half = d / H / 2;
+  if (half % VEC == 0 && d % VEC == 0 && ((uintptr_t)qkv & 15) == 0) {
+    const long long total = (long long)rows * 2 * H * (half / VEC);
+    if (total > 0)
+      rope_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((T*)qkv, total, Tp, S, d, H, tab);
+  } else {
+    const long long total = (long long)rows * 2 * H * half;
+    if (total > 0)
+      rope_scalar_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((T*)qkv, total, Tp, S, d, H, tab);
+  }
+}
 void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, int d, int H,
                  const float* tab) {
-  const long long total = (long long)rows * 2 * H * (d / H / 2);
-  if (total <= 0) return;
-  const unsigned grid = (unsigned)((total + 255) / 256);
-  if (bf)
-    rope_kernel<bf16><<<grid, 256, 0, st>>>((bf16*)qkv, total, Tp, S, d, H, tab);
-  else
-    rope_kernel<float><<<grid, 256, 0, st>>>((float*)qkv, total, Tp, S, d, H, tab);
+  if (bf) rope_dispatch<bf16>(st, qkv, rows, Tp, S, d, H, tab);
+  else rope_dispatch<float>(st, qkv, rows, Tp, S, d, H, tab);
 }
 
 // =========================================================================================

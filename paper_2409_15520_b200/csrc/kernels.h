@@ -33,6 +33,7 @@ struct GemmDesc {
   int act;
   int swiglu;                   // 1: W = [gate rows | up rows] (N = 2 * d_ffn), out = silu(g)*u
   const LoraDesc* lora;         // null: plain GEMM
+  int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int single_cta;               // 1: one CTA per 128-row tile instead of CTA pairs on 256-row tiles
 };
 
@@ -54,11 +55,10 @@ void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, in
                  const float* tab);
 void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, int E,
                            int S, int Tp, int d, int H);
-// Tensor-core causal attention for bf16 with head_dim 64 or 128; applies the rotary embedding to
-// q and k on the fly when rope != null (table rows: cos[0..dh/2) | sin[0..dh/2)).
+// Tensor-core causal attention for bf16 with head_dim 64 or 128 (q, k already rotated).
 bool attention_mma_supported(int dh);
 void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp,
-                          int d, int H, const float* rope);
+                          int d, int H);
 void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows, int ffn);
 void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
                        int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status);

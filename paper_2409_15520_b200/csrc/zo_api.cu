@@ -133,7 +133,8 @@ Plan make_plan(const zo_config& c) {
 }  // namespace
 
 enum { PC_GEMM_TC = 0, PC_GEMM_SIMT, PC_ATTN, PC_NORM, PC_LORA_DOWN, PC_LORA_APPLY, PC_ROPE,
-       PC_SWIGLU, PC_LOSS, PC_UPDATE, PC_MISC, PC_COUNT };
+       PC_SWIGLU, PC_LOSS, PC_UPDATE, PC_MISC, PC_GEMM_QKV, PC_GEMM_O, PC_GEMM_FC1, PC_GEMM_FC2,
+       PC_GEMM_HEAD, PC_COUNT };
 static_assert(PC_COUNT == ZO_PROFILE_CLASSES, "profile classes out of sync with zo.h");
 
 struct ProfRec { int cat; double flops; cudaEvent_t e0, e1; };
@@ -192,7 +193,8 @@ zo_status fail(zo_ctx* c, zo_status s, const char* fmt, const char* a = "") {
 zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const GemmDesc& G,
                    uint32_t* status, int n_sms, int* launches, char* err, size_t errn) {
   const bool tcore = bf && !(flags & ZO_FLAG_SIMT_GEMM);
-  ProfScope ps(c, tcore ? PC_GEMM_TC : PC_GEMM_SIMT, 2.0 * G.M * (double)G.N * G.K);
+  ProfScope ps(c, tcore ? (G.prof_class ? G.prof_class : PC_GEMM_TC) : PC_GEMM_SIMT,
+               2.0 * G.M * (double)G.N * G.K);
   if (tcore) {
     GemmDesc Gt = G;
     Gt.single_cta = (flags & ZO_FLAG_GEMM_1CTA) ? 1 : 0;
@@ -328,6 +330,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     }
     GemmDesc G{};
     G.A = xn; G.lda = d; G.W = W.w_qkv; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
+    G.prof_class = PC_GEMM_QKV;
     if (first) {
       // first perturbed layer: one base product on the shared block, expanded to 2q outputs
       G.out = qkv0; G.ldo = 3 * d;
@@ -341,19 +344,19 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(G);
       if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
+    if (!opt) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
     if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
-      PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, E, S, Tp, d, H, opt ? nullptr : rope));
+      PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, E, S, Tp, d, H));
     } else {
-      if (!opt) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
       PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H));
     }
     GemmDesc O{};
     O.A = x; O.lda = d; O.W = W.w_o; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
-    O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0;
+    O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0; O.prof_class = PC_GEMM_O;
     GEMM(O);
     PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0));
     GemmDesc F1{};
-    F1.A = x; F1.lda = d; F1.W = W.w_fc1; F1.M = M; F1.K = d; F1.bias = W.b_fc1;
+    F1.A = x; F1.lda = d; F1.W = W.w_fc1; F1.M = M; F1.K = d; F1.bias = W.b_fc1; F1.prof_class = PC_GEMM_FC1;
     if (opt) {
       F1.N = f; F1.out = a; F1.ldo = f; F1.act = ACT_RELU;
       GEMM(F1);
@@ -367,7 +370,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     }
     GemmDesc F2{};
     F2.A = a; F2.lda = f; F2.W = W.w_fc2; F2.M = M; F2.N = d; F2.K = f; F2.out = h; F2.ldo = d;
-    F2.bias = W.b_fc2; F2.res = h; F2.ldr = d;
+    F2.bias = W.b_fc2; F2.res = h; F2.ldr = d; F2.prof_class = PC_GEMM_FC2;
     GEMM(F2);
   }
 
@@ -380,7 +383,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     float* logits = c->at<float>(c->plan.logits);
     GemmDesc Hd{};
     Hd.A = xh; Hd.lda = d; Hd.W = head; Hd.M = Mh; Hd.N = cf.vocab; Hd.K = d;
-    Hd.out = logits; Hd.ldo = cf.vocab; Hd.out_f32 = 1;
+    Hd.out = logits; Hd.ldo = cf.vocab; Hd.out_f32 = 1; Hd.prof_class = PC_GEMM_HEAD;
     GEMM(Hd);
     PROF(PC_LOSS, 0.0, launch_ce_rows(st, logits, cf.vocab, cf.vocab, lab_val, EP, Mh, rowloss));
   } else {
