@@ -154,12 +154,18 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the depth (profiling captures of a small case)")
     ap.add_argument("--q", type=int, default=0, help="override q (profiling captures of a small case)")
     ap.add_argument("--flags", type=int, default=0, help="zo_config.flags (diagnostic kernel switches)")
+    ap.add_argument("--targets", type=int, default=-1, help="override lora_targets (0 = no adapted projection)")
+    ap.add_argument("--rank", type=int, default=0, help="override the LoRA rank")
     args = ap.parse_args()
     spec = config(args.workload)
     if args.layers:
         spec = spec.with_(n_layers=args.layers)
     if args.q:
         spec = spec.with_(q=args.q)
+    if args.targets >= 0:
+        spec = spec.with_(lora_targets=args.targets)
+    if args.rank:
+        spec = spec.with_(lora_rank=args.rank)
     if args.impl == "reference":
         return run_reference(args, spec)
 
