@@ -76,6 +76,22 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(values, device):
+    """Slowest rank's figure for each entry of `values` (the job is N independent replicas of the
+    step, so whole-job throughput = N * units per step / the slowest rank's time)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(world, units_per_step, steps, ms):
+    return world * units_per_step * steps / (ms * 1e-3)
+
+
 def load_problem(spec, seed=1234, b_std=0.01):
     """Synthetic weights on the device, one decoder block in host memory at a time."""
     import paper_2409_15520_b200 as zo
@@ -227,10 +243,7 @@ def main():
         prob.host_labels.numel() * prob.host_labels.element_size()
     d2h = (2 * q + q) * 4 + 4
 
-    if world > 1:
-        t = torch.tensor([ms, ms_e2e], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = t.tolist()
+    ms, ms_e2e = max_over_ranks([ms, ms_e2e], "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -244,7 +257,7 @@ def main():
     peak = peaks["tflops_sustained"] if inside_long_step else peaks["tflops"]
     total_prof = sum(v[0] for v in prof.values())
     line = {
-        "metric": METRIC, "value": world * tokens_per_step * args.steps / (ms * 1e-3), "unit": UNIT,
+        "metric": METRIC, "value": whole_job_value(world, tokens_per_step, args.steps, ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if spec.bf16 else "f32", "data": "synthetic",
@@ -257,7 +270,7 @@ def main():
         "zo_steps_per_s": world * args.steps / (ms * 1e-3),
         "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,
         "clocks": clocks,
-        "e2e": {"value": world * tokens_per_step * args.steps / (ms_e2e * 1e-3), "unit": UNIT,
+        "e2e": {"value": whole_job_value(world, tokens_per_step, args.steps, ms_e2e), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tflops, "peak": peak,
