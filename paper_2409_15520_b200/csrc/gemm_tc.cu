@@ -240,6 +240,26 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
   tm = gm0 + (r - tn * gsz);
 }
 
+// Columns of perturbed B staged per generation phase: as many as fit the 16 KiB staging area,
+// a multiple of 32, at most one tile.
+__device__ __forceinline__ int lora_phase_cols(int r) {
+  const int g = ((int)(2 * LORA_BUF_FLOATS) / r) & ~31;
+  return g > 256 ? 256 : g;
+}
+// Up to 16 consecutive floats of a U row (zero-padded), issued back to back.
+__device__ __forceinline__ void load_u16(const float* p, int left, bool vec, float (&u)[16]) {
+  if (vec && left >= 16) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float4 t = reinterpret_cast<const float4*>(p)[i];
+      u[4 * i] = t.x; u[4 * i + 1] = t.y; u[4 * i + 2] = t.z; u[4 * i + 3] = t.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) u[i] = i < left ? p[i] : 0.f;
+  }
+}
+
 template <bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -401,11 +421,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int rep = P.has_lora ? m0 / P.L.rows_per_replica : 0;
       const float sgn = (rep & 1) ? -P.L.eps : P.L.eps;
       const float* urow = P.has_lora ? P.L.U + (size_t)min(row, P.M - 1) * P.L.ldu : nullptr;
+      const bool u_vec = P.has_lora && (P.L.ldu % 4 == 0) && (P.L.r % 4 == 0) && (((uintptr_t)P.L.U & 15) == 0);
       const int nchunk = ncol_tile / 32;
-      uint32_t lc = 0;                             // LoRA chunks so far: picks the staging buffer
+      // The perturbed B columns are staged G columns at a time (the whole 256-column tile for
+      // rank <= 16): one generation phase, two barriers, then barrier-free chunks.
+      const int G = P.has_lora ? lora_phase_cols(P.L.r) : 256;
+      const int cpp = G / 32;                      // chunks per generation phase
       for (int c = 0; c < nchunk; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= P.N) break;
+        int lslot = -1;
+        float u[16];
+        if (P.has_lora && !P.swiglu) {
+          if (c % cpp == 0) {
+            bool any = false;
+            for (int cc = c; cc < c + cpp && cc < nchunk; ++cc) {
+              const int col = n0 + cc * 32;
+              any = any || (col < P.N && P.L.slot_of_sec[col / P.L.width] >= 0);
+            }
+            if (any) {                             // uniform over the CTA
+              ep_bar();                            // everyone is done with the previous phase
+              const int g4 = G / 4;
+              for (int idx = et; idx < P.L.r * g4; idx += 128) {
+                const int k = idx / g4, c4 = (idx - k * g4) * 4;
+                const int col = col0 + c4;
+                float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (col < P.N) {
+                  const int sec = col / P.L.width;
+                  const int slot = P.L.slot_of_sec[sec];
+                  if (slot >= 0) {
+                    const size_t e = (size_t)k * P.L.width + (col - sec * P.L.width);
+                    b = *reinterpret_cast<const float4*>(P.L.B + (size_t)slot * P.L.r * P.L.width + e);
+                    if (P.L.eps != 0.f) {
+                      const float4 z = z_block(P.L.seed, P.L.tensor_base + slot, (uint32_t)(rep >> 1),
+                                               (uint32_t)(e >> 2));
+                      b.x = fmaf(sgn, z.x, b.x); b.y = fmaf(sgn, z.y, b.y);
+                      b.z = fmaf(sgn, z.z, b.z); b.w = fmaf(sgn, z.w, b.w);
+                    }
+                    b.x *= P.L.scale; b.y *= P.L.scale; b.z *= P.L.scale; b.w *= P.L.scale;
+                  }
+                }
+                *reinterpret_cast<float4*>(lbuf + k * G + c4) = b;
+              }
+              ep_bar();
+            }
+          }
+          lslot = P.L.slot_of_sec[col0 / P.L.width];
+          if (lslot >= 0) load_u16(urow + lslot * P.L.r, P.L.r, u_vec, u);
+        }
         uint32_t v[32];
         tc_ld32(taddr + c * 32, v);
         float f[32];
@@ -426,38 +489,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) f[j] = __uint_as_float(v[j]);
-          if (P.has_lora) {
-            const int sec = col0 / P.L.width;
-            const int slot = P.L.slot_of_sec[sec];
-            if (slot >= 0) {                       // uniform over the CTA
-              float* lb = lbuf + (lc++ & 1u) * LORA_BUF_FLOATS;
-              const int cs = col0 - sec * P.L.width;
-              const float* Bm = P.L.B + (size_t)slot * P.L.r * P.L.width;
-              for (int idx = et; idx < P.L.r * 8; idx += 128) {
-                const int k = idx >> 3, c4 = (idx & 7) * 4;
-                const size_t e = (size_t)k * P.L.width + cs + c4;
-                float4 b = *reinterpret_cast<const float4*>(Bm + e);
-                if (P.L.eps != 0.f) {
-                  const float4 z = z_block(P.L.seed, P.L.tensor_base + slot, (uint32_t)(rep >> 1),
-                                           (uint32_t)(e >> 2));
-                  b.x = fmaf(sgn, z.x, b.x); b.y = fmaf(sgn, z.y, b.y);
-                  b.z = fmaf(sgn, z.z, b.z); b.w = fmaf(sgn, z.w, b.w);
-                }
-                b.x *= P.L.scale; b.y *= P.L.scale; b.z *= P.L.scale; b.w *= P.L.scale;
-                *reinterpret_cast<float4*>(lb + k * 32 + c4) = b;
-              }
-              ep_bar();
-              const float* up = urow + slot * P.L.r;
-              for (int k = 0; k < P.L.r; ++k) {
-                const float u = up[k];
-                const float4* b4 = reinterpret_cast<const float4*>(lb + k * 32);
+          if (lslot >= 0) {
+            // f += U[row, :] * (s (B + k eps z))[:, chunk]; 16 rank indices at a time, the first 16
+            // values of U were requested before the accumulator load
+            const float* lb = lbuf + (c % cpp) * 32;
+            for (int kb = 0; kb < P.L.r; kb += 16) {
+              if (kb) load_u16(urow + lslot * P.L.r + kb, P.L.r - kb, u_vec, u);
 #pragma unroll
-                for (int j4 = 0; j4 < 8; ++j4) {
-                  const float4 b = b4[j4];
-                  f[4 * j4 + 0] = fmaf(u, b.x, f[4 * j4 + 0]);
-                  f[4 * j4 + 1] = fmaf(u, b.y, f[4 * j4 + 1]);
-                  f[4 * j4 + 2] = fmaf(u, b.z, f[4 * j4 + 2]);
-                  f[4 * j4 + 3] = fmaf(u, b.w, f[4 * j4 + 3]);
+              for (int i = 0; i < 16; ++i) {
+                if (kb + i < P.L.r) {
+                  const float4* b4 = reinterpret_cast<const float4*>(lb + (kb + i) * G);
+#pragma unroll
+                  for (int j4 = 0; j4 < 8; ++j4) {
+                    const float4 b = b4[j4];
+                    f[4 * j4 + 0] = fmaf(u[i], b.x, f[4 * j4 + 0]);
+                    f[4 * j4 + 1] = fmaf(u[i], b.y, f[4 * j4 + 1]);
+                    f[4 * j4 + 2] = fmaf(u[i], b.z, f[4 * j4 + 2]);
+                    f[4 * j4 + 3] = fmaf(u[i], b.w, f[4 * j4 + 3]);
+                  }
                 }
               }
             }

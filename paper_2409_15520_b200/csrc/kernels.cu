@@ -814,7 +814,8 @@ __global__ void zo_update_kernel(UpdateDesc D, const double* __restrict__ losses
 void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g) {
   const long long blks = (D.elems_per_slot + 3) / 4;
-  dim3 grid((unsigned)((blks + 127) / 128), D.n_slots, D.count);
+  // a model without adapted projections still gets its g[] written by one (idle) block
+  dim3 grid((unsigned)(blks > 0 ? (blks + 127) / 128 : 1), D.n_slots > 0 ? D.n_slots : 1, D.count > 0 ? D.count : 1);
   zo_update_kernel<<<grid, 128, 0, st>>>(D, losses, g, q, eps, lr, seed, status, write_g);
 }
 
