@@ -4,7 +4,7 @@
 //     4-deep shared-memory ring, one elected thread issues tcgen05.mma (128 x 256 x 16 per
 //     instruction), fp32 accumulators live in tensor memory, two accumulator buffers so the
 //     epilogue of tile i overlaps the main loop of tile i+1; persistent CTAs, one per SM.
-//   * epilogue (4 warps, tcgen05.ld): bias, ReLU, residual add, SiLU(gate)*up, float or
+//   * epilogue (8 warps, two per tensor-memory lane quarter, tcgen05.ld): bias, ReLU, residual add, SiLU(gate)*up, float or
 //     bfloat16 output, and the MP-LoRA term of the paper's layer equation
 //         Y_n = X_n W + s * U_n (B + k_n eps z_i)
 //     with z_i regenerated from the Philox seed inside the epilogue (never in HBM).  Every
@@ -40,7 +40,9 @@ constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;     // clears the CTA-rank bit of a 
 constexpr int LORA_MAXR = 64;
 constexpr uint32_t LORA_BUF_FLOATS = LORA_MAXR * 32;  // one 32-column chunk of s*(B + k eps z)
 constexpr uint32_t TMEM_COLS = 512;
-constexpr int THREADS = 192;                    // warp 0: TMA, warp 1: MMA, warps 2-5: epilogue
+constexpr int EP_WARPS = 8;                     // two per tensor-memory lane quarter, alternating chunks
+constexpr int EP_THREADS = EP_WARPS * 32;
+constexpr int THREADS = 64 + EP_THREADS;        // warp 0: TMA, warp 1: MMA, warps 2-9: epilogue
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct Ctrl {
@@ -196,7 +198,7 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 __device__ __forceinline__ void tc_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void ep_bar() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void ep_bar() { asm volatile("bar.sync 1, %0;" ::"n"(EP_THREADS) : "memory"); }
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 B apart.
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
@@ -291,7 +293,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctrl->tfull[a]), 1);
-      mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 8 : 4);
+      mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 2 * EP_WARPS : EP_WARPS);
     }
     mbar_init(smem_u32(&ctrl->drain), 1);
     ctrl->abort = 0u;
@@ -398,7 +400,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else {
     // ------------------------------------------------------------------ epilogue warps
     const int wq = warp & 3;                       // tensor-memory lane quarter of this warp
-    const int et = threadIdx.x - 64;               // 0..127
+    const int et = threadIdx.x - 64;               // 0..EP_THREADS-1
+    const int half = (warp - 2) >> 2;              // which of the quarter's two warps: even or odd chunks
     const bool out_vec_ok = ((uintptr_t)P.out & 15) == 0 && (P.ldo % (P.out_f32 ? 4 : 8)) == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
     uint32_t titer = 0;
@@ -442,7 +445,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (any) {                             // uniform over the CTA
               ep_bar();                            // everyone is done with the previous phase
               const int g4 = G / 4;
-              for (int idx = et; idx < P.L.r * g4; idx += 128) {
+              for (int idx = et; idx < P.L.r * g4; idx += EP_THREADS) {
                 const int k = idx / g4, c4 = (idx - k * g4) * 4;
                 const int col = col0 + c4;
                 float4 b = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -466,8 +469,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               ep_bar();
             }
           }
+          if ((c & 1) != half) continue;           // the sibling warp's chunk
           lslot = P.L.slot_of_sec[col0 / P.L.width];
           if (lslot >= 0) load_u16(urow + lslot * P.L.r, P.L.r, u_vec, u);
+        } else if ((c & 1) != half) {
+          continue;
         }
         uint32_t v[32];
         tc_ld32(taddr + c * 32, v);
