@@ -17,6 +17,7 @@ pytestmark = pytest.mark.gpu
 
 SIMT = 1  # ZO_FLAG_SIMT_GEMM
 ONE_CTA = 2  # ZO_FLAG_GEMM_1CTA
+NO_PF = 4  # ZO_FLAG_GEMM_NO_L2_PREFETCH
 
 
 def test_perturbation_words_bit_exact_and_normals_close():
@@ -86,7 +87,7 @@ def test_decoder_fp32_head_dims_and_ragged_sequence():
         _check_fp32(spec, seed=4, b_std=0.05)
 
 
-@pytest.mark.parametrize("flags", [SIMT, 0, ONE_CTA])
+@pytest.mark.parametrize("flags", [SIMT, 0, ONE_CTA, NO_PF, ONE_CTA | NO_PF])
 @pytest.mark.parametrize("arch", [ARCH_OPT, ARCH_LLAMA])
 def test_decoder_bf16(arch, flags):
     """bf16 storage; flags=SIMT runs the validation GEMM, 0 the tensor-core path.
