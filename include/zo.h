@@ -70,12 +70,9 @@ enum { ZO_TARGET_Q = 1, ZO_TARGET_K = 2, ZO_TARGET_V = 4 };
 /* flags: ZO_FLAG_SIMT_GEMM routes every bf16 GEMM (and attention) through the plain
  * CUDA-core validation kernels instead of the tensor-core ones (cross-checking only). */
 enum { ZO_FLAG_SIMT_GEMM = 1,
-       /* ZO_FLAG_GEMM_1CTA: tensor-core GEMMs run one CTA per 128-row tile instead of the default
-        * CTA pairs on 256-row tiles (diagnostic A/B switch; same results up to rounding order). */
-       ZO_FLAG_GEMM_1CTA = 2,
-       /* ZO_FLAG_GEMM_NO_L2_PREFETCH: the tensor-core GEMM's producer does not warm L2 ahead of its
-        * loads (diagnostic A/B switch; identical results). */
-       ZO_FLAG_GEMM_NO_L2_PREFETCH = 4 };
+       /* ZO_FLAG_GEMM_PAIR: tensor-core GEMMs run CTA pairs (tcgen05 cta_group::2) on 256-row
+        * tiles instead of the default one CTA per 128-row tile (A/B switch; bit-identical results). */
+       ZO_FLAG_GEMM_PAIR = 2 };
 
 typedef struct zo_ctx zo_ctx; /* opaque; owned by the library; released by zo_free */
 

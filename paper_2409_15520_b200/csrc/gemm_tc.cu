@@ -10,7 +10,8 @@
 //     with z_i regenerated from the Philox seed inside the epilogue (never in HBM).  Every
 //     128-row tile lies inside one replica, so the perturbed B columns of the tile are built
 //     once in shared memory and reused by its 128 rows.
-//   * PAIR variant (default): two CTAs of a cluster work on one 256 x 256 tile with
+//   * PAIR variant (opt-in; measured slower under the 1 kW power cap than one CTA per tile, see
+//     the design notes): two CTAs of a cluster work on one 256 x 256 tile with
 //     tcgen05.mma.cta_group::2 - each CTA stages its own 128 rows of A and its 128-row half of
 //     the weight tile, so the shared-memory traffic per SM drops by a third; 6 stages.  The
 //     leader CTA issues the MMAs and releases stages/accumulators in both CTAs with multicast
@@ -59,7 +60,6 @@ struct Params {
   const bf16* bias;
   const bf16* res; int ldr; int res_mod;
   int act, swiglu;
-  int l2_ahead;             // k-blocks the L2 prefetch runs ahead of the TMA loads (0 = off)
   int has_lora;
   LoraDesc L;
   uint32_t* status;
@@ -147,11 +147,6 @@ __device__ __forceinline__ uint32_t cluster_rank() {
 }
 __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// Warm L2 with a box that a later TMA load will fetch (no shared memory, no completion to wait for).
-__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int x, int y) {
-  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(map), "r"(x), "r"(y)
-               : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -333,32 +328,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       uint32_t issued = 0;
       bool ok = true;
-      // L2 prefetch cursor: runs L2_AHEAD k-blocks ahead of the loads (across tile boundaries), so
-      // that a panel nobody has touched yet comes from DRAM well before the ring needs it; the
-      // ring itself (4-6 stages, ~0.4 us each) only covers an L2 hit.
-      int pf_tile = unit, pf_kb = 0, pf_m0 = 0, pf_b0 = 0, pf_b1 = 0;
-      bool pf_live = P.l2_ahead > 0 && pf_tile < num_tiles;
-      auto pf_coords = [&]() {
-        int tm, tn;
-        tile_coords(pf_tile, tiles_m, tiles_n, GROUP_M, tm, tn);
-        pf_m0 = tm * TILE_M + (int)rank * BM;
-        pf_b0 = tn * ncol_tile;
-        pf_b1 = P.swiglu ? P.N + pf_b0 : pf_b0 + 128;
-      };
-      auto pf_step = [&]() {
-        if (!pf_live) return;
-        tma_prefetch_2d(&tmA, pf_kb * BK, pf_m0);
-        if (!PAIR || rank == 0) tma_prefetch_2d(&tmB, pf_kb * BK, pf_b0);
-        if (!PAIR || rank == 1) tma_prefetch_2d(&tmB, pf_kb * BK, pf_b1);
-        if (++pf_kb == num_kb) {
-          pf_kb = 0;
-          pf_tile += n_units;
-          pf_live = pf_tile < num_tiles;
-          if (pf_live) pf_coords();
-        }
-      };
-      if (pf_live) pf_coords();
-      for (int i = 0; i < P.l2_ahead; ++i) pf_step();
       for (int tile = unit; tile < num_tiles && ok; tile += n_units) {
         int tm, tn;
         tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
@@ -366,7 +335,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int brow0 = tn * ncol_tile;
         const int brow1 = P.swiglu ? P.N + brow0 : brow0 + 128;
         for (int kb = 0; kb < num_kb; ++kb, ++issued) {
-          pf_step();
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
@@ -690,12 +658,11 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.bias = (const bf16*)G.bias;
   P.res = (const bf16*)G.res; P.ldr = G.ldr; P.res_mod = G.res_mod;
   P.act = G.act; P.swiglu = G.swiglu;
-  P.l2_ahead = G.no_l2_prefetch ? 0 : 8;
   P.has_lora = G.lora ? 1 : 0;
   if (G.lora) P.L = *G.lora; else P.L = LoraDesc{};
   P.status = status;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
-  if (!G.single_cta && P.M > tc::BM) {
+  if (G.cta_pair && P.M > tc::BM) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
     static int max_clusters = 0;                       // co-resident pairs on this device
     cudaLaunchConfig_t cfg = {};

@@ -34,8 +34,7 @@ struct GemmDesc {
   int swiglu;                   // 1: W = [gate rows | up rows] (N = 2 * d_ffn), out = silu(g)*u
   const LoraDesc* lora;         // null: plain GEMM
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
-  int no_l2_prefetch;           // 1: do not warm L2 ahead of the TMA loads (diagnostic)
-  int single_cta;               // 1: one CTA per 128-row tile instead of CTA pairs on 256-row tiles
+  int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
 };
 
 // --- elementwise / reduction kernels (bf = 1: bfloat16 tensors, 0: float) -------------------

@@ -197,8 +197,7 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
                2.0 * G.M * (double)G.N * G.K);
   if (tcore) {
     GemmDesc Gt = G;
-    Gt.single_cta = (flags & ZO_FLAG_GEMM_1CTA) ? 1 : 0;
-    Gt.no_l2_prefetch = (flags & ZO_FLAG_GEMM_NO_L2_PREFETCH) ? 1 : 0;
+    Gt.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
     const int e = launch_gemm_tc(st, Gt, status, n_sms);
     if (e) {
       snprintf(err, errn, "tensor-core GEMM launch failed (code %d: %s)", e,
@@ -220,8 +219,7 @@ zo_status run_lora_down(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, cons
   if (bf && !(flags & ZO_FLAG_SIMT_GEMM) && K % 8 == 0 && ldx % 8 == 0) {
     GemmDesc G{};
     G.A = X; G.lda = ldx; G.W = A; G.M = rows; G.N = J; G.K = K; G.out = U; G.ldo = J; G.out_f32 = 1;
-    G.single_cta = (flags & ZO_FLAG_GEMM_1CTA) ? 1 : 0;
-    G.no_l2_prefetch = (flags & ZO_FLAG_GEMM_NO_L2_PREFETCH) ? 1 : 0;
+    G.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
     ProfScope ps(c, PC_LORA_DOWN, 2.0 * rows * (double)J * K);
     const int e = launch_gemm_tc(st, G, status, n_sms);
     if (e) {

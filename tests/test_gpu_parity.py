@@ -16,8 +16,7 @@ from gpu_util import make_problem, old_B, run_gpu, run_oracle, update_rel_err
 pytestmark = pytest.mark.gpu
 
 SIMT = 1  # ZO_FLAG_SIMT_GEMM
-ONE_CTA = 2  # ZO_FLAG_GEMM_1CTA
-NO_PF = 4  # ZO_FLAG_GEMM_NO_L2_PREFETCH
+PAIR = 2  # ZO_FLAG_GEMM_PAIR
 
 
 def test_perturbation_words_bit_exact_and_normals_close():
@@ -87,7 +86,7 @@ def test_decoder_fp32_head_dims_and_ragged_sequence():
         _check_fp32(spec, seed=4, b_std=0.05)
 
 
-@pytest.mark.parametrize("flags", [SIMT, 0, ONE_CTA, NO_PF, ONE_CTA | NO_PF])
+@pytest.mark.parametrize("flags", [SIMT, 0, PAIR])
 @pytest.mark.parametrize("arch", [ARCH_OPT, ARCH_LLAMA])
 def test_decoder_bf16(arch, flags):
     """bf16 storage; flags=SIMT runs the validation GEMM, 0 the tensor-core path.
@@ -111,10 +110,10 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
     ref = run_oracle(spec, p, tok, lab, 31)
     got = run_gpu(spec, p, 31)
     simt = run_gpu(spec, p, 31, flags=SIMT)
-    one = run_gpu(spec, p, 31, flags=ONE_CTA)
+    pair = run_gpu(spec, p, 31, flags=PAIR)
     assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
     # CTA-pair and single-CTA tensor-core kernels accumulate in the same order: bit-identical
-    assert np.array_equal(got["losses"], one["losses"]) and np.array_equal(got["rows"], one["rows"])
+    assert np.array_equal(got["losses"], pair["losses"]) and np.array_equal(got["rows"], pair["rows"])
     # the two bf16 GEMM implementations agree far more closely with each other
     assert np.allclose(got["losses"], simt["losses"], rtol=2e-3, atol=0), (got["losses"], simt["losses"])
     assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
@@ -161,13 +160,13 @@ def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
     dev = lambda a: torch.tensor(a, device="cuda").to(torch.bfloat16).contiguous()
     Bd = torch.tensor(B, device="cuda")
     outs = {}
-    for flags in (0, SIMT, ONE_CTA):
+    for flags in (0, SIMT, PAIR):
         Y = zo.mp_lora_linear(dev(X.reshape(-1, ki)), dev(W), dev(bias), dev(A), Bd, T, q, scale, seed,
                               tid, eps, x_replicated, flags=flags)
         outs[flags] = Y.float().cpu().numpy().astype(np.float64)
         err = np.max(np.abs(outs[flags] - ref))
         assert err < 2e-2 * np.max(np.abs(ref)), (flags, err, np.max(np.abs(ref)))
-    assert np.array_equal(outs[0], outs[ONE_CTA])
+    assert np.array_equal(outs[0], outs[PAIR])
     # the perturbation must be visible in the outputs: replicas 0 and 1 differ as the oracle's do
     d_gpu, d_ref = outs[0][0] - outs[0][1], ref[0] - ref[1]
     assert np.max(np.abs(d_ref)) > 0
