@@ -135,6 +135,54 @@ def oracle_sample(spec, seed=1234):
     return dt, 2 * small.S, spec.n_layers / L, f"q=1, 1 sequence of {small.S} tokens, {L} of {spec.n_layers} blocks (time scaled by depth)"
 
 
+def run_sweep(args):
+    """MP-LoRA linear micro-benchmark (d_in = d_out = 4096, 4096 tokens, rank x q grid): one JSON line per
+    point with the shared-input form (one base GEMM amortised over the 2q replicas, then the expand
+    kernel: bound by writing 2q*T*k outputs) and the replicated-input form (one GEMM over 2q*T rows with
+    the low-rank term in its epilogue: bound by the tensor pipe)."""
+    import torch
+    import paper_2409_15520_b200 as zo
+    peaks = _peaks()
+    T = k = 4096
+    dev = "cuda"
+    g = torch.Generator(device=dev).manual_seed(1234)
+    W = (0.02 * torch.randn(k, k, device=dev, generator=g)).to(torch.bfloat16)
+    bias = (0.02 * torch.randn(k, device=dev, generator=g)).to(torch.bfloat16)
+    ranks = [args.rank] if args.rank else [8, 16, 64]
+    qs = [args.q] if args.q else [1, 2, 4, 8, 16, 32]
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    for r in ranks:
+        A = (0.02 * torch.randn(r, k, device=dev, generator=g)).to(torch.bfloat16)
+        B = 0.01 * torch.randn(r, k, device=dev, generator=g)
+        for q in qs:
+            n = 2 * q
+            X = torch.randn(n * T, k, device=dev, generator=g).to(torch.bfloat16)
+            Y = torch.empty(n, T, k, device=dev, dtype=torch.bfloat16)
+            out = {"r": r, "q": q, "replicas": n}
+            for mode, x_rep in (("shared_input", 0), ("replicated_input", 1)):
+                call = lambda: zo.mp_lora_linear(X, W, bias, A, B, T, q, 1.0, 7, 0, 1e-3, x_rep,
+                                                 flags=args.flags, out=Y, sync=False)
+                for _ in range(3):
+                    call()
+                torch.cuda.synchronize()
+                e0, e1 = ev(), ev()
+                reps = max(3, min(20, 64 // n))
+                e0.record()
+                for _ in range(reps):
+                    call()
+                e1.record()
+                torch.cuda.synchronize()
+                ms = e0.elapsed_time(e1) / reps
+                flops = 2.0 * (n if x_rep else 1) * T * k * k
+                out[mode] = {"ms": round(ms, 4), "gemm_tflops": round(flops / (ms * 1e-3) / 1e12, 1),
+                             "frac_of_bf16_peak": round(flops / (ms * 1e-3) / 1e12 / peaks["tflops"], 3),
+                             "out_gbs": round(n * T * k * 2 / (ms * 1e-3) / 1e9, 1),
+                             "frac_of_hbm_peak": round(n * T * k * 2 / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], 3),
+                             "tokens_per_s": round(n * T / (ms * 1e-3))}
+            out["replicated_over_shared_time"] = round(out["replicated_input"]["ms"] / out["shared_input"]["ms"], 2)
+            print(json.dumps(out), flush=True)
+
+
 def run_reference(args, spec):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -172,12 +220,23 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="zo_config.flags (diagnostic kernel switches)")
     ap.add_argument("--targets", type=int, default=-1, help="override lora_targets (0 = no adapted projection)")
     ap.add_argument("--rank", type=int, default=0, help="override the LoRA rank")
+    ap.add_argument("--sweep", action="store_true", help="MP-LoRA linear micro-benchmark grid (rank x q)")
+    ap.add_argument("--schedule", default="full", choices=["full", "outer_only", "inner_only", "sequential"],
+                    help="how the step is cut into forward passes (the paper's ablation)")
+    ap.add_argument("--E", type=int, default=0, help="override the number of sequences")
+    ap.add_argument("--S", type=int, default=0, help="override the sequence length")
     args = ap.parse_args()
+    if args.sweep:
+        return run_sweep(args)
     spec = config(args.workload)
     if args.layers:
         spec = spec.with_(n_layers=args.layers)
     if args.q:
         spec = spec.with_(q=args.q)
+    if args.E:
+        spec = spec.with_(E=args.E)
+    if args.S:
+        spec = spec.with_(S=args.S, n_labelled=min(spec.n_labelled, args.S - 1))
     if args.targets >= 0:
         spec = spec.with_(lora_targets=args.targets)
     if args.rank:
@@ -199,6 +258,7 @@ def main():
 
     prob = load_problem(spec)
     est = zo.Estimator(zo.make_config(spec, flags=args.flags))
+    est.set_schedule(args.schedule)
     E, S, q, eps, lr = spec.E, spec.S, spec.q, spec.eps, spec.lr
     tokens_per_step = 2 * q * E * S
 
@@ -266,6 +326,7 @@ def main():
                    "lora_rank": spec.lora_rank, "q": q, "E": E, "S": S, "replicas": 2 * q,
                    "token_rows_per_step": tokens_per_step, "eps": eps, "lr": lr,
                    "l2": "inputs larger than L2 (weights and activations of several GB stream every step)",
+                   "schedule": args.schedule,
                    "parallelism": "replicas only" if world > 1 else "1 gpu"},
         "zo_steps_per_s": world * args.steps / (ms * 1e-3),
         "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,

@@ -179,6 +179,18 @@ ZO_API zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g);
  * ZO_ARCH_LINEAR: one value per token row (mean over k_out).  Synchronises the stream. */
 ZO_API zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows);
 
+/* How a step is cut into forward passes (the paper's ablation of its two parallelisations; the
+ * results of a step do not depend on it, only its cost does):
+ *   ZO_SCHEDULE_FULL        one pass over all 2q replicas (outer and inner loop in parallel; default)
+ *   ZO_SCHEDULE_OUTER_ONLY  two passes of q replicas: every +eps path, then every -eps path
+ *   ZO_SCHEDULE_INNER_ONLY  q passes of 2 replicas: the +/- pair of one query at a time
+ *   ZO_SCHEDULE_SEQUENTIAL  2q passes of one replica: the order of forward passes of sequential
+ *                           MeZO with LoRA-FA (appendix "MeZO with q>1"), without its in-place
+ *                           parameter sweeps since the perturbed copy is formed on the fly. */
+enum { ZO_SCHEDULE_FULL = 0, ZO_SCHEDULE_OUTER_ONLY = 1, ZO_SCHEDULE_INNER_ONLY = 2,
+       ZO_SCHEDULE_SEQUENTIAL = 3 };
+ZO_API zo_status zo_set_schedule(zo_ctx* ctx, int32_t schedule);
+
 /* Number of kernels the last zo_step enqueued. */
 ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 

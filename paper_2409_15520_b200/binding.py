@@ -74,6 +74,8 @@ zo_step_host = _sig("zo_step_host", C.c_int, _STEP_ARGS)
 zo_losses = _sig("zo_losses", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p])
 zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)])
 zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
+zo_set_schedule = _sig("zo_set_schedule", C.c_int, [C.c_void_p, C.c_int32])
+SCHEDULES = {"full": 0, "outer_only": 1, "inner_only": 2, "sequential": 3}
 zo_free = _sig("zo_free", None, [C.c_void_p])
 zo_profile_enable = _sig("zo_profile_enable", C.c_int, [C.c_void_p, C.c_int32])
 zo_profile_read = _sig("zo_profile_read", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p])
@@ -229,6 +231,9 @@ class Estimator:
         self._check(zo_row_losses(self._h, out.ctypes.data_as(C.c_void_p), C.byref(n)))
         return out
 
+    def set_schedule(self, name):
+        self._check(zo_set_schedule(self._h, SCHEDULES[name]))
+
     def profile_enable(self, on=True):
         self._check(zo_profile_enable(self._h, int(on)))
 
@@ -267,24 +272,35 @@ def perturbation(seed, tensor_id, query, n, device="cuda"):
     return u.cpu().numpy().view(np.uint32), z.cpu().numpy()
 
 
-def mp_lora_linear(X, W, bias, A, B, T, q, scale, seed, tensor_id, eps, x_replicated, flags=0):
-    """Y [2q, T, k_out] = MP-LoRA linear of torch device tensors (float32 or bfloat16)."""
+_SCRATCH = {}
+
+
+def mp_lora_linear(X, W, bias, A, B, T, q, scale, seed, tensor_id, eps, x_replicated, flags=0,
+                   out=None, sync=True):
+    """Y [2q, T, k_out] = MP-LoRA linear of torch device tensors (float32 or bfloat16).  With
+    sync=False the call only enqueues (scratch is cached per size; the device status word is
+    not read back)."""
     bf = X.dtype == torch.bfloat16
     k_out, k_in = W.shape
     r = A.shape[0]
-    Y = torch.empty((2 * q, T, k_out), dtype=X.dtype, device=X.device)
+    Y = torch.empty((2 * q, T, k_out), dtype=X.dtype, device=X.device) if out is None else out
     nb = zo_mp_lora_scratch_bytes(int(bf), T, k_in, k_out, r, q, int(x_replicated))
-    scratch = torch.empty(nb + 256, dtype=torch.uint8, device=X.device)
+    key = (X.device, nb)
+    if key not in _SCRATCH:
+        _SCRATCH.clear()
+        _SCRATCH[key] = torch.empty(nb + 256, dtype=torch.uint8, device=X.device)
+    scratch = _SCRATCH[key]
     base = (scratch.data_ptr() + 255) // 256 * 256
     st = zo_mp_lora_linear(C.c_void_p(torch.cuda.current_stream().cuda_stream), int(bf), _ptr(X),
                            _ptr(W), _ptr(bias), _ptr(A), _ptr(B), _ptr(Y), T, k_in, k_out, r, scale,
                            seed, tensor_id, q, eps, int(x_replicated), C.c_void_p(base), nb, flags)
     if st:
         raise ZoError(st)
-    torch.cuda.synchronize()
-    status = int(scratch.view(torch.int32)[(base - scratch.data_ptr()) // 4].item())
-    if status:
-        raise ZoError(5, f"device status word {status}")
+    if sync:
+        torch.cuda.synchronize()
+        status = int(scratch.view(torch.int32)[(base - scratch.data_ptr()) // 4].item())
+        if status:
+            raise ZoError(5, f"device status word {status}")
     return Y
 
 

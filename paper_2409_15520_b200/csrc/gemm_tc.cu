@@ -422,7 +422,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + a * BN;
       const int rrow = P.res ? (P.res_mod > 0 ? row % P.res_mod : row) : 0;
       // per-tile LoRA constants: all rows of the tile belong to one replica
-      const int rep = P.has_lora ? m0 / P.L.rows_per_replica : 0;
+      const int rep = P.has_lora ? P.L.rep_base + P.L.rep_stride * (m0 / P.L.rows_per_replica) : 0;
       const float sgn = (rep & 1) ? -P.L.eps : P.L.eps;
       const float* urow = P.has_lora ? P.L.U + (size_t)min(row, P.M - 1) * P.L.ldu : nullptr;
       const bool u_vec = P.has_lora && (P.L.ldu % 4 == 0) && (P.L.r % 4 == 0) && (((uintptr_t)P.L.U & 15) == 0);

@@ -293,8 +293,9 @@ __global__ void lora_apply_kernel(const T* base, int ldb, int base_shared,
     }
   }
   if (slot >= 0) {
-    const float sgn = (n & 1) ? -L.eps : L.eps;
-    const uint32_t query = (uint32_t)(n >> 1);
+    const int rid = L.rep_base + L.rep_stride * n;   // replica id within the step
+    const float sgn = (rid & 1) ? -L.eps : L.eps;
+    const uint32_t query = (uint32_t)(rid >> 1);
     const float* Bs = L.B + (size_t)slot * L.r * L.width;
     float la[LA_ROWS][4];
 #pragma unroll
@@ -730,17 +731,21 @@ void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target
 // loss of a path is the mean over the labelled positions of the batch).
 // =========================================================================================
 __global__ void replica_mean_kernel(const double* __restrict__ row_loss,
-                                    const int32_t* __restrict__ lab_val, int rows,
+                                    const int32_t* __restrict__ lab_val, int rows, int rep_base,
+                                    int rep_stride, double* __restrict__ rows_out,
                                     float* __restrict__ losses, double* __restrict__ losses_d,
                                     uint32_t* status) {
   __shared__ double sd[256];
   __shared__ int sc[256];
   const int n = blockIdx.x;
+  const int rid = rep_base + rep_stride * n;     // replica id within the step
   double s = 0.0;
   int c = 0;
   for (int i = threadIdx.x; i < rows; i += 256) {
+    const double v = row_loss[(size_t)n * rows + i];
+    rows_out[(size_t)rid * rows + i] = v;
     if (!lab_val || lab_val[i] >= 0) {
-      s += row_loss[(size_t)n * rows + i];
+      s += v;
       ++c;
     }
   }
@@ -757,15 +762,17 @@ __global__ void replica_mean_kernel(const double* __restrict__ row_loss,
   if (threadIdx.x == 0) {
     const double ld = sc[0] > 0 ? sd[0] / (double)sc[0] : 0.0;
     const float l = (float)ld;
-    losses[n] = l;
-    losses_d[n] = ld;
+    losses[rid] = l;
+    losses_d[rid] = ld;
     if (!isfinite(l)) atomicOr(status, ST_NONFINITE);
   }
 }
 void launch_replica_mean(cudaStream_t st, const double* row_loss, const int32_t* lab_val, int n,
-                         int rows_per_replica, float* losses, double* losses_d, uint32_t* status) {
+                         int rows_per_replica, int rep_base, int rep_stride, double* rows_out,
+                         float* losses, double* losses_d, uint32_t* status) {
   if (n <= 0) return;
-  replica_mean_kernel<<<n, 256, 0, st>>>(row_loss, lab_val, rows_per_replica, losses, losses_d, status);
+  replica_mean_kernel<<<n, 256, 0, st>>>(row_loss, lab_val, rows_per_replica, rep_base, rep_stride,
+                                         rows_out, losses, losses_d, status);
 }
 
 // =========================================================================================

@@ -17,6 +17,7 @@ struct LoraDesc {
   uint64_t seed;
   uint32_t tensor_base;  // tensor_id of slot 0
   int rows_per_replica;  // rows of one replica in the (padded) activation layout
+  int rep_base, rep_stride;  // replica id of the j-th replica in the buffers = rep_base + rep_stride * j
 };
 
 enum { ACT_NONE = 0, ACT_RELU = 1 };
@@ -71,8 +72,11 @@ void launch_mse_rows(cudaStream_t st, int bf, const void* Y, const float* target
                      int Tp, int k_out, double* row_loss);
 // losses[n] = mean of the valid rows of replica n (fixed order, fp64 accumulation); the fp64
 // copy feeds the projected gradients, whose loss difference would drown in fp32 rounding.
+// The j-th replica of the pass is replica rep_base + rep_stride * j of the step: its mean goes to
+// losses[that id] and its rows are copied to rows_out[that id] (the per-step row-loss table).
 void launch_replica_mean(cudaStream_t st, const double* row_loss, const int32_t* lab_val, int n,
-                         int rows_per_replica, float* losses, double* losses_d, uint32_t* status);
+                         int rows_per_replica, int rep_base, int rep_stride, double* rows_out,
+                         float* losses, double* losses_d, uint32_t* status);
 
 struct UpdateDesc {
   enum { MAX_T = 96 };

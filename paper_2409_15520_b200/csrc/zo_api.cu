@@ -18,7 +18,7 @@ char g_init_error[256] = "";
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
-      xh, logits, rowloss, losses, losses_d, g, status, total;
+      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, total;
 };
 
 inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -100,6 +100,7 @@ Plan make_plan(const zo_config& c) {
     p.tok_stage = take(Tm * c.d_model * es);          // host-variant staging of X
     p.lab_stage = take(Tm * c.d_out * 4);             // and of the targets
     p.rowloss = take(n * Tm * 8);
+    p.rowloss_pass = take(n * Tm * 8);
   } else {
     const size_t d = c.d_model, f = c.d_ffn, J = (size_t)n_targets(c) * c.lora_rank;
     const size_t P = c.max_labelled, Mh = n * c.max_E * P;
@@ -121,6 +122,7 @@ Plan make_plan(const zo_config& c) {
     p.xh = take(Mh * d * es);
     if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
     p.rowloss = take(Mh * 8);
+    p.rowloss_pass = take(Mh * 8);
   }
   p.losses = take(n * 4);
   p.losses_d = take(n * 8);
@@ -151,6 +153,7 @@ struct zo_ctx {
   int slot_of_sec[3];
   int launches;
   int stepped, last_q, last_E, last_S;
+  int schedule;
   char err[256];
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -234,6 +237,27 @@ zo_status run_lora_down(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, cons
   return ZO_OK;
 }
 
+// The forward passes a step is cut into.  Pass p covers the replicas base + stride * j, j < count.
+struct Pass { int base, stride, count; };
+inline int make_passes(int schedule, int q, Pass* out) {   // out holds up to 2q entries
+  int np = 0;
+  switch (schedule) {
+    case ZO_SCHEDULE_OUTER_ONLY:   // all +eps replicas, then all -eps replicas
+      out[np++] = Pass{0, 2, q};
+      out[np++] = Pass{1, 2, q};
+      break;
+    case ZO_SCHEDULE_INNER_ONLY:   // the +/- pair of one query at a time
+      for (int i = 0; i < q; ++i) out[np++] = Pass{2 * i, 1, 2};
+      break;
+    case ZO_SCHEDULE_SEQUENTIAL:   // one perturbed forward at a time
+      for (int n = 0; n < 2 * q; ++n) out[np++] = Pass{n, 1, 1};
+      break;
+    default:                       // everything in one pass
+      out[np++] = Pass{0, 1, 2 * q};
+  }
+  return np;
+}
+
 // Can the MP-LoRA term ride in the tensor-core GEMM's epilogue?
 inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
   return bf && !(flags & ZO_FLAG_SIMT_GEMM) && Tp % 128 == 0 && width % 32 == 0;
@@ -242,7 +266,7 @@ inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
 zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* X,
                       const void* target, int T, uint64_t seed, int q, float eps, float lr) {
   const zo_config& cf = c->cfg;
-  const int bf = c->bf, n = 2 * q, r = cf.lora_rank, ki = cf.d_model, ko = cf.d_out;
+  const int bf = c->bf, r = cf.lora_rank, ki = cf.d_model, ko = cf.d_out;
   const int Tp = (int)up(T, row_pad(cf));
   cudaStream_t st = c->st;
   uint32_t* status = c->at<uint32_t>(c->plan.status);
@@ -250,9 +274,14 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   void* base = c->at<uint8_t>(c->plan.qkv0);
   void* Y = c->at<uint8_t>(c->plan.qkv);
   double* rowloss = c->at<double>(c->plan.rowloss);
+  double* rowloss_pass = c->at<double>(c->plan.rowloss_pass);
   float* losses = c->at<float>(c->plan.losses);
   double* losses_d = c->at<double>(c->plan.losses_d);
-
+  Pass passes[64];
+  const int n_pass = make_passes(c->schedule, q, passes);
+  for (int pi = 0; pi < n_pass; ++pi) {
+  const Pass ps = passes[pi];
+  const int n = ps.count;
   zo_status s = run_lora_down(c, st, bf, cf.flags, X, ki, lora->A[0], U, T, ki, r, status, c->n_sms,
                               &c->launches, c->err, sizeof(c->err));
   if (s) return s;
@@ -265,9 +294,11 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   L.U = U; L.ldu = r; L.B = lora->B[0]; L.r = r; L.width = ko;
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
+  L.rep_base = ps.base; L.rep_stride = ps.stride;
   PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
-  PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss));
-  PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss, nullptr, n, T, losses, losses_d, status));
+  PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss_pass));
+  PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, nullptr, n, T, ps.base, ps.stride, rowloss, losses, losses_d, status));
+  }
   UpdateDesc D{};
   D.B[0] = lora->B[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
   D.elems_per_slot = (long long)r * ko;
@@ -279,8 +310,8 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
                        const int32_t* labels, int E, int S, uint64_t seed, int q, float eps,
                        float lr) {
   const zo_config& cf = c->cfg;
-  const int bf = c->bf, n = 2 * q, r = cf.lora_rank, d = cf.d_model, f = cf.d_ffn, H = cf.n_heads;
-  const int T = E * S, Tp = (int)up(T, row_pad(cf)), M = n * Tp;
+  const int bf = c->bf, r = cf.lora_rank, d = cf.d_model, f = cf.d_ffn, H = cf.n_heads;
+  const int T = E * S, Tp = (int)up(T, row_pad(cf));
   const int nt = c->nt, J = nt * r;
   const bool opt = cf.arch == ZO_ARCH_OPT;
   const int nkind = opt ? 0 : 1;
@@ -296,6 +327,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   int32_t *lab_idx = c->at<int32_t>(c->plan.lab_idx), *lab_val = c->at<int32_t>(c->plan.lab_val);
   int32_t* lab_cnt = c->at<int32_t>(c->plan.lab_cnt);
   double* rowloss = c->at<double>(c->plan.rowloss);
+  double* rowloss_pass = c->at<double>(c->plan.rowloss_pass);
   float* losses = c->at<float>(c->plan.losses);
   double* losses_d = c->at<double>(c->plan.losses_d);
   zo_status s;
@@ -305,11 +337,17 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     if (s) return s;                                                                             \
   } while (0)
 
-  // shared prefix: embedding on the T shared tokens, once for all 2q replicas
-  PROF(PC_MISC, 0.0, launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, S, d, cf.vocab, status));
   const int P = cf.max_labelled, EP = E * P;
   const int n_classes = cf.loss_kind == ZO_LOSS_CE_LABEL_WORDS ? 2 : cf.vocab;
   PROF(PC_MISC, 0.0, launch_label_scan(st, labels, E, S, P, n_classes, lab_idx, lab_val, lab_cnt, status));
+
+  Pass passes[64];
+  const int n_pass = make_passes(c->schedule, q, passes);
+  for (int pi = 0; pi < n_pass; ++pi) {
+  const Pass ps = passes[pi];
+  const int n = ps.count, M = n * Tp;          // replicas and token rows of this forward pass
+  // shared prefix: embedding on the T shared tokens, once for all replicas of the pass
+  PROF(PC_MISC, 0.0, launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, S, d, cf.vocab, status));
 
   for (int l = 0; l < cf.n_layers; ++l) {
     const zo_layer_weights& W = w->layers[l];
@@ -323,6 +361,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     for (int j = 0; j < 3; ++j) L.slot_of_sec[j] = c->slot_of_sec[j];
     L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = (uint32_t)(l * nt);
     L.rows_per_replica = Tp;
+    L.rep_base = ps.base; L.rep_stride = ps.stride;
     if (J) {
       s = run_lora_down(c, st, bf, cf.flags, xn, d, lora->A[l], U, rows, d, J, status, c->n_sms,
                         &c->launches, c->err, sizeof(c->err));
@@ -385,11 +424,12 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     Hd.A = xh; Hd.lda = d; Hd.W = head; Hd.M = Mh; Hd.N = cf.vocab; Hd.K = d;
     Hd.out = logits; Hd.ldo = cf.vocab; Hd.out_f32 = 1; Hd.prof_class = PC_GEMM_HEAD;
     GEMM(Hd);
-    PROF(PC_LOSS, 0.0, launch_ce_rows(st, logits, cf.vocab, cf.vocab, lab_val, EP, Mh, rowloss));
+    PROF(PC_LOSS, 0.0, launch_ce_rows(st, logits, cf.vocab, cf.vocab, lab_val, EP, Mh, rowloss_pass));
   } else {
-    PROF(PC_LOSS, 0.0, launch_label_word_rows(st, bf, xh, head, d, cf.label_words[0], cf.label_words[1], lab_val, EP, Mh, rowloss));
+    PROF(PC_LOSS, 0.0, launch_label_word_rows(st, bf, xh, head, d, cf.label_words[0], cf.label_words[1], lab_val, EP, Mh, rowloss_pass));
   }
-  PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss, lab_val, n, EP, losses, losses_d, status));
+  PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, lab_val, n, EP, ps.base, ps.stride, rowloss, losses, losses_d, status));
+  }  // passes
 
   // projected gradients and ZO-SGD update of every B tensor
   float* g = c->at<float>(c->plan.g);
@@ -598,6 +638,14 @@ zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows) {
 
 int32_t zo_launch_count(const zo_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+zo_status zo_set_schedule(zo_ctx* ctx, int32_t schedule) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (schedule < ZO_SCHEDULE_FULL || schedule > ZO_SCHEDULE_SEQUENTIAL)
+    return fail(ctx, ZO_ERR_INVALID_ARG, "unknown schedule");
+  ctx->schedule = schedule;
+  return ZO_OK;
+}
+
 void zo_free(zo_ctx* ctx) {
   if (!ctx) return;
   if (ctx->prof) {
@@ -690,6 +738,7 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
   L.scale = scale; L.eps = eps; L.seed = seed; L.tensor_base = tensor_id; L.rows_per_replica = T;
+  L.rep_base = 0; L.rep_stride = 1;
   GemmDesc G{};
   G.A = X; G.lda = k_in; G.W = W; G.M = (int)rows; G.N = k_out; G.K = k_in; G.bias = bias;
   G.ldo = k_out;

@@ -15,7 +15,7 @@ def make_problem(spec, seed=1234, b_std=0.0):
     return p, p["tokens"], p["labels"]
 
 
-def run_gpu(spec, p, seed, q=None, eps=None, lr=None, flags=0, host=False, **cfg_kw):
+def run_gpu(spec, p, seed, q=None, eps=None, lr=None, flags=0, host=False, schedule=None, **cfg_kw):
     import paper_2409_15520_b200 as zo
     q = spec.q if q is None else q
     eps = spec.eps if eps is None else eps
@@ -23,6 +23,8 @@ def run_gpu(spec, p, seed, q=None, eps=None, lr=None, flags=0, host=False, **cfg
     cfg = zo.make_config(spec, flags=flags, max_q=max(q, spec.q), **cfg_kw)
     est = zo.Estimator(cfg)
     prob = zo.DeviceProblem(p, spec.bf16)
+    if schedule:
+        est.set_schedule(schedule)
     (est.step_host if host else est.step)(prob, spec.E, spec.S, seed, q, eps, lr)
     losses, g = est.losses()
     rows = est.row_losses()

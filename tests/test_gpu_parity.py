@@ -173,6 +173,31 @@ def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
     assert np.max(np.abs(d_gpu - d_ref)) < 0.1 * np.max(np.abs(d_ref)) + 2 * 2.0 ** -8 * np.max(np.abs(ref))
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+def test_schedules_give_the_same_step(bf16):
+    """Outer-only, inner-only and sequential cuts of the step (the paper's ablation of its two
+    parallelisations) reproduce the single-pass step: same losses, projected gradients and update."""
+    spec = ModelSpec(arch=ARCH_LLAMA, bf16=bf16, **{**TINY, "d_model": 128, "n_heads": 2, "S": 40,
+                                                   "max_seq": 40, "q": 3})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    full = run_gpu(spec, p, 17)
+    ref = run_oracle(spec, p, tok, lab, 17)
+    assert np.allclose(full["losses"], ref["losses"], rtol=2e-2 if bf16 else 1e-4)
+    for sched in ("outer_only", "inner_only", "sequential"):
+        got = run_gpu(spec, p, 17, schedule=sched)
+        assert np.array_equal(got["losses"], full["losses"]), sched
+        assert np.array_equal(got["g"], full["g"]), sched
+        assert np.array_equal(got["rows"], full["rows"]), sched
+        assert all(np.array_equal(a, b) for a, b in zip(got["B"], full["B"])), sched
+        assert got["launches"] > full["launches"]
+    lin = config("linear_fp32", q=3)
+    pl, _, _ = make_problem(lin, b_std=0.02)
+    a = run_gpu(lin, pl, 4)
+    for sched in ("outer_only", "inner_only", "sequential"):
+        b = run_gpu(lin, pl, 4, schedule=sched)
+        assert np.array_equal(a["losses"], b["losses"]) and np.array_equal(a["B"][0], b["B"][0])
+
+
 def test_degenerate_steps():
     spec = ModelSpec(arch=ARCH_OPT, tie_lm_head=True, bf16=False, **TINY)
     p, tok, lab = make_problem(spec, b_std=0.05)
