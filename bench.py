@@ -189,6 +189,49 @@ def run_sweep(args):
             print(json.dumps(out), flush=True)
 
 
+def run_ablation(args, spec):
+    """The paper's runtime ablations on this GPU (fixed-length synthetic batches on the 7B shape):
+    inner-loop (q = 1: the +/- pair in one pass vs two sequential passes) over seq x batch, and
+    outer-loop (q*E = 16 fixed) over (q, E) x seq, each under the schedules that apply.  One JSON
+    line per point, ms per step (median of 5 after 2 warm-ups) and ratios."""
+    import torch
+    import paper_2409_15520_b200 as zo
+    from workloads import next_token_labels
+    big = spec.with_(q=16, E=16, S=256)
+    prob = load_problem(big)
+    est = zo.Estimator(zo.make_config(big, flags=args.flags))
+    rng = np.random.default_rng(7)
+
+    def time_point(q, E, S, schedule):
+        tok = rng.integers(0, spec.vocab, size=(E, S), dtype=np.int32)
+        lab = next_token_labels(tok, min(spec.n_labelled, S - 1))
+        dt, dl = torch.tensor(tok, device="cuda"), torch.tensor(lab, device="cuda")
+        est.set_schedule(schedule)
+        ts = []
+        for i in range(7):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            est.step(prob, E, S, 50 + i, q, spec.eps, spec.lr, tokens=dt, labels=dl)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        est.losses()
+        return float(np.median(ts[2:]))
+
+    for S in (64, 128, 256):
+        for E in (1, 8, 16):
+            par, seq = time_point(1, E, S, "full"), time_point(1, E, S, "sequential")
+            print(json.dumps({"table": "inner_loop", "q": 1, "seq": S, "batch": E, "ms_parallel_pair": round(par, 3),
+                              "ms_sequential_pair": round(seq, 3), "speedup": round(seq / par, 3)}), flush=True)
+    for S in (64, 128, 256):
+        for q, E in ((1, 16), (4, 4), (16, 1)):
+            r = {"table": "outer_loop", "q": q, "E": E, "seq": S}
+            for sched in ("full", "outer_only", "inner_only", "sequential"):
+                r["ms_" + sched] = round(time_point(q, E, S, sched), 3)
+            r["speedup_full_vs_sequential"] = round(r["ms_sequential"] / r["ms_full"], 3)
+            print(json.dumps(r), flush=True)
+
+
 def run_reference(args, spec):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -227,6 +270,7 @@ def main():
     ap.add_argument("--targets", type=int, default=-1, help="override lora_targets (0 = no adapted projection)")
     ap.add_argument("--rank", type=int, default=0, help="override the LoRA rank")
     ap.add_argument("--sweep", action="store_true", help="MP-LoRA linear micro-benchmark grid (rank x q)")
+    ap.add_argument("--ablation", action="store_true", help="the paper's inner/outer-loop runtime grids on this GPU")
     ap.add_argument("--schedule", default="full", choices=["full", "outer_only", "inner_only", "sequential"],
                     help="how the step is cut into forward passes (the paper's ablation)")
     ap.add_argument("--E", type=int, default=0, help="override the number of sequences")
@@ -249,6 +293,8 @@ def main():
         spec = spec.with_(lora_rank=args.rank)
     if args.impl == "reference":
         return run_reference(args, spec)
+    if args.ablation:
+        return run_ablation(args, spec)
 
     import torch
     import torch.distributed as dist
