@@ -72,7 +72,11 @@ enum { ZO_TARGET_Q = 1, ZO_TARGET_K = 2, ZO_TARGET_V = 4 };
 enum { ZO_FLAG_SIMT_GEMM = 1,
        /* ZO_FLAG_GEMM_PAIR: tensor-core GEMMs run CTA pairs (tcgen05 cta_group::2) on 256-row
         * tiles instead of the default one CTA per 128-row tile (A/B switch; bit-identical results). */
-       ZO_FLAG_GEMM_PAIR = 2 };
+       ZO_FLAG_GEMM_PAIR = 2,
+       /* ZO_FLAG_LORA_EPILOGUE: the MP-LoRA term is always added on CUDA cores in the GEMM epilogue
+        * from fp32 U and fp32 (B + k eps z), never as the extra tensor-core k-block (which rounds
+        * U, B and k eps z to bfloat16).  A/B switch. */
+       ZO_FLAG_LORA_EPILOGUE = 4 };
 
 typedef struct zo_ctx zo_ctx; /* opaque; owned by the library; released by zo_free */
 

@@ -10,6 +10,14 @@
 //     with z_i regenerated from the Philox seed inside the epilogue (never in HBM).  Every
 //     128-row tile lies inside one replica, so the perturbed B columns of the tile are built
 //     once in shared memory and reused by its 128 rows.
+//   * Tensor-core form of the MP-LoRA term (rank <= 32, sections that are a multiple of the
+//     256-column tile, single-CTA variant): the term becomes one extra 64-deep k-block of the
+//     same accumulator.  Its A operand is a bf16 copy of U laid out [U | U] (written by the
+//     down-projection's epilogue, loaded by TMA), its B operand [s B ; s k eps z] is generated
+//     by the epilogue warps straight into shared memory in the swizzled K-major layout the MMA
+//     expects, one tile ahead.  Keeping B and k eps z in separate K ranges keeps the
+//     perturbation's resolution in bf16 whatever the magnitude of B.  Otherwise the term is
+//     added on CUDA cores in the epilogue from fp32 U and fp32 (B + k eps z).
 //   * PAIR variant (opt-in; measured slower under the 1 kW power cap than one CTA per tile, see
 //     the design notes): two CTAs of a cluster work on one 256 x 256 tile with
 //     tcgen05.mma.cta_group::2 - each CTA stages its own 128 rows of A and its 128-row half of
@@ -47,12 +55,13 @@ constexpr int THREADS = 64 + EP_THREADS;        // warp 0: TMA, warp 1: MMA, war
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct Ctrl {
-  unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2], drain;
+  unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2], drain, lfull;
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
 };
-constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + 2 * LORA_BUF_FLOATS * 4 + sizeof(Ctrl);  // both variants: 192 KiB of stages
+constexpr uint32_t SLAB_BYTES = BN * BK * 2;     // generated B operand of the LoRA k-block (aliases the fp32 staging)
+constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + SLAB_BYTES + sizeof(Ctrl);  // both variants: 192 KiB of stages
 
 struct Params {
   int M, N, K;              // N: accumulator columns (swiglu: d_ffn, the number of OUTPUT columns)
@@ -61,6 +70,10 @@ struct Params {
   const bf16* res; int ldr; int res_mod;
   int act, swiglu;
   int has_lora;
+  int slab;                 // 1: the LoRA term is an extra k-block on the tensor cores
+  int kslot, khalf;         // K extent of one slot in the packed bf16 U, offset of its second copy
+  bf16* pack_out; int pack_ld;  // down-projection: also write the packed bf16 U here (or null)
+  int pack_r;
   LoraDesc L;
   uint32_t* status;
 };
@@ -263,10 +276,15 @@ __device__ __forceinline__ void load_u16(const float* p, int left, bool vec, flo
   }
 }
 
+// Slab mode: the LoRA slot of the tile whose first output column is n0 (-1: not adapted).
+__device__ __forceinline__ int tile_slot(const Params& P, int n0) {
+  return P.slab ? P.L.slot_of_sec[n0 / P.L.width] : -1;
+}
+
 template <bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const Params P) {
+               const __grid_constant__ CUtensorMap tmU, const Params P) {
   constexpr int STAGES = Cfg<PAIR>::STAGES;
   constexpr uint32_t STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
   constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
@@ -274,7 +292,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   float* lbuf = (float*)(smem + STAGES * STAGE_BYTES);
-  Ctrl* ctrl = (Ctrl*)(smem + STAGES * STAGE_BYTES + 2 * LORA_BUF_FLOATS * 4);
+  Ctrl* ctrl = (Ctrl*)(smem + STAGES * STAGE_BYTES + SLAB_BYTES);
   const uint32_t tiles_base = smem_u32(smem);
   const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -297,6 +315,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 2 * EP_WARPS : EP_WARPS);
     }
     mbar_init(smem_u32(&ctrl->drain), 1);
+    mbar_init(smem_u32(&ctrl->lfull), EP_WARPS);
     ctrl->abort = 0u;
     ctrl->ep_go = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -351,6 +370,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
           }
         }
+        const int lslot = PAIR ? -1 : tile_slot(P, brow0);
+        if (ok && lslot >= 0) {
+          // LoRA k-block: only the A operand (packed U) travels through the ring
+          const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
+          if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
+          const uint32_t bar = smem_u32(&ctrl->full[s]);
+          mbar_expect_tx(bar, A_BYTES);
+          tma_load_2d(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot, m0, bar);
+          ++issued;
+        }
       }
       if (!ok && (!PAIR || rank == 0)) {
         // abort: let the copies already issued land before the CTA goes away
@@ -362,7 +391,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
-      uint32_t consumed = 0, titer = 0;
+      uint32_t consumed = 0, titer = 0, ltiles = 0;
       bool ok = true;
       for (int tile = unit; tile < num_tiles && ok; tile += n_units, ++titer) {
         const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -388,6 +417,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (PAIR) tc_commit_pair(smem_u32(&ctrl->empty[s]));
           else tc_commit(smem_u32(&ctrl->empty[s]));
         }
+        if (!PAIR && ok) {
+          int tm, tn;
+          tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+          if (tile_slot(P, tn * ncol_tile) >= 0) {
+            const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
+            if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
+                !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status)) { ok = false; break; }
+            ++ltiles;
+            tc_fence_after();
+            const uint64_t ad = smem_desc(tiles_base + s * STAGE_BYTES);
+            const uint64_t bd = smem_desc(tiles_base + STAGES * STAGE_BYTES);
+#pragma unroll
+            for (int k = 0; k < BK / 16; ++k)
+              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC, 1u);
+            tc_commit(smem_u32(&ctrl->empty[s]));
+            ++consumed;
+          }
+        }
         if (ok) {
           if (PAIR) tc_commit_pair(smem_u32(&ctrl->tfull[a]));
           else tc_commit(smem_u32(&ctrl->tfull[a]));
@@ -405,6 +452,58 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;              // which of the quarter's two warps: even or odd chunks
     const bool out_vec_ok = ((uintptr_t)P.out & 15) == 0 && (P.ldo % (P.out_f32 ? 4 : 8)) == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
+    uint8_t* slab = smem + STAGES * STAGE_BYTES;
+    // Slab mode: build the B operand [s B ; s k eps z] of a tile's LoRA k-block: 256 rows (output
+    // columns) x 64 K-elements, K-major with the 128-byte swizzle.  Rank index k sits at K = k
+    // (B part) and K = khalf + k (perturbation part); all other K positions stay zero.
+    auto gen_slab = [&](int g_tile) {
+      int tm, tn;
+      tile_coords(g_tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+      const int n0g = tn * ncol_tile;
+      const int slot = tile_slot(P, n0g);
+      if (slot < 0) return;                         // uniform over the CTA
+      const int sec = n0g / P.L.width, cs = n0g - sec * P.L.width;
+      const int repg = P.L.rep_base + P.L.rep_stride * ((tm * TILE_M) / P.L.rows_per_replica);
+      const float sz = ((repg & 1) ? -P.L.eps : P.L.eps) * P.L.scale;
+      const float* Bm = P.L.B + (size_t)slot * P.L.r * P.L.width;
+      const int kgroups = (P.L.r + 7) / 8;
+      for (int unit_i = et; unit_i < 64 * kgroups; unit_i += EP_THREADS) {
+        const int c4 = (unit_i & 63) * 4, k0 = (unit_i >> 6) * 8;
+        float bb[8][4], zz[8][4];
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const int k = k0 + kk;
+          float4 b = make_float4(0.f, 0.f, 0.f, 0.f), z = b;
+          if (k < P.L.r) {
+            const size_t e = (size_t)k * P.L.width + cs + c4;
+            b = *reinterpret_cast<const float4*>(Bm + e);
+            if (P.L.eps != 0.f) z = z_block(P.L.seed, P.L.tensor_base + slot, (uint32_t)(repg >> 1), (uint32_t)(e >> 2));
+          }
+          bb[kk][0] = b.x * P.L.scale; bb[kk][1] = b.y * P.L.scale; bb[kk][2] = b.z * P.L.scale; bb[kk][3] = b.w * P.L.scale;
+          zz[kk][0] = z.x * sz; zz[kk][1] = z.y * sz; zz[kk][2] = z.z * sz; zz[kk][3] = z.w * sz;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int n = c4 + j;                       // row of the operand tile = output column
+          const uint4 vb = make_uint4(pack_bf16(bb[0][j], bb[1][j]), pack_bf16(bb[2][j], bb[3][j]),
+                                      pack_bf16(bb[4][j], bb[5][j]), pack_bf16(bb[6][j], bb[7][j]));
+          const uint4 vz = make_uint4(pack_bf16(zz[0][j], zz[1][j]), pack_bf16(zz[2][j], zz[3][j]),
+                                      pack_bf16(zz[4][j], zz[5][j]), pack_bf16(zz[6][j], zz[7][j]));
+          const int cb = k0 >> 3, cz = (P.khalf + k0) >> 3;  // 16-byte chunk index along K
+          *reinterpret_cast<uint4*>(slab + n * 128 + ((cb ^ (n & 7)) << 4)) = vb;
+          *reinterpret_cast<uint4*>(slab + n * 128 + ((cz ^ (n & 7)) << 4)) = vz;
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->lfull));
+    };
+    if (!PAIR && P.slab) {
+      for (int i = et; i < (int)(SLAB_BYTES / 16); i += EP_THREADS)
+        reinterpret_cast<uint4*>(slab)[i] = make_uint4(0, 0, 0, 0);
+      ep_bar();
+      if (unit < num_tiles) gen_slab(unit);
+    }
     uint32_t titer = 0;
     for (int tile = unit; tile < num_tiles; tile += n_units, ++titer) {
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -414,6 +513,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ep_bar();                                    // ep_go may be rewritten after this point
       if (!go) break;
       tc_fence_after();
+      // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
+      if (!PAIR && P.slab && tile + n_units < num_tiles) gen_slab(tile + n_units);
       int tm, tn;
       tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
       const int m0 = tm * TILE_M + (int)rank * BM, n0 = tn * ncol_tile;
@@ -436,7 +537,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (col0 >= P.N) break;
         int lslot = -1;
         float u[16];
-        if (P.has_lora && !P.swiglu) {
+        if (P.has_lora && !P.slab && !P.swiglu) {
           if (c % cpp == 0) {
             bool any = false;
             for (int cc = c; cc < c + cpp && cc < nchunk; ++cc) {
@@ -529,6 +630,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         if (!row_ok) continue;
+        if (P.pack_out) {
+          // bf16 copy of U for the tensor-core LoRA k-block: rank index k of slot t goes to
+          // K = t*kslot + k and again to K = t*kslot + khalf + k
+          bf16* pr = P.pack_out + (size_t)row * P.pack_ld;
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int col = col0 + j;
+            if (col < P.N) {
+              const int t = col / P.pack_r, k = col - t * P.pack_r;
+              const bf16 hv = __float2bfloat16_rn(f[j]);
+              pr[t * P.kslot + k] = hv;
+              pr[t * P.kslot + P.khalf + k] = hv;
+            }
+          }
+        }
         const bool full_chunk = col0 + 32 <= P.N;
         // 16-byte vector accesses need the row pitch (and base) to keep rows 16-byte aligned
         const bool vec_out = full_chunk && out_vec_ok;
@@ -660,6 +776,14 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.act = G.act; P.swiglu = G.swiglu;
   P.has_lora = G.lora ? 1 : 0;
   if (G.lora) P.L = *G.lora; else P.L = LoraDesc{};
+  P.slab = (G.lora && G.lora_slab) ? 1 : 0;
+  P.kslot = G.kslot; P.khalf = G.khalf;
+  P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
+  CUtensorMap tmU = tmA;
+  if (P.slab) {
+    e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)G.M, (uint64_t)G.pack_ld);
+    if (e) return 10000 + e;
+  }
   P.status = status;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
   if (G.cta_pair && P.M > tc::BM) {
@@ -683,12 +807,13 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     const long long tiles = (long long)((P.M + 2 * tc::BM - 1) / (2 * tc::BM)) * tiles_n;
     const int pairs = (int)(tiles < max_clusters ? tiles : max_clusters);
     cfg.gridDim = dim3(2 * pairs);
-    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true>, tmA, tmB, P);
+    P.slab = 0;
+    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true>, tmA, tmB, tmU, P);
   }
   const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
   const long long tiles = (long long)tiles_m * tiles_n;
   const int grid = (int)(tiles < n_sms ? tiles : n_sms);
-  tc::gemm_tc_kernel<false><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, P);
+  tc::gemm_tc_kernel<false><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
   return (int)cudaGetLastError();
 }
 

@@ -34,6 +34,10 @@ struct GemmDesc {
   int act;
   int swiglu;                   // 1: W = [gate rows | up rows] (N = 2 * d_ffn), out = silu(g)*u
   const LoraDesc* lora;         // null: plain GEMM
+  int lora_slab;                // 1: the LoRA term runs as an extra tensor-core k-block fed from pack_u
+  const void* pack_u;           // bf16 [M, pack_ld]: per slot [U | U] in kslot columns (second copy at khalf)
+  void* pack_out;               // down-projection: write that packed copy here (bf16 [M, pack_ld]) or null
+  int pack_ld, pack_r, kslot, khalf;
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
 };
