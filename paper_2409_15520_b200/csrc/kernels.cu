@@ -170,12 +170,104 @@ norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T*
   }
 }
 
+// One warp per row: the row is read once (16-byte accesses, all issued before the first use),
+// kept packed in registers, reduced with shuffles only.  Requires d % VEC == 0, d <= 32*VEC*NV.
+template <typename T, int NV>
+__global__ void __launch_bounds__(128)
+norm_warp_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
+                 const T* __restrict__ b, int rows, int d, float eps,
+                 const int32_t* __restrict__ lab_idx, int EP, int Tp) {
+  constexpr int VEC = 16 / sizeof(T);
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 4 + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  long long src = row;
+  if (lab_idx) {
+    const int n = row / EP, j = row % EP;
+    const int li = lab_idx[j];
+    src = li < 0 ? -1 : (long long)n * Tp + li;
+  }
+  T* o = out + (size_t)row * d;
+  const int nvec = d / VEC;
+  if (src < 0) {
+    for (int v = lane; v < nvec; v += 32) *reinterpret_cast<uint4*>(o + v * VEC) = make_uint4(0, 0, 0, 0);
+    return;
+  }
+  const T* xr = x + (size_t)src * d;
+  uint4 raw[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int v = lane + 32 * i;
+    raw[i] = v < nvec ? *reinterpret_cast<const uint4*>(xr + v * VEC) : make_uint4(0, 0, 0, 0);
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const T* e = reinterpret_cast<const T*>(&raw[i]);
+#pragma unroll
+    for (int j = 0; j < VEC; ++j) {
+      const float t = to_f(e[j]);
+      s += kind == 0 ? t : t * t;
+    }
+  }
+  s = warp_sum(s);
+  float mu = 0.f, rstd;
+  if (kind == 0) {
+    mu = s / d;
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      if (lane + 32 * i < nvec) {
+        const T* e = reinterpret_cast<const T*>(&raw[i]);
+#pragma unroll
+        for (int j = 0; j < VEC; ++j) {
+          const float t = to_f(e[j]) - mu;
+          q += t * t;
+        }
+      }
+    }
+    rstd = rsqrtf(warp_sum(q) / d + eps);
+  } else {
+    rstd = rsqrtf(s / d + eps);
+  }
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int v = lane + 32 * i;
+    if (v < nvec) {
+      const uint4 graw = *reinterpret_cast<const uint4*>(g + v * VEC);
+      const T* ge = reinterpret_cast<const T*>(&graw);
+      uint4 braw = make_uint4(0, 0, 0, 0);
+      if (kind == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
+      const T* be = reinterpret_cast<const T*>(&braw);
+      const T* e = reinterpret_cast<const T*>(&raw[i]);
+      uint4 oraw;
+      T* oe = reinterpret_cast<T*>(&oraw);
+#pragma unroll
+      for (int j = 0; j < VEC; ++j)
+        oe[j] = from_f<T>((to_f(e[j]) - mu) * rstd * to_f(ge[j]) + ((kind == 0 && b) ? to_f(be[j]) : 0.f));
+      *reinterpret_cast<uint4*>(o + v * VEC) = oraw;
+    }
+  }
+}
+
 template <typename T>
 static void norm_dispatch(cudaStream_t st, int kind, const void* x, void* out, const void* g,
                           const void* b, int rows, int d, float eps, const int32_t* lab_idx, int EP,
                           int Tp) {
   constexpr int VEC = 16 / sizeof(T);
   const bool aligned = (((uintptr_t)x | (uintptr_t)out | (uintptr_t)g | (uintptr_t)b) & 15) == 0;
+  if (aligned && d % VEC == 0 && d <= 32 * VEC * 16) {
+    const int nv = (d / VEC + 31) / 32;
+    const int grid = (rows + 3) / 4;
+#define ZO_NW(NV) norm_warp_kernel<T, NV><<<grid, 128, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp)
+    if (nv <= 1) ZO_NW(1);
+    else if (nv <= 2) ZO_NW(2);
+    else if (nv <= 4) ZO_NW(4);
+    else if (nv <= 8) ZO_NW(8);
+    else ZO_NW(16);
+#undef ZO_NW
+    return;
+  }
   if (aligned && d % VEC == 0 && d <= 256 * VEC * 4) {
     const int nvec = d / VEC;
     int th = nvec < 256 ? ((nvec + 31) / 32) * 32 : 256;
@@ -268,84 +360,74 @@ void launch_lora_down(cudaStream_t st, int bf, const void* X, int ldx, const voi
 // z regenerated from the seed in registers (never stored).  Each thread owns 4 consecutive
 // columns (= one Philox block per rank index) and LA_ROWS rows of one replica.
 // =========================================================================================
-constexpr int LA_ROWS = 8;
+constexpr int LA_ROWS = 64, LA_COLS = 128;
 template <typename T>
-__global__ void lora_apply_kernel(const T* base, int ldb, int base_shared,
-                                  T* out, int ldo, int Tn, LoraDesc L, int nsec) {
-  const int c0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
-  if (c0 >= nsec * L.width) return;
+__global__ void __launch_bounds__(256)
+lora_apply_kernel(const T* base, int ldb, int base_shared, T* out, int ldo, int Tn, LoraDesc L,
+                  int /*nsec*/) {
+  extern __shared__ float sB[];                       // [r][LA_COLS]: s * (B + k eps z) of this tile
   const int n = blockIdx.z;
+  const int tiles_per_sec = (L.width + LA_COLS - 1) / LA_COLS;   // tiles never straddle two sections
+  const int sec = blockIdx.x / tiles_per_sec, cc_t = (blockIdx.x - sec * tiles_per_sec) * LA_COLS;
+  const int col_t = sec * L.width + cc_t;             // first column of the tile
   const int t0 = blockIdx.y * LA_ROWS;
-  const int sec = c0 / L.width, cc = c0 - sec * L.width;
-  const int slot = L.slot_of_sec[sec];
+  const int slot = L.slot_of_sec[sec];                // uniform over the block
   const int Tp = L.rows_per_replica;
-  float acc[LA_ROWS][4];
-#pragma unroll
-  for (int i = 0; i < LA_ROWS; ++i) {
-    const int t = t0 + i;
-    if (t < Tn) {
-      const T* bp = base + (size_t)(base_shared ? t : n * Tp + t) * ldb + c0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] = to_f(bp[j]);
-    } else {
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
-    }
-  }
+  const int ncols = min(LA_COLS, L.width - cc_t);
   if (slot >= 0) {
-    const int rid = L.rep_base + L.rep_stride * n;   // replica id within the step
+    const int rid = L.rep_base + L.rep_stride * n;    // replica id within the step
     const float sgn = (rid & 1) ? -L.eps : L.eps;
     const uint32_t query = (uint32_t)(rid >> 1);
     const float* Bs = L.B + (size_t)slot * L.r * L.width;
-    float la[LA_ROWS][4];
-#pragma unroll
-    for (int i = 0; i < LA_ROWS; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) la[i][j] = 0.f;
-    for (int k = 0; k < L.r; ++k) {
-      const size_t e = (size_t)k * L.width + cc;
-      const float4 bm = *reinterpret_cast<const float4*>(Bs + e);
-      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (L.eps != 0.f) z = z_block(L.seed, L.tensor_base + slot, query, (uint32_t)(e >> 2));
-      const float b0 = fmaf(sgn, z.x, bm.x), b1 = fmaf(sgn, z.y, bm.y);
-      const float b2 = fmaf(sgn, z.z, bm.z), b3 = fmaf(sgn, z.w, bm.w);
-#pragma unroll
-      for (int i = 0; i < LA_ROWS; ++i) {
-        const int t = t0 + i;
-        if (t < Tn) {
-          const float u = L.U[(size_t)(base_shared ? t : n * Tp + t) * L.ldu + slot * L.r + k];
-          la[i][0] = fmaf(u, b0, la[i][0]);
-          la[i][1] = fmaf(u, b1, la[i][1]);
-          la[i][2] = fmaf(u, b2, la[i][2]);
-          la[i][3] = fmaf(u, b3, la[i][3]);
+    for (int i = threadIdx.x; i < L.r * (LA_COLS / 4); i += blockDim.x) {
+      const int k = i / (LA_COLS / 4), c4 = (i % (LA_COLS / 4)) * 4;
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c4 < ncols) {
+        const size_t e = (size_t)k * L.width + cc_t + c4;
+        v = *reinterpret_cast<const float4*>(Bs + e);
+        if (L.eps != 0.f) {
+          const float4 z = z_block(L.seed, L.tensor_base + slot, query, (uint32_t)(e >> 2));
+          v.x = fmaf(sgn, z.x, v.x); v.y = fmaf(sgn, z.y, v.y);
+          v.z = fmaf(sgn, z.z, v.z); v.w = fmaf(sgn, z.w, v.w);
         }
+        v.x *= L.scale; v.y *= L.scale; v.z *= L.scale; v.w *= L.scale;
+      }
+      *reinterpret_cast<float4*>(sB + k * LA_COLS + c4) = v;
+    }
+    __syncthreads();
+  }
+  const int c4 = (threadIdx.x & 31) * 4;
+  if (c4 >= ncols) return;
+  for (int i = threadIdx.x >> 5; i < LA_ROWS; i += 8) {
+    const int t = t0 + i;
+    if (t >= Tn) break;
+    const size_t brow = base_shared ? (size_t)t : (size_t)n * Tp + t;
+    const T* bp = base + brow * ldb + col_t + c4;
+    float a0 = to_f(bp[0]), a1 = to_f(bp[1]), a2 = to_f(bp[2]), a3 = to_f(bp[3]);
+    if (slot >= 0) {
+      const float* up = L.U + brow * L.ldu + slot * L.r;
+      for (int k = 0; k < L.r; ++k) {
+        const float u = up[k];
+        const float4 bv = *reinterpret_cast<const float4*>(sB + k * LA_COLS + c4);
+        a0 = fmaf(u, bv.x, a0); a1 = fmaf(u, bv.y, a1);
+        a2 = fmaf(u, bv.z, a2); a3 = fmaf(u, bv.w, a3);
       }
     }
-#pragma unroll
-    for (int i = 0; i < LA_ROWS; ++i)
-#pragma unroll
-      for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(L.scale, la[i][j], acc[i][j]);
-  }
-#pragma unroll
-  for (int i = 0; i < LA_ROWS; ++i) {
-    const int t = t0 + i;
-    if (t < Tn) {
-      T* op = out + (size_t)(n * Tp + t) * ldo + c0;
-#pragma unroll
-      for (int j = 0; j < 4; ++j) op[j] = from_f<T>(acc[i][j]);
-    }
+    T* op = out + ((size_t)n * Tp + t) * ldo + col_t + c4;
+    op[0] = from_f<T>(a0); op[1] = from_f<T>(a1); op[2] = from_f<T>(a2); op[3] = from_f<T>(a3);
   }
 }
 
 void launch_lora_apply(cudaStream_t st, int bf, const void* base, int ldb, int base_shared,
                        void* out, int ldo, int n, int T, const LoraDesc& L, int nsec) {
   if (n <= 0 || T <= 0) return;
-  const int cols4 = nsec * L.width / 4;
-  dim3 grid((cols4 + 127) / 128, (T + LA_ROWS - 1) / LA_ROWS, n);
+  const int tiles_per_sec = (L.width + LA_COLS - 1) / LA_COLS;
+  dim3 grid(nsec * tiles_per_sec, (T + LA_ROWS - 1) / LA_ROWS, n);
+  const size_t smem = (size_t)L.r * LA_COLS * sizeof(float);
   if (bf)
-    lora_apply_kernel<bf16><<<grid, 128, 0, st>>>((const bf16*)base, ldb, base_shared, (bf16*)out, ldo, T, L, nsec);
+    lora_apply_kernel<bf16><<<grid, 256, smem, st>>>((const bf16*)base, ldb, base_shared, (bf16*)out, ldo, T, L, nsec);
   else
-    lora_apply_kernel<float><<<grid, 128, 0, st>>>((const float*)base, ldb, base_shared, (float*)out, ldo, T, L, nsec);
+    lora_apply_kernel<float><<<grid, 256, smem, st>>>((const float*)base, ldb, base_shared, (float*)out, ldo, T, L, nsec);
 }
 
 // =========================================================================================
