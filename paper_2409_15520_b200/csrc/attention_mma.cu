@@ -2,7 +2,9 @@
 // sequences of the replicated batch (q and k already carry their rotary embedding).
 //
 // One CTA (4 warps) per (64-query tile, head, sequence); each warp owns 16 query rows.
-// K/V tiles of 64 keys stream through a double-buffered cp.async pipeline; scores and P V on
+// K/V tiles of 64 keys stream through cp.async with one buffer each: the next K tile is fetched
+// under the softmax and P V of the current one, the next V tile under the next Q K^T, which keeps
+// shared memory at three tiles (three CTAs per SM); scores and P V on
 // warp-level tensor-core MMAs (m16n8k16, bf16 in, fp32 accumulate) with an online softmax;
 // fully masked key tiles are skipped.  Attention is
 // ~1 % of the step's flops, so this kernel only has to stay off the critical path.
@@ -70,13 +72,14 @@ template <int N> __device__ __forceinline__ void cp_wait() {
 }
 
 template <int DH>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, 3)
 attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E, int S, int Tp,
                      int d) {
   extern __shared__ __align__(16) uint8_t sm_raw[];
   constexpr int LDS = DH + 8;
   bf16* Qs = reinterpret_cast<bf16*>(sm_raw);
-  bf16* KVs = Qs + 64 * LDS;                           // [2 buffers][K tile | V tile]
+  bf16* Ks = Qs + 64 * LDS;
+  bf16* Vs = Ks + 64 * LDS;
   const int qt = gridDim.x - 1 - blockIdx.x;          // longest tiles first
   const int q0 = qt * 64, h = blockIdx.y, sq = blockIdx.z;
   const int n = sq / E, b = sq % E;
@@ -88,10 +91,11 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
   const int kend = min(S, q0 + 64);
   const int n_kt = (kend + 63) / 64;
   stage_tile_async<DH>(Qs, qkv, row_base, ld, h * DH, q0, S);
-  stage_tile_async<DH>(KVs, qkv, row_base, ld, d + h * DH, 0, S);
-  stage_tile_async<DH>(KVs + 64 * LDS, qkv, row_base, ld, 2 * d + h * DH, 0, S);
+  stage_tile_async<DH>(Ks, qkv, row_base, ld, d + h * DH, 0, S);
   cp_commit();
-  cp_wait<0>();
+  stage_tile_async<DH>(Vs, qkv, row_base, ld, 2 * d + h * DH, 0, S);
+  cp_commit();
+  cp_wait<1>();                                        // Q and K tile 0 have landed (V may be in flight)
   __syncthreads();
   // Q fragments of this warp's 16 rows stay in registers for the whole kernel
   uint32_t qf[DH / 16][4];
@@ -114,14 +118,7 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
 
   for (int kt = 0; kt < n_kt; ++kt) {
     const int k0 = kt * 64;
-    const bf16* Ks = KVs + (kt & 1) * 2 * 64 * LDS;
-    const bf16* Vs = Ks + 64 * LDS;
-    if (kt + 1 < n_kt) {                                        // prefetch the next K/V tile
-      bf16* nb = KVs + ((kt + 1) & 1) * 2 * 64 * LDS;
-      stage_tile_async<DH>(nb, qkv, row_base, ld, d + h * DH, k0 + 64, S);
-      stage_tile_async<DH>(nb + 64 * LDS, qkv, row_base, ld, 2 * d + h * DH, k0 + 64, S);
-      cp_commit();
-    }
+    const bool more = kt + 1 < n_kt;
     // scores S = Q K^T for 16 rows x 64 keys
     float sc[8][4];
 #pragma unroll
@@ -139,6 +136,11 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
         mma_bf16(sc[2 * jp], qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3], b0, b1);
         mma_bf16(sc[2 * jp + 1], qf[kk][0], qf[kk][1], qf[kk][2], qf[kk][3], b2, b3);
       }
+    }
+    __syncthreads();                                            // every warp is done with this K tile
+    if (more) {                                                 // next K tile streams in under the rest
+      stage_tile_async<DH>(Ks, qkv, row_base, ld, d + h * DH, k0 + 64, S);
+      cp_commit();
     }
     // causal / length mask (only the diagonal tile and a ragged last tile need it)
     const bool need_mask = (k0 + 64 > q0) || (k0 + 64 > S);
@@ -187,7 +189,9 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
       o[j][0] *= corr[0]; o[j][1] *= corr[0];
       o[j][2] *= corr[1]; o[j][3] *= corr[1];
     }
-    // O += P V
+    // O += P V (the V tile was requested one phase earlier)
+    if (more) cp_wait<1>(); else cp_wait<0>();
+    __syncthreads();
 #pragma unroll
     for (int kk = 0; kk < 4; ++kk) {                            // 16 keys per step
 #pragma unroll
@@ -200,8 +204,13 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
         mma_bf16(o[2 * jp + 1], pf[kk][0], pf[kk][1], pf[kk][2], pf[kk][3], b2, b3);
       }
     }
-    cp_wait<0>();                                               // next tile has landed ...
-    __syncthreads();                                            // ... and this one is fully consumed
+    __syncthreads();                                            // every warp is done with this V tile
+    if (more) {
+      stage_tile_async<DH>(Vs, qkv, row_base, ld, 2 * d + h * DH, k0 + 64, S);
+      cp_commit();
+      cp_wait<1>();                                             // the next K tile has landed
+      __syncthreads();
+    }
   }
   // normalise and store
 #pragma unroll
@@ -223,7 +232,7 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
 
 template <int DH>
 void launch_t(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp, int d, int H) {
-  const size_t smem = (size_t)5 * 64 * (DH + 8) * sizeof(bf16);
+  const size_t smem = (size_t)3 * 64 * (DH + 8) * sizeof(bf16);
   cudaFuncSetAttribute(attention_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid((S + 63) / 64, H, n * E);
   attention_mma_kernel<DH><<<grid, 128, smem, st>>>((const bf16*)qkv, (bf16*)ctx, E, S, Tp, d);

@@ -253,6 +253,27 @@ def test_degenerate_steps():
     assert update_rel_err(spec, p0, got["B"], ref["B"]) < 2e-3
 
 
+def test_maximum_queries_and_no_labelled_positions():
+    """q = 32 (64 replicas, the largest the library accepts) on a small model in both precisions;
+    a batch without any labelled position gives zero losses and leaves B untouched."""
+    for bf16 in (False, True):
+        spec = ModelSpec(arch=ARCH_OPT, tie_lm_head=True, bf16=bf16,
+                         **{**TINY, "q": 32, "E": 1, "S": 9, "max_seq": 9, "n_layers": 1, "n_labelled": 2})
+        p, tok, lab = make_problem(spec, b_std=0.05)
+        ref = run_oracle(spec, p, tok, lab, 13)
+        got = run_gpu(spec, p, 13)
+        assert got["losses"].shape == (64,)
+        assert np.allclose(got["losses"], ref["losses"], rtol=2e-2 if bf16 else 1e-4)
+        if not bf16:
+            assert np.all(np.abs(got["g"] - ref["g"]) <= 1e-2 * np.abs(ref["g"]).max())
+    spec = ModelSpec(arch=ARCH_LLAMA, bf16=False, **TINY)
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    p["labels"] = np.full_like(lab, -1)
+    got = run_gpu(spec, p, 2)
+    assert np.all(got["losses"] == 0) and np.all(got["g"] == 0)
+    assert all(np.array_equal(a, b.astype(np.float32)) for a, b in zip(got["B"], old_B(spec, p)))
+
+
 def test_argument_errors_are_reported_not_faulted():
     import ctypes as C
     import paper_2409_15520_b200 as zo
@@ -262,7 +283,7 @@ def test_argument_errors_are_reported_not_faulted():
     cfg = zo.make_config(spec)
     est = zo.Estimator(cfg)
     prob = zo.DeviceProblem(p, False)
-    for kw, code in [(dict(q=0), 1), (dict(q=spec.q + 1), 1), (dict(E=spec.E + 1), 1),
+    for kw, code in [(dict(q=0), 1), (dict(q=spec.q + 1), 1), (dict(E=spec.E + 1), 1), (dict(E=0), 1), (dict(S=0), 1),
                      (dict(S=spec.max_seq + 1), 1), (dict(eps=-1.0), 1), (dict(eps=float("nan")), 1)]:
         a = dict(E=spec.E, S=spec.S, seed=1, q=spec.q, eps=1e-3, lr=1e-3)
         a.update(kw)
