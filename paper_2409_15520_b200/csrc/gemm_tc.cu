@@ -70,7 +70,8 @@ struct Params {
   const bf16* res; int ldr; int res_mod;
   int act, swiglu;
   int has_lora;
-  int slab;                 // 1: the LoRA term is an extra k-block on the tensor cores
+  int slab;                 // 1: the LoRA term is one or two extra k-blocks on the tensor cores
+  int a_mod;                // > 0: the packed-U rows of tile row m are m % a_mod (input shared by all replicas)
   int kslot, khalf;         // K extent of one slot in the packed bf16 U, offset of its second copy
   bf16* pack_out; int pack_ld;  // down-projection: also write the packed bf16 U here (or null)
   int pack_r;
@@ -285,14 +286,15 @@ template <bool PAIR>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmU, const Params P) {
-  constexpr int STAGES = Cfg<PAIR>::STAGES;
+  // ring depth: one stage is given up when the LoRA term needs two generated k-blocks (rank > 32)
+  const int STAGES = PAIR ? Cfg<PAIR>::STAGES : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0);
   constexpr uint32_t STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
   constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
   constexpr int GROUP_M = PAIR ? 8 : 16;             // 16 row tiles of 128 per raster group
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   float* lbuf = (float*)(smem + STAGES * STAGE_BYTES);
-  Ctrl* ctrl = (Ctrl*)(smem + STAGES * STAGE_BYTES + SLAB_BYTES);
+  Ctrl* ctrl = (Ctrl*)(smem + Cfg<PAIR>::STAGES * STAGE_BYTES + SLAB_BYTES);
   const uint32_t tiles_base = smem_u32(smem);
   const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -306,7 +308,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int num_kb = (P.K + BK - 1) / BK;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < MAX_STAGES; ++s) {
       mbar_init(smem_u32(&ctrl->full[s]), 1);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
@@ -371,15 +373,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         const int lslot = PAIR ? -1 : tile_slot(P, brow0);
-        if (ok && lslot >= 0) {
-          // LoRA k-block: only the A operand (packed U) travels through the ring
+        for (int lkb = 0; ok && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued) {
+          // LoRA k-blocks: only the A operand (packed U) travels through the ring
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
           mbar_expect_tx(bar, A_BYTES);
-          tma_load_2d(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot, m0, bar);
-          ++issued;
+          tma_load_2d(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot + lkb * BK,
+                      P.a_mod > 0 ? m0 % P.a_mod : m0, bar);
         }
+        if (!ok) break;
       }
       if (!ok && (!PAIR || rank == 0)) {
         // abort: let the copies already issued land before the CTA goes away
@@ -421,18 +424,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           int tm, tn;
           tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
           if (tile_slot(P, tn * ncol_tile) >= 0) {
-            const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
-            if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
-                !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status)) { ok = false; break; }
-            ++ltiles;
-            tc_fence_after();
-            const uint64_t ad = smem_desc(tiles_base + s * STAGE_BYTES);
-            const uint64_t bd = smem_desc(tiles_base + STAGES * STAGE_BYTES);
+            for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++consumed) {
+              const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
+              if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
+                  (lkb == 0 && !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status))) { ok = false; break; }
+              tc_fence_after();
+              const uint64_t ad = smem_desc(tiles_base + s * STAGE_BYTES);
+              const uint64_t bd = smem_desc(tiles_base + STAGES * STAGE_BYTES + lkb * SLAB_BYTES);
 #pragma unroll
-            for (int k = 0; k < BK / 16; ++k)
-              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC, 1u);
-            tc_commit(smem_u32(&ctrl->empty[s]));
-            ++consumed;
+              for (int k = 0; k < BK / 16; ++k)
+                tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC,
+                       (uint32_t)((num_kb | lkb | k) != 0));
+              tc_commit(smem_u32(&ctrl->empty[s]));
+            }
+            if (!ok) break;
+            ++ltiles;
           }
         }
         if (ok) {
@@ -489,9 +495,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                       pack_bf16(bb[4][j], bb[5][j]), pack_bf16(bb[6][j], bb[7][j]));
           const uint4 vz = make_uint4(pack_bf16(zz[0][j], zz[1][j]), pack_bf16(zz[2][j], zz[3][j]),
                                       pack_bf16(zz[4][j], zz[5][j]), pack_bf16(zz[6][j], zz[7][j]));
-          const int cb = k0 >> 3, cz = (P.khalf + k0) >> 3;  // 16-byte chunk index along K
+          // 16-byte chunk index along K; K >= 64 lives in the second generated k-block
+          const int cb = k0 >> 3, pz = P.khalf + k0, cz = (pz & 63) >> 3;
           *reinterpret_cast<uint4*>(slab + n * 128 + ((cb ^ (n & 7)) << 4)) = vb;
-          *reinterpret_cast<uint4*>(slab + n * 128 + ((cz ^ (n & 7)) << 4)) = vz;
+          *reinterpret_cast<uint4*>(slab + (pz >> 6) * SLAB_BYTES + n * 128 + ((cz ^ (n & 7)) << 4)) = vz;
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
@@ -499,7 +506,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->lfull));
     };
     if (!PAIR && P.slab) {
-      for (int i = et; i < (int)(SLAB_BYTES / 16); i += EP_THREADS)
+      for (int i = et; i < (int)(SLAB_BYTES / 16) * (P.kslot / BK); i += EP_THREADS)
         reinterpret_cast<uint4*>(slab)[i] = make_uint4(0, 0, 0, 0);
       ep_bar();
       if (unit < num_tiles) gen_slab(unit);
@@ -528,6 +535,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const float* urow = P.has_lora ? P.L.U + (size_t)min(row, P.M - 1) * P.L.ldu : nullptr;
       const bool u_vec = P.has_lora && (P.L.ldu % 4 == 0) && (P.L.r % 4 == 0) && (((uintptr_t)P.L.U & 15) == 0);
       const int nchunk = ncol_tile / 32;
+      const bool acc_valid = num_kb > 0 || tile_slot(P, n0) >= 0;
       // The perturbed B columns are staged G columns at a time (the whole 256-column tile for
       // rank <= 16): one generation phase, two barriers, then barrier-free chunks.
       const int G = P.has_lora ? lora_phase_cols(P.L.r) : 256;
@@ -578,7 +586,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           continue;
         }
         uint32_t v[32];
-        tc_ld32(taddr + c * 32, v);
+        if (acc_valid) {
+          tc_ld32(taddr + c * 32, v);
+        } else {                                     // no k-block at all fed this tile: the sum is empty
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
+        }
         float f[32];
         if (P.swiglu) {
           uint32_t up[32];
@@ -756,16 +769,19 @@ static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, 
 }
 
 int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_sms) {
-  if (G.M <= 0 || G.N <= 0 || G.K <= 0) return 0;
+  if (G.M <= 0 || G.N <= 0 || G.K < 0 || (G.K == 0 && !(G.lora && G.lora_slab))) return 0;
   if (!g_encode) {
     const int e = gemm_tc_init();
     if (e) return e;
   }
   CUtensorMap tmA, tmB;
-  int e = make_map(&tmA, G.A, (uint64_t)G.K, (uint64_t)G.M, (uint64_t)G.lda);
-  if (e) return 10000 + e;
-  e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
-  if (e) return 10000 + e;
+  int e = 0;
+  if (G.K > 0) {
+    e = make_map(&tmA, G.A, (uint64_t)G.K, (uint64_t)G.M, (uint64_t)G.lda);
+    if (e) return 10000 + e;
+    e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
+    if (e) return 10000 + e;
+  }
   tc::Params P;
   P.M = G.M;
   P.N = G.swiglu ? G.N / 2 : G.N;
@@ -780,13 +796,15 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.kslot = G.kslot; P.khalf = G.khalf;
   P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
   CUtensorMap tmU = tmA;
+  P.a_mod = G.a_mod;
   if (P.slab) {
-    e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)G.M, (uint64_t)G.pack_ld);
+    e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)(G.a_mod > 0 ? G.a_mod : G.M), (uint64_t)G.pack_ld);
     if (e) return 10000 + e;
+    if (G.K == 0) tmA = tmB = tmU;                   // expansion only: no base product in this launch
   }
   P.status = status;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
-  if (G.cta_pair && P.M > tc::BM) {
+  if (G.cta_pair && P.M > tc::BM && G.K > 0) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
     static int max_clusters = 0;                       // co-resident pairs on this device
     cudaLaunchConfig_t cfg = {};

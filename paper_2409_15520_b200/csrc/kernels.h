@@ -38,6 +38,7 @@ struct GemmDesc {
   const void* pack_u;           // bf16 [M, pack_ld]: per slot [U | U] in kslot columns (second copy at khalf)
   void* pack_out;               // down-projection: write that packed copy here (bf16 [M, pack_ld]) or null
   int pack_ld, pack_r, kslot, khalf;
+  int a_mod;                    // > 0 with lora_slab: packed-U row of output row m is m % a_mod (shared input)
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
 };

@@ -113,7 +113,7 @@ Plan make_plan(const zo_config& c) {
     p.a = take(Mp * f * es);
     if (c.arch == ZO_ARCH_LLAMA && unfused_mlp) p.gu = take(Mp * 2 * f * es);
     p.U = take(Mp * (J ? J : 1) * 4);
-    if (c.precision == ZO_BF16) p.ub = take(Mp * (size_t)(n_targets(c) ? n_targets(c) : 1) * 64 * 2);  // packed bf16 U
+    if (c.precision == ZO_BF16) p.ub = take(Mp * (size_t)(n_targets(c) ? n_targets(c) : 1) * (c.lora_rank > 32 ? 128 : 64) * 2);  // packed bf16 U
     if (c.arch == ZO_ARCH_LLAMA) p.rope = take((size_t)c.max_seq * (d / c.n_heads) * 4);
     p.lab_idx = take(c.max_E * P * 4);
     p.lab_val = take(c.max_E * P * 4);
@@ -220,12 +220,12 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
 zo_status run_lora_down(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const void* X, int ldx,
                         const void* A, float* U, int rows, int K, int J, uint32_t* status, int n_sms,
                         int* launches, char* err, size_t errn, void* pack_out = nullptr, int pack_ld = 0,
-                        int pack_r = 0) {
+                        int pack_r = 0, int kslot = 64) {
   if (bf && !(flags & ZO_FLAG_SIMT_GEMM) && K % 8 == 0 && ldx % 8 == 0) {
     GemmDesc G{};
     G.A = X; G.lda = ldx; G.W = A; G.M = rows; G.N = J; G.K = K; G.out = U; G.ldo = J; G.out_f32 = 1;
     G.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
-    G.pack_out = pack_out; G.pack_ld = pack_ld; G.pack_r = pack_r; G.kslot = 64; G.khalf = 32;
+    G.pack_out = pack_out; G.pack_ld = pack_ld; G.pack_r = pack_r; G.kslot = kslot; G.khalf = kslot / 2;
     ProfScope ps(c, PC_LORA_DOWN, 2.0 * rows * (double)J * K);
     const int e = launch_gemm_tc(st, G, status, n_sms);
     if (e) {
@@ -265,11 +265,11 @@ inline int make_passes(int schedule, int q, Pass* out) {   // out holds up to 2q
 inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
   return bf && !(flags & ZO_FLAG_SIMT_GEMM) && Tp % 128 == 0 && width % 32 == 0;
 }
-// ... and as an extra k-block on the tensor cores?  (rank <= 32: both copies of U fit one
-// 64-deep block; every 256-column tile inside one section; single-CTA kernel)
+// ... and as extra k-blocks on the tensor cores?  (rank <= 64; every 256-column tile inside one
+// section; single-CTA kernel)
 inline bool slab_lora_ok(int bf, uint32_t flags, int Tp, int width, int r) {
   return fused_lora_ok(bf, flags, Tp, width) && !(flags & (ZO_FLAG_GEMM_PAIR | ZO_FLAG_LORA_EPILOGUE)) &&
-         width % 256 == 0 && r <= 32;
+         width % 256 == 0 && r <= 64;
 }
 
 zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* X,
@@ -371,11 +371,12 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = (uint32_t)(l * nt);
     L.rows_per_replica = Tp;
     L.rep_base = ps.base; L.rep_stride = ps.stride;
-    const bool slab = J && !first && slab_lora_ok(bf, cf.flags, Tp, d, r);
+    const bool slab = J && slab_lora_ok(bf, cf.flags, Tp, d, r);
+    const int kslot = r > 32 ? 128 : 64;       // K extent of one slot of the packed bf16 U
     void* ub = c->at<uint8_t>(c->plan.ub);
     if (J) {
       s = run_lora_down(c, st, bf, cf.flags, xn, d, lora->A[l], U, rows, d, J, status, c->n_sms,
-                        &c->launches, c->err, sizeof(c->err), slab ? ub : nullptr, nt * 64, r);
+                        &c->launches, c->err, sizeof(c->err), slab ? ub : nullptr, nt * kslot, r, kslot);
       if (s) return s;
     }
     GemmDesc G{};
@@ -385,10 +386,20 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       // first perturbed layer: one base product on the shared block, expanded to 2q outputs
       G.out = qkv0; G.ldo = 3 * d;
       GEMM(G);
-      PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
+      if (slab) {
+        // expansion on the tensor cores: no base k-blocks, only the LoRA block(s), base added as a
+        // residual that every replica shares
+        GemmDesc X{};
+        X.M = M; X.N = 3 * d; X.K = 0; X.out = qkv; X.ldo = 3 * d; X.res = qkv0; X.ldr = 3 * d; X.res_mod = Tp;
+        X.lora = &L; X.lora_slab = 1; X.pack_u = ub; X.pack_ld = nt * kslot; X.pack_r = r; X.kslot = kslot;
+        X.khalf = kslot / 2; X.a_mod = Tp; X.prof_class = PC_LORA_APPLY;
+        GEMM(X);
+      } else {
+        PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
+      }
     } else if (J && fused_lora_ok(bf, cf.flags, Tp, d)) {
       G.out = qkv; G.ldo = 3 * d; G.lora = &L;
-      if (slab) { G.lora_slab = 1; G.pack_u = ub; G.pack_ld = nt * 64; G.pack_r = r; G.kslot = 64; G.khalf = 32; }
+      if (slab) { G.lora_slab = 1; G.pack_u = ub; G.pack_ld = nt * kslot; G.pack_r = r; G.kslot = kslot; G.khalf = kslot / 2; }
       GEMM(G);
     } else {
       G.out = qkv; G.ldo = 3 * d;
@@ -711,7 +722,7 @@ size_t zo_mp_lora_scratch_bytes(int32_t precision, int32_t T, int32_t k_in, int3
   const size_t rows = x_replicated ? (size_t)2 * q * T : (size_t)T;
   size_t b = 256 + up(rows * r * 4, 256);
   if (!x_replicated) b += up((size_t)T * k_out * es, 256);
-  else if (precision == ZO_BF16) b += up(rows * 64 * 2, 256);   // packed bf16 U of the tensor-core LoRA block
+  if (precision == ZO_BF16) b += up(rows * 128 * 2, 256);       // packed bf16 U of the tensor-core LoRA blocks
   return b;
 }
 
@@ -740,14 +751,16 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   uint8_t* sp = (uint8_t*)scratch;
   uint32_t* status = (uint32_t*)sp;
   float* U = (float*)(sp + 256);
-  void* base = sp + 256 + up(rows * r * 4, 256);   // shared input: base product; replicated: packed U
+  void* base = sp + 256 + up(rows * r * 4, 256);   // shared input: base product X W^T
+  void* pack = (uint8_t*)base + (x_replicated ? 0 : up((size_t)T * k_out * (bf ? 2 : 4), 256));
   if (cudaMemsetAsync(status, 0, 4, st) != cudaSuccess) return ZO_ERR_CUDA;
-  const bool slab = x_replicated && slab_lora_ok(bf, flags, T, k_out, r);
-  if (slab && cudaMemsetAsync(base, 0, rows * 64 * 2, st) != cudaSuccess) return ZO_ERR_CUDA;
+  const bool slab = slab_lora_ok(bf, flags, T, k_out, r);
+  const int kslot = r > 32 ? 128 : 64;
+  if (slab && cudaMemsetAsync(pack, 0, rows * kslot * 2, st) != cudaSuccess) return ZO_ERR_CUDA;
   int launches = 0;
   char err[128];
   zo_status s = run_lora_down(nullptr, st, bf, flags, X, k_in, A, U, (int)rows, k_in, r, status, sms,
-                              &launches, err, sizeof(err), slab ? base : nullptr, 64, r);
+                              &launches, err, sizeof(err), slab ? pack : nullptr, kslot, r, kslot);
   if (s) return s;
   LoraDesc L{};
   L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
@@ -761,10 +774,19 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
     G.out = base;
     s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
     if (s) return s;
-    launch_lora_apply(st, bf, base, k_out, 1, Y, k_out, n, T, L, 1);
+    if (slab) {
+      GemmDesc X{};
+      X.M = n * T; X.N = k_out; X.K = 0; X.out = Y; X.ldo = k_out; X.res = base; X.ldr = k_out; X.res_mod = T;
+      X.lora = &L; X.lora_slab = 1; X.pack_u = pack; X.pack_ld = kslot; X.pack_r = r; X.kslot = kslot;
+      X.khalf = kslot / 2; X.a_mod = T;
+      s = run_gemm(nullptr, st, bf, flags, X, status, sms, &launches, err, sizeof(err));
+      if (s) return s;
+    } else {
+      launch_lora_apply(st, bf, base, k_out, 1, Y, k_out, n, T, L, 1);
+    }
   } else if (fused_lora_ok(bf, flags, T, k_out)) {
     G.out = Y; G.lora = &L;
-    if (slab) { G.lora_slab = 1; G.pack_u = base; G.pack_ld = 64; G.pack_r = r; G.kslot = 64; G.khalf = 32; }
+    if (slab) { G.lora_slab = 1; G.pack_u = pack; G.pack_ld = kslot; G.pack_r = r; G.kslot = kslot; G.khalf = kslot / 2; }
     s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
     if (s) return s;
   } else {

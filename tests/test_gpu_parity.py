@@ -199,10 +199,12 @@ def test_schedules_give_the_same_step(bf16):
         assert np.array_equal(a["losses"], b["losses"]) and np.array_equal(a["B"][0], b["B"][0])
 
 
-@pytest.mark.parametrize("r", [4, 16, 24, 32])
-def test_mp_lora_linear_tensor_core_lora_block(r):
-    """Replicated input, k_out a multiple of the 256-column tile, rank <= 32: the low-rank term
-    runs as an extra tensor-core k-block (bf16 U, B and k eps z).  Checked against the oracle's
+@pytest.mark.parametrize("x_replicated", [1, 0])
+@pytest.mark.parametrize("r", [4, 16, 24, 32, 48, 64])
+def test_mp_lora_linear_tensor_core_lora_block(r, x_replicated):
+    """k_out a multiple of the 256-column tile: the low-rank term runs as one (rank <= 32) or two
+    extra tensor-core k-blocks (bf16 U, B and k eps z); with a shared input the expansion to the 2q
+    outputs is a GEMM made of those blocks alone.  Checked against the oracle's
     layer, against the CUDA-core epilogue form, and for the visibility of the perturbation when
     |B| is 100x larger than eps."""
     import torch
@@ -211,19 +213,19 @@ def test_mp_lora_linear_tensor_core_lora_block(r):
     rng = np.random.default_rng(r)
     T, ki, ko, q, eps, scale, seed, tid = 256, 192, 768, 3, 1e-3, 2.0, 91, 5
     n = 2 * q
-    X = bf16_round(rng.standard_normal((n, T, ki)).astype(np.float32))
+    X = bf16_round(rng.standard_normal((n if x_replicated else 1, T, ki)).astype(np.float32))
     W = bf16_round(0.05 * rng.standard_normal((ko, ki)).astype(np.float32))
     A = bf16_round(0.05 * rng.standard_normal((r, ki)).astype(np.float32))
     B = (0.1 * rng.standard_normal((r, ko))).astype(np.float32)
     Bn = np.stack([B.astype(np.float64) + (1 if i % 2 == 0 else -1) * eps * perturbation(seed, tid, i // 2, (r, ko))
                    for i in range(n)])
-    ref = oracle.mp_lora_linear(X.astype(np.float64), W, None, A, Bn, scale)
+    ref = oracle.mp_lora_linear(np.broadcast_to(X, (n, T, ki)).astype(np.float64), W, None, A, Bn, scale)
     dev = lambda a: torch.tensor(a, device="cuda").to(torch.bfloat16).contiguous()
     Bd = torch.tensor(B, device="cuda")
     outs = {}
     for flags in (0, LORA_EPI):
-        Y = zo.mp_lora_linear(dev(X.reshape(-1, ki)), dev(W), None, dev(A), Bd, T, q, scale, seed, tid, eps, 1,
-                              flags=flags)
+        Y = zo.mp_lora_linear(dev(X.reshape(-1, ki)), dev(W), None, dev(A), Bd, T, q, scale, seed, tid, eps,
+                              x_replicated, flags=flags)
         outs[flags] = Y.float().cpu().numpy().astype(np.float64)
         assert np.max(np.abs(outs[flags] - ref)) < 2e-2 * np.max(np.abs(ref)), flags
     assert np.max(np.abs(outs[0] - outs[LORA_EPI])) < 1e-2 * np.max(np.abs(ref))
