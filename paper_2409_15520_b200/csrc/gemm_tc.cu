@@ -69,6 +69,8 @@ struct Params {
   const bf16* bias;
   const bf16* res; int ldr; int res_mod;
   int act, swiglu;
+  const float* rope_tab;    // non-null: rotate q and k (columns < rope_cols) in the epilogue
+  int rope_cols, rope_dh, rope_s, rope_tp;
   int has_lora;
   int slab;                 // 1: the LoRA term is one or two extra k-blocks on the tensor cores
   int a_mod;                // > 0: the packed-U rows of tile row m are m % a_mod (input shared by all replicas)
@@ -535,11 +537,61 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const float* urow = P.has_lora ? P.L.U + (size_t)min(row, P.M - 1) * P.L.ldu : nullptr;
       const bool u_vec = P.has_lora && (P.L.ldu % 4 == 0) && (P.L.r % 4 == 0) && (((uintptr_t)P.L.U & 15) == 0);
       const int nchunk = ncol_tile / 32;
+      const int po = P.rope_tab ? (P.rope_dh >> 6) : 0;          // 128 -> 2, 64 -> 1, <= 32 -> 0 (same chunk)
+      const int pshift = po == 1 ? 1 : 0;                      // keep both chunks of a pair with one warp
       const bool acc_valid = num_kb > 0 || tile_slot(P, n0) >= 0;
       // The perturbed B columns are staged G columns at a time (the whole 256-column tile for
       // rank <= 16): one generation phase, two barriers, then barrier-free chunks.
       const int G = P.has_lora ? lora_phase_cols(P.L.r) : 256;
       const int cpp = G / 32;                      // chunks per generation phase
+      // residual add and store of one 32-column chunk of this thread's row
+      auto emit = [&](int col0, float (&f)[32]) {
+        const bool full_chunk = col0 + 32 <= P.N;
+        // 16-byte vector accesses need the row pitch (and base) to keep rows 16-byte aligned
+        const bool vec_out = full_chunk && out_vec_ok;
+        if (P.res) {
+          const bf16* rp = P.res + (size_t)rrow * P.ldr + col0;
+          if (full_chunk && res_vec_ok) {
+#pragma unroll
+            for (int j8 = 0; j8 < 4; ++j8) {
+              float t[8];
+              unpack8(*reinterpret_cast<const uint4*>(rp + 8 * j8), t);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) f[8 * j8 + j] += t[j];
+            }
+          } else {
+            #pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < P.N) f[j] += to_f(rp[j]);
+          }
+        }
+        if (P.out_f32) {
+          float* op = (float*)P.out + (size_t)row * P.ldo + col0;
+          if (vec_out) {
+#pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4)
+              *reinterpret_cast<float4*>(op + 4 * j4) =
+                  make_float4(f[4 * j4], f[4 * j4 + 1], f[4 * j4 + 2], f[4 * j4 + 3]);
+          } else {
+            #pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < P.N) op[j] = f[j];
+          }
+        } else {
+          bf16* op = (bf16*)P.out + (size_t)row * P.ldo + col0;
+          if (vec_out) {
+#pragma unroll
+            for (int j8 = 0; j8 < 4; ++j8)
+              *reinterpret_cast<uint4*>(op + 8 * j8) =
+                  make_uint4(pack_bf16(f[8 * j8], f[8 * j8 + 1]), pack_bf16(f[8 * j8 + 2], f[8 * j8 + 3]),
+                             pack_bf16(f[8 * j8 + 4], f[8 * j8 + 5]), pack_bf16(f[8 * j8 + 6], f[8 * j8 + 7]));
+          } else {
+            #pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < P.N) op[j] = __float2bfloat16_rn(f[j]);
+          }
+        }
+      };
       for (int c = 0; c < nchunk; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= P.N) break;
@@ -579,12 +631,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               ep_bar();
             }
           }
-          if ((c & 1) != half) continue;           // the sibling warp's chunk
+          if (((c >> pshift) & 1) != half) continue;   // the sibling warp's chunk
           lslot = P.L.slot_of_sec[col0 / P.L.width];
           if (lslot >= 0) load_u16(urow + lslot * P.L.r, P.L.r, u_vec, u);
-        } else if ((c & 1) != half) {
+        } else if (((c >> pshift) & 1) != half) {
           continue;
         }
+        // rotary embedding fused here: the pair (j, j + dh/2) of a head sits po chunks apart
+        const bool rope_here = P.rope_tab != nullptr && col0 < P.rope_cols;
+        if (rope_here && po > 0 && (c % (2 * po)) >= po) continue;   // done with its low partner
         uint32_t v[32];
         if (acc_valid) {
           tc_ld32(taddr + c * 32, v);
@@ -642,7 +697,54 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int j = 0; j < 32; ++j) f[j] = fmaxf(f[j], 0.f);
           }
         }
+        float f2[32];
+        const bool have2 = rope_here && po > 0;
+        if (have2) {
+          uint32_t v2[32];
+          tc_ld32(taddr + (c + po) * 32, v2);
+          tc_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            f2[j] = __uint_as_float(v2[j]);
+            if (P.bias) f2[j] += to_f(P.bias[col0 + po * 32 + j]);
+          }
+        }
         if (!row_ok) continue;
+        if (rope_here) {
+          const int dh = P.rope_dh, hd = dh >> 1;
+          const float* cs = P.rope_tab + (size_t)((row % P.rope_tp) % P.rope_s) * dh;   // cos[0..hd) | sin[0..hd)
+          if (po > 0) {
+            const int h0 = col0 % dh;                  // head-local index of this chunk's first column (< hd)
+#pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4) {
+              const float4 c4 = *reinterpret_cast<const float4*>(cs + h0 + 4 * j4);
+              const float4 s4 = *reinterpret_cast<const float4*>(cs + hd + h0 + 4 * j4);
+              const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float x1 = f[4 * j4 + j], x2 = f2[4 * j4 + j];
+                f[4 * j4 + j] = x1 * cc[j] - x2 * ss[j];
+                f2[4 * j4 + j] = x2 * cc[j] + x1 * ss[j];
+              }
+            }
+          } else if (dh == 32) {                       // both halves inside this chunk
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float x1 = f[j], x2 = f[j + 16], cc = cs[j], sn = cs[16 + j];
+              f[j] = x1 * cc - x2 * sn;
+              f[j + 16] = x2 * cc + x1 * sn;
+            }
+          } else {                                     // dh = 16: two heads inside this chunk
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float x1 = f[16 * hh + j], x2 = f[16 * hh + j + 8], cc = cs[j], sn = cs[8 + j];
+                f[16 * hh + j] = x1 * cc - x2 * sn;
+                f[16 * hh + j + 8] = x2 * cc + x1 * sn;
+              }
+          }
+        }
         if (P.pack_out) {
           // bf16 copy of U for the tensor-core LoRA k-block: rank index k of slot t goes to
           // K = t*kslot + k and again to K = t*kslot + khalf + k
@@ -658,51 +760,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
         }
-        const bool full_chunk = col0 + 32 <= P.N;
-        // 16-byte vector accesses need the row pitch (and base) to keep rows 16-byte aligned
-        const bool vec_out = full_chunk && out_vec_ok;
-        if (P.res) {
-          const bf16* rp = P.res + (size_t)rrow * P.ldr + col0;
-          if (full_chunk && res_vec_ok) {
-#pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8) {
-              float t[8];
-              unpack8(*reinterpret_cast<const uint4*>(rp + 8 * j8), t);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) f[8 * j8 + j] += t[j];
-            }
-          } else {
-            #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < P.N) f[j] += to_f(rp[j]);
-          }
-        }
-        if (P.out_f32) {
-          float* op = (float*)P.out + (size_t)row * P.ldo + col0;
-          if (vec_out) {
-#pragma unroll
-            for (int j4 = 0; j4 < 8; ++j4)
-              *reinterpret_cast<float4*>(op + 4 * j4) =
-                  make_float4(f[4 * j4], f[4 * j4 + 1], f[4 * j4 + 2], f[4 * j4 + 3]);
-          } else {
-            #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < P.N) op[j] = f[j];
-          }
-        } else {
-          bf16* op = (bf16*)P.out + (size_t)row * P.ldo + col0;
-          if (vec_out) {
-#pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8)
-              *reinterpret_cast<uint4*>(op + 8 * j8) =
-                  make_uint4(pack_bf16(f[8 * j8], f[8 * j8 + 1]), pack_bf16(f[8 * j8 + 2], f[8 * j8 + 3]),
-                             pack_bf16(f[8 * j8 + 4], f[8 * j8 + 5]), pack_bf16(f[8 * j8 + 6], f[8 * j8 + 7]));
-          } else {
-            #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < P.N) op[j] = __float2bfloat16_rn(f[j]);
-          }
-        }
+        emit(col0, f);
+        if (have2) emit(col0 + po * 32, f2);
       }
       // accumulator buffer drained: hand it back to the MMA warp
       tc_fence_before();
@@ -797,6 +856,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
   CUtensorMap tmU = tmA;
   P.a_mod = G.a_mod;
+  P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp;
   if (P.slab) {
     e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)(G.a_mod > 0 ? G.a_mod : G.M), (uint64_t)G.pack_ld);
     if (e) return 10000 + e;

@@ -38,6 +38,9 @@ struct GemmDesc {
   const void* pack_u;           // bf16 [M, pack_ld]: per slot [U | U] in kslot columns (second copy at khalf)
   void* pack_out;               // down-projection: write that packed copy here (bf16 [M, pack_ld]) or null
   int pack_ld, pack_r, kslot, khalf;
+  const float* rope_tab;        // tensor-core kernel: rotate columns < rope_cols (q, k) in the epilogue; table
+                                // rows cos[0..dh/2) | sin[0..dh/2); position of row m = (m % rope_tp) % rope_s
+  int rope_cols, rope_dh, rope_s, rope_tp;
   int a_mod;                    // > 0 with lora_slab: packed-U row of output row m is m % a_mod (shared input)
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile

@@ -379,6 +379,13 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
                         &c->launches, c->err, sizeof(c->err), slab ? ub : nullptr, nt * kslot, r, kslot);
       if (s) return s;
     }
+    // The rotary embedding rides in the epilogue of whichever tensor-core GEMM writes q|k|v last.
+    bool rope_done = opt;
+    auto with_rope = [&](GemmDesc& D) {
+      D.rope_tab = rope; D.rope_cols = 2 * d; D.rope_dh = d / H; D.rope_s = S; D.rope_tp = Tp;
+      rope_done = true;
+    };
+    const bool tcore = bf && !(cf.flags & ZO_FLAG_SIMT_GEMM);
     GemmDesc G{};
     G.A = xn; G.lda = d; G.W = W.w_qkv; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
     G.prof_class = PC_GEMM_QKV;
@@ -393,6 +400,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
         X.M = M; X.N = 3 * d; X.K = 0; X.out = qkv; X.ldo = 3 * d; X.res = qkv0; X.ldr = 3 * d; X.res_mod = Tp;
         X.lora = &L; X.lora_slab = 1; X.pack_u = ub; X.pack_ld = nt * kslot; X.pack_r = r; X.kslot = kslot;
         X.khalf = kslot / 2; X.a_mod = Tp; X.prof_class = PC_LORA_APPLY;
+        if (!opt) with_rope(X);
         GEMM(X);
       } else {
         PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
@@ -400,13 +408,15 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     } else if (J && fused_lora_ok(bf, cf.flags, Tp, d)) {
       G.out = qkv; G.ldo = 3 * d; G.lora = &L;
       if (slab) { G.lora_slab = 1; G.pack_u = ub; G.pack_ld = nt * kslot; G.pack_r = r; G.kslot = kslot; G.khalf = kslot / 2; }
+      if (slab && !opt) with_rope(G);
       GEMM(G);
     } else {
       G.out = qkv; G.ldo = 3 * d;
+      if (!J && tcore && !opt) with_rope(G);
       GEMM(G);
       if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
-    if (!opt) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
+    if (!rope_done) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
     if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
       PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, E, S, Tp, d, H));
     } else {

@@ -255,6 +255,23 @@ def test_degenerate_steps():
     assert update_rel_err(spec, p0, got["B"], ref["B"]) < 2e-3
 
 
+@pytest.mark.parametrize("heads,targets", [(2, TARGET_Q | TARGET_V), (4, TARGET_Q | TARGET_K | TARGET_V),
+                                           (8, TARGET_V), (16, TARGET_Q | TARGET_V), (4, 0)])
+def test_llama_bf16_fused_rope_all_head_dims(heads, targets):
+    """d = 256 (one 256-column tile per section): the rotary embedding is applied in the epilogue of the
+    q|k|v GEMM for head_dim 128, 64 (pairs in different 32-column chunks), 32 and 16 (pairs inside a
+    chunk), with adapted q/k/v sections in any combination and with no adapted section at all."""
+    spec = ModelSpec(arch=ARCH_LLAMA, bf16=True, lora_targets=targets,
+                     **{**TINY, "d_model": 256, "n_heads": heads, "d_ffn": 264, "vocab": 517, "S": 72,
+                        "E": 2, "max_seq": 72, "q": 2, "n_layers": 2, "lora_rank": 8})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 43)
+    got = run_gpu(spec, p, 43)
+    simt = run_gpu(spec, p, 43, flags=SIMT)
+    assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
+    assert np.allclose(got["losses"], simt["losses"], rtol=3e-3, atol=0), (got["losses"], simt["losses"])
+
+
 def test_maximum_queries_and_no_labelled_positions():
     """q = 32 (64 replicas, the largest the library accepts) on a small model in both precisions;
     a batch without any labelled position gives zero losses and leaves B untouched."""
