@@ -544,27 +544,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // rank <= 16): one generation phase, two barriers, then barrier-free chunks.
       const int G = P.has_lora ? lora_phase_cols(P.L.r) : 256;
       const int cpp = G / 32;                      // chunks per generation phase
-      // residual add and store of one 32-column chunk of this thread's row
+      // residual add (before any rotation: the rotary embedding applies to the finished projection)
+      auto add_res = [&](int col0, float (&f)[32]) {
+        if (!P.res) return;
+        const bool full_chunk = col0 + 32 <= P.N;
+        const bf16* rp = P.res + (size_t)rrow * P.ldr + col0;
+        if (full_chunk && res_vec_ok) {
+#pragma unroll
+          for (int j8 = 0; j8 < 4; ++j8) {
+            float t[8];
+            unpack8(*reinterpret_cast<const uint4*>(rp + 8 * j8), t);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) f[8 * j8 + j] += t[j];
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (col0 + j < P.N) f[j] += to_f(rp[j]);
+        }
+      };
+      // store of one 32-column chunk of this thread's row
       auto emit = [&](int col0, float (&f)[32]) {
         const bool full_chunk = col0 + 32 <= P.N;
         // 16-byte vector accesses need the row pitch (and base) to keep rows 16-byte aligned
         const bool vec_out = full_chunk && out_vec_ok;
-        if (P.res) {
-          const bf16* rp = P.res + (size_t)rrow * P.ldr + col0;
-          if (full_chunk && res_vec_ok) {
-#pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8) {
-              float t[8];
-              unpack8(*reinterpret_cast<const uint4*>(rp + 8 * j8), t);
-#pragma unroll
-              for (int j = 0; j < 8; ++j) f[8 * j8 + j] += t[j];
-            }
-          } else {
-            #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < P.N) f[j] += to_f(rp[j]);
-          }
-        }
         if (P.out_f32) {
           float* op = (float*)P.out + (size_t)row * P.ldo + col0;
           if (vec_out) {
@@ -710,6 +713,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         if (!row_ok) continue;
+        add_res(col0, f);
+        if (have2) add_res(col0 + po * 32, f2);
         if (rope_here) {
           const int dh = P.rope_dh, hd = dh >> 1;
           const float* cs = P.rope_tab + (size_t)((row % P.rope_tp) % P.rope_s) * dh;   // cos[0..hd) | sin[0..hd)
