@@ -704,8 +704,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool have2 = rope_here && po > 0;
         if (have2) {
           uint32_t v2[32];
-          tc_ld32(taddr + (c + po) * 32, v2);
-          tc_ld_wait();
+          if (acc_valid) {
+            tc_ld32(taddr + (c + po) * 32, v2);
+            tc_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v2[j] = 0u;
+          }
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             f2[j] = __uint_as_float(v2[j]);
