@@ -27,7 +27,7 @@ def draw_z(spec, p, seed, i):
     zs = []
     for l, L in enumerate(p["layers"]):
         zs.append(np.stack([perturbation(seed, l * nt + t, i, L["B"].shape[1:])
-                            for t in range(nt)]))
+                            for t in range(nt)]) if nt else np.zeros(np.shape(L["B"])))
     return zs
 
 
