@@ -67,6 +67,15 @@ enum { ZO_ARCH_LINEAR = 0, ZO_ARCH_OPT = 1, ZO_ARCH_LLAMA = 2 };
 enum { ZO_FP32 = 0, ZO_BF16 = 1 };
 enum { ZO_LOSS_MSE = 0, ZO_LOSS_CE_FULL_VOCAB = 1, ZO_LOSS_CE_LABEL_WORDS = 2 };
 enum { ZO_TARGET_Q = 1, ZO_TARGET_K = 2, ZO_TARGET_V = 4 };
+/* Storage of the four frozen linear weights of a decoder block (w_qkv, w_o, w_fc1, w_fc2), after the
+ * paper's appendix "MobiZO with weight-only quantization" (Q-LoRA style): stored low-bit, dequantised
+ * to the compute type once per forward pass, i.e. once per step for all 2q replicas.
+ *   ZO_W_NATIVE  element type of `precision`
+ *   ZO_W_INT8    int8 codes [k_out, k_in] + float32 scale [k_out]:      w = code * scale[row]
+ *   ZO_W_NF4     4-bit NormalFloat codes, two per byte (even element in the high nibble), uint8
+ *                [k_out, k_in/2] + float32 absmax [k_out, k_in/64]:     w = level[code] * absmax[row, col/64]
+ * The dequantised value is rounded once to the compute type. */
+enum { ZO_W_NATIVE = 0, ZO_W_INT8 = 1, ZO_W_NF4 = 2 };
 /* flags: ZO_FLAG_SIMT_GEMM routes every bf16 GEMM (and attention) through the plain
  * CUDA-core validation kernels instead of the tensor-core ones (cross-checking only). */
 enum { ZO_FLAG_SIMT_GEMM = 1,
@@ -104,6 +113,7 @@ typedef struct zo_config {
   float rope_theta;
   int32_t tie_lm_head; /* 1: LM head = token embedding                               */
   uint32_t flags;
+  int32_t weight_format; /* ZO_W_*; quantised formats need k_in % 64 == 0 (NF4) and decoders   */
 } zo_config;
 
 /* Frozen tensors of one decoder block (device pointers; element type per precision).
@@ -117,6 +127,8 @@ typedef struct zo_layer_weights {
   const void* norm2_g; const void* norm2_b;
   const void* w_fc1;   const void* b_fc1;
   const void* w_fc2;   const void* b_fc2;  /* [d, d_ffn], [d] */
+  /* ZO_W_INT8 / ZO_W_NF4 only: float32 scales of the four weights above (else NULL) */
+  const float* s_qkv; const float* s_o; const float* s_fc1; const float* s_fc2;
 } zo_layer_weights;
 
 typedef struct zo_weights {
@@ -207,7 +219,7 @@ ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 enum { ZO_PROF_GEMM_TC = 0, ZO_PROF_GEMM_SIMT, ZO_PROF_ATTENTION, ZO_PROF_NORM, ZO_PROF_LORA_DOWN,
        ZO_PROF_LORA_APPLY, ZO_PROF_ROPE, ZO_PROF_SWIGLU, ZO_PROF_LOSS, ZO_PROF_UPDATE,
        ZO_PROF_MISC, ZO_PROF_GEMM_QKV, ZO_PROF_GEMM_O, ZO_PROF_GEMM_FC1, ZO_PROF_GEMM_FC2,
-       ZO_PROF_GEMM_HEAD, ZO_PROFILE_CLASSES };
+       ZO_PROF_GEMM_HEAD, ZO_PROF_DEQUANT, ZO_PROFILE_CLASSES };
 ZO_API zo_status zo_profile_enable(zo_ctx* ctx, int32_t on);
 ZO_API zo_status zo_profile_read(zo_ctx* ctx, double* host_ms, double* host_flops,
                                  int32_t* host_launches);
@@ -220,6 +232,12 @@ ZO_API const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo
  * NULL) of tensor `tensor_id`, query `query`.  Asynchronous on `cuda_stream`. */
 ZO_API zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, uint32_t query,
                           int64_t n, uint32_t* dev_u32, float* dev_z);
+
+/* The weight decoder on its own (for bit-level checks): out [rows, k_in] in the element type of
+ * `precision` from codes and scales in the given ZO_W_INT8 / ZO_W_NF4 format.  Asynchronous. */
+ZO_API zo_status zo_dequantize(void* cuda_stream, int32_t weight_format, int32_t precision,
+                               const void* codes, const float* scale, void* out, int32_t rows,
+                               int32_t k_in);
 
 /* The MP-LoRA linear on its own ("MP-LoRA" paragraph, layer equation):
  *   Y[n] = X[n or shared] W^T + bias + scale * (X A^T) (B + k_n eps z_{n>>1}),  n < 2q.

@@ -12,6 +12,8 @@ library in the tests.
 """
 import numpy as np
 
+from .quant import weight as _wq
+
 ARCH_LINEAR, ARCH_OPT, ARCH_LLAMA = 0, 1, 2
 LOSS_MSE, LOSS_CE_FULL, LOSS_CE_LABEL_WORDS = 0, 1, 2
 
@@ -75,9 +77,10 @@ def _section_lora(spec, L, Bn_layer, d):
 def _qkv(spec, L, x, Bn_layer):
     d = spec.d_model
     lora = _section_lora(spec, L, Bn_layer, d)
+    Wqkv = _wq(L["w_qkv"], spec.bf16)
     outs = []
     for sec in range(3):
-        W = L["w_qkv"][sec * d:(sec + 1) * d]
+        W = Wqkv[sec * d:(sec + 1) * d]
         b = L["b_qkv"][sec * d:(sec + 1) * d] if "b_qkv" in L else None
         if sec in lora:
             A, Bn = lora[sec]
@@ -108,20 +111,20 @@ def decoder_hidden(spec, p, Bn, tokens):
         if spec.arch == ARCH_LLAMA:
             q, k = _rope(q, spec.rope_theta), _rope(k, spec.rope_theta)
         ctx = _causal_attention(q, k, v).reshape(n, E * S, d)
-        o = ctx @ _f64(L["w_o"]).T
+        o = ctx @ _wq(L["w_o"], spec.bf16).T
         if "b_o" in L:
             o = o + _f64(L["b_o"])
         h = h + o
         if spec.arch == ARCH_OPT:
             x = _layer_norm(h, L["norm2_g"], L["norm2_b"], spec.norm_eps)
-            a = np.maximum(x @ _f64(L["w_fc1"]).T + _f64(L["b_fc1"]), 0.0)
-            h = h + a @ _f64(L["w_fc2"]).T + _f64(L["b_fc2"])
+            a = np.maximum(x @ _wq(L["w_fc1"], spec.bf16).T + _f64(L["b_fc1"]), 0.0)
+            h = h + a @ _wq(L["w_fc2"], spec.bf16).T + _f64(L["b_fc2"])
         else:
             x = _rms_norm(h, L["norm2_g"], spec.norm_eps)
-            gu = x @ _f64(L["w_fc1"]).T
+            gu = x @ _wq(L["w_fc1"], spec.bf16).T
             g, u = gu[..., :spec.d_ffn], gu[..., spec.d_ffn:]
             a = g / (1.0 + np.exp(-g)) * u                 # SiLU(gate) * up
-            h = h + a @ _f64(L["w_fc2"]).T
+            h = h + a @ _wq(L["w_fc2"], spec.bf16).T
     return h
 
 

@@ -36,7 +36,7 @@ class ZoConfig(C.Structure):
                 ("lora_scale", C.c_float), ("lora_targets", C.c_uint32),
                 ("label_words", C.c_int32 * 2), ("max_q", C.c_int32), ("max_E", C.c_int32),
                 ("max_labelled", C.c_int32), ("norm_eps", C.c_float), ("rope_theta", C.c_float),
-                ("tie_lm_head", C.c_int32), ("flags", C.c_uint32)]
+                ("tie_lm_head", C.c_int32), ("flags", C.c_uint32), ("weight_format", C.c_int32)]
 
 
 _LAYER_FIELDS = ["norm1_g", "norm1_b", "w_qkv", "b_qkv", "w_o", "b_o", "norm2_g", "norm2_b",
@@ -44,7 +44,7 @@ _LAYER_FIELDS = ["norm1_g", "norm1_b", "w_qkv", "b_qkv", "w_o", "b_o", "norm2_g"
 
 
 class ZoLayerWeights(C.Structure):
-    _fields_ = [(f, C.c_void_p) for f in _LAYER_FIELDS]
+    _fields_ = [(f, C.c_void_p) for f in _LAYER_FIELDS] + [(f, C.c_void_p) for f in ("s_qkv", "s_o", "s_fc1", "s_fc2")]
 
 
 class ZoWeights(C.Structure):
@@ -81,10 +81,12 @@ zo_profile_enable = _sig("zo_profile_enable", C.c_int, [C.c_void_p, C.c_int32])
 zo_profile_read = _sig("zo_profile_read", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p])
 PROFILE_CLASSES = ["gemm_tc", "gemm_simt", "attention", "norm", "lora_down", "lora_apply", "rope",
                    "swiglu", "loss", "update", "misc", "gemm_qkv", "gemm_o", "gemm_fc1", "gemm_fc2",
-                   "gemm_head"]
+                   "gemm_head", "dequant"]
 zo_last_error = _sig("zo_last_error", C.c_char_p, [C.c_void_p])
 zo_perturbation = _sig("zo_perturbation", C.c_int, [C.c_void_p, C.c_uint64, C.c_uint32, C.c_uint32,
                                                     C.c_int64, C.c_void_p, C.c_void_p])
+zo_dequantize = _sig("zo_dequantize", C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                                C.c_void_p, C.c_int32, C.c_int32])
 zo_mp_lora_scratch_bytes = _sig("zo_mp_lora_scratch_bytes", C.c_size_t, [C.c_int32] * 7)
 zo_mp_lora_linear = _sig("zo_mp_lora_linear", C.c_int, [
     C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -99,8 +101,11 @@ zo_mp_lora_linear_static = _sig("zo_mp_lora_linear_static", C.c_int, [
 STATIC_SCRATCH_BYTES = 16 << 20
 
 
+WEIGHT_FORMATS = {None: 0, "native": 0, "int8": 1, "nf4": 2}
+
+
 def make_config(spec, *, max_q=None, max_E=None, max_seq=None, max_labelled=None, flags=0,
-                precision=None) -> ZoConfig:
+                precision=None, weight_format=None) -> ZoConfig:
     """zo_config from a shape record with the attribute names of workloads.ModelSpec."""
     c = ZoConfig()
     c.struct_size = C.sizeof(ZoConfig)
@@ -115,6 +120,7 @@ def make_config(spec, *, max_q=None, max_E=None, max_seq=None, max_labelled=None
     c.max_labelled = max_labelled or spec.n_labelled
     c.norm_eps, c.rope_theta = spec.norm_eps, spec.rope_theta
     c.tie_lm_head, c.flags = int(spec.tie_lm_head), flags
+    c.weight_format = WEIGHT_FORMATS[weight_format]
     return c
 
 
@@ -154,7 +160,15 @@ class DeviceProblem:
             self._A, self.B = [], []
             for l, L in enumerate(p["layers"]):
                 for f in _LAYER_FIELDS:
-                    setattr(self._layers[l], f, _ptr(self._up(L.get(f))))
+                    v = L.get(f)
+                    if isinstance(v, dict):       # quantised record: codes + float32 scales
+                        codes = torch.tensor(v["codes"], device=device).contiguous()
+                        scale = torch.tensor(v["scale"], dtype=torch.float32, device=device).contiguous()
+                        self._keep += [codes, scale]
+                        setattr(self._layers[l], f, _ptr(codes))
+                        setattr(self._layers[l], "s_" + f[2:], _ptr(scale))
+                    else:
+                        setattr(self._layers[l], f, _ptr(self._up(v)))
                 self._A.append(self._up(L["A"]) if L["A"].size else None)
                 self.B.append(torch.tensor(L["B"], dtype=torch.float32, device=device).contiguous()
                               if L["B"].size else None)

@@ -908,6 +908,57 @@ void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses
   zo_update_kernel<<<grid, 128, 0, st>>>(D, losses, g, q, eps, lr, seed, status, write_g);
 }
 
+// =========================================================================================
+// Weight-only dequantisation, once per forward pass for all replicas (appendix "MobiZO with
+// weight-only quantization").  16 elements per thread; one fp32 product, one rounding.
+// =========================================================================================
+__constant__ float c_nf4[16] = {-1.0f, -0.6961928009986877f, -0.5250730514526367f, -0.39491748809814453f,
+                                -0.28444138169288635f, -0.18477343022823334f, -0.09105003625154495f, 0.0f,
+                                0.07958029955625534f, 0.16093020141124725f, 0.24611230194568634f,
+                                0.33791524171829224f, 0.44070982933044434f, 0.5626170039176941f,
+                                0.7229568362236023f, 1.0f};
+template <typename T>
+__global__ void dequant_kernel(int fmt, const uint8_t* __restrict__ codes, const float* __restrict__ scale,
+                               T* __restrict__ out, long long total16, int K) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // group of 16 elements
+  if (i >= total16) return;
+  const long long e0 = i * 16;
+  const long long row = e0 / K;
+  const int col = (int)(e0 - row * K);
+  float w[16];
+  if (fmt == 1) {
+    const uint4 raw = *reinterpret_cast<const uint4*>(codes + e0);
+    const int8_t* c = reinterpret_cast<const int8_t*>(&raw);
+    const float s = scale[row];
+#pragma unroll
+    for (int j = 0; j < 16; ++j) w[j] = (float)c[j] * s;
+  } else {
+    const uint2 raw = *reinterpret_cast<const uint2*>(codes + e0 / 2);
+    const uint8_t* c = reinterpret_cast<const uint8_t*>(&raw);
+    const float s = scale[row * (K / 64) + col / 64];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      w[2 * j] = c_nf4[c[j] >> 4] * s;
+      w[2 * j + 1] = c_nf4[c[j] & 15] * s;
+    }
+  }
+  __align__(16) T o[16];
+#pragma unroll
+  for (int j = 0; j < 16; ++j) o[j] = from_f<T>(w[j]);
+  uint4* dst = reinterpret_cast<uint4*>(out + e0);
+  const uint4* srcv = reinterpret_cast<const uint4*>(o);
+#pragma unroll
+  for (int j = 0; j < (int)(16 * sizeof(T) / 16); ++j) dst[j] = srcv[j];
+}
+void launch_dequant(cudaStream_t st, int bf, int fmt, const void* codes, const float* scale, void* out,
+                    int rows, int K) {
+  const long long total16 = (long long)rows * K / 16;
+  if (total16 <= 0) return;
+  const unsigned grid = (unsigned)((total16 + 255) / 256);
+  if (bf) dequant_kernel<bf16><<<grid, 256, 0, st>>>(fmt, (const uint8_t*)codes, scale, (bf16*)out, total16, K);
+  else dequant_kernel<float><<<grid, 256, 0, st>>>(fmt, (const uint8_t*)codes, scale, (float*)out, total16, K);
+}
+
 __global__ void perturbation_kernel(uint64_t seed, uint32_t tensor, uint32_t query, long long n,
                                     uint32_t* u32, float* z) {
   const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;

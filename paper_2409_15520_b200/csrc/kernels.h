@@ -101,6 +101,10 @@ void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses
 void launch_perturbation(cudaStream_t st, uint64_t seed, uint32_t tensor, uint32_t query,
                          long long n, uint32_t* u32, float* z);
 
+// Weight-only dequantisation (fmt 1 = int8 per-row scale, 2 = NF4 with 64-element blocks) to T.
+void launch_dequant(cudaStream_t st, int bf, int fmt, const void* codes, const float* scale, void* out,
+                    int rows, int K);
+
 // --- GEMMs ---------------------------------------------------------------------------------
 void launch_gemm_simt(cudaStream_t st, int bf, const GemmDesc& G);
 // bf16 tensor-core GEMM (tcgen05 + TMEM + TMA).  Returns a CUDA error code (0 = ok).

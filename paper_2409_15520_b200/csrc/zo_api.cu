@@ -18,7 +18,7 @@ char g_init_error[256] = "";
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
-      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, total;
+      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, total;
 };
 
 inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -48,7 +48,9 @@ zo_status check_config(const zo_config* c, char* err, size_t errn) {
   if (c->d_model < 1) BAD(ZO_ERR_INVALID_ARG, "d_model must be >= 1");
   if (!isfinite(c->lora_scale)) BAD(ZO_ERR_INVALID_ARG, "lora_scale not finite");
   const bool bf = c->precision == ZO_BF16;
+  if (c->weight_format < ZO_W_NATIVE || c->weight_format > ZO_W_NF4) BAD(ZO_ERR_INVALID_ARG, "bad weight_format");
   if (c->arch == ZO_ARCH_LINEAR) {
+    if (c->weight_format != ZO_W_NATIVE) BAD(ZO_ERR_UNSUPPORTED, "quantised weights are for decoders");
     if (c->loss_kind != ZO_LOSS_MSE) BAD(ZO_ERR_INVALID_ARG, "ZO_ARCH_LINEAR requires ZO_LOSS_MSE");
     if (c->d_out < 1) BAD(ZO_ERR_INVALID_ARG, "d_out must be >= 1");
     if (c->d_out % 4) BAD(ZO_ERR_UNSUPPORTED, "d_out must be a multiple of 4");
@@ -72,6 +74,8 @@ zo_status check_config(const zo_config* c, char* err, size_t errn) {
     for (int i = 0; i < 2; ++i)
       if (c->label_words[i] < 0 || c->label_words[i] >= c->vocab)
         BAD(ZO_ERR_INVALID_ARG, "label word out of the vocabulary");
+  if (c->weight_format != ZO_W_NATIVE && (c->d_model % 64 || c->d_ffn % 64))
+    BAD(ZO_ERR_UNSUPPORTED, "quantised weights need d_model and d_ffn to be multiples of 64");
   if (!(c->norm_eps > 0.f)) BAD(ZO_ERR_INVALID_ARG, "norm_eps must be > 0");
   if (c->arch == ZO_ARCH_LLAMA && !(c->rope_theta > 1.f)) BAD(ZO_ERR_INVALID_ARG, "rope_theta must be > 1");
   return ZO_OK;
@@ -124,6 +128,12 @@ Plan make_plan(const zo_config& c) {
     if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
     p.rowloss = take(Mh * 8);
     p.rowloss_pass = take(Mh * 8);
+    if (c.weight_format != ZO_W_NATIVE) {   // one dequantised weight at a time
+      size_t big = 3 * d * d;
+      const size_t f1 = (c.arch == ZO_ARCH_LLAMA ? 2 : 1) * f * d;
+      if (f1 > big) big = f1;
+      p.wdq = take(big * es);
+    }
   }
   p.losses = take(n * 4);
   p.losses_d = take(n * 8);
@@ -137,7 +147,7 @@ Plan make_plan(const zo_config& c) {
 
 enum { PC_GEMM_TC = 0, PC_GEMM_SIMT, PC_ATTN, PC_NORM, PC_LORA_DOWN, PC_LORA_APPLY, PC_ROPE,
        PC_SWIGLU, PC_LOSS, PC_UPDATE, PC_MISC, PC_GEMM_QKV, PC_GEMM_O, PC_GEMM_FC1, PC_GEMM_FC2,
-       PC_GEMM_HEAD, PC_COUNT };
+       PC_GEMM_HEAD, PC_DEQUANT, PC_COUNT };
 static_assert(PC_COUNT == ZO_PROFILE_CLASSES, "profile classes out of sync with zo.h");
 
 struct ProfRec { int cat; double flops; cudaEvent_t e0, e1; };
@@ -379,6 +389,13 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
                         &c->launches, c->err, sizeof(c->err), slab ? ub : nullptr, nt * kslot, r, kslot);
       if (s) return s;
     }
+    // quantised storage: decode each weight right before its GEMM, once for all replicas of the pass
+    void* wdq = c->at<uint8_t>(c->plan.wdq);
+    auto weight = [&](const void* wq, const float* sc, int n_rows, int k_in) -> const void* {
+      if (cf.weight_format == ZO_W_NATIVE) return wq;
+      PROF(PC_DEQUANT, 0.0, launch_dequant(st, bf, cf.weight_format, wq, sc, wdq, n_rows, k_in));
+      return wdq;
+    };
     // The rotary embedding rides in the epilogue of whichever tensor-core GEMM writes q|k|v last.
     bool rope_done = opt;
     auto with_rope = [&](GemmDesc& D) {
@@ -387,7 +404,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     };
     const bool tcore = bf && !(cf.flags & ZO_FLAG_SIMT_GEMM);
     GemmDesc G{};
-    G.A = xn; G.lda = d; G.W = W.w_qkv; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
+    G.A = xn; G.lda = d; G.W = weight(W.w_qkv, W.s_qkv, 3 * d, d); G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
     G.prof_class = PC_GEMM_QKV;
     if (first) {
       // first perturbed layer: one base product on the shared block, expanded to 2q outputs
@@ -423,12 +440,12 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H));
     }
     GemmDesc O{};
-    O.A = x; O.lda = d; O.W = W.w_o; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
+    O.A = x; O.lda = d; O.W = weight(W.w_o, W.s_o, d, d); O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
     O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0; O.prof_class = PC_GEMM_O;
     GEMM(O);
     PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0));
     GemmDesc F1{};
-    F1.A = x; F1.lda = d; F1.W = W.w_fc1; F1.M = M; F1.K = d; F1.bias = W.b_fc1; F1.prof_class = PC_GEMM_FC1;
+    F1.A = x; F1.lda = d; F1.W = weight(W.w_fc1, W.s_fc1, opt ? f : 2 * f, d); F1.M = M; F1.K = d; F1.bias = W.b_fc1; F1.prof_class = PC_GEMM_FC1;
     if (opt) {
       F1.N = f; F1.out = a; F1.ldo = f; F1.act = ACT_RELU;
       GEMM(F1);
@@ -441,7 +458,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(F1);
     }
     GemmDesc F2{};
-    F2.A = a; F2.lda = f; F2.W = W.w_fc2; F2.M = M; F2.N = d; F2.K = f; F2.out = h; F2.ldo = d;
+    F2.A = a; F2.lda = f; F2.W = weight(W.w_fc2, W.s_fc2, d, f); F2.M = M; F2.N = d; F2.K = f; F2.out = h; F2.ldo = d;
     F2.bias = W.b_fc2; F2.res = h; F2.ldr = d; F2.prof_class = PC_GEMM_FC2;
     GEMM(F2);
   }
@@ -512,6 +529,8 @@ zo_status check_step_args(zo_ctx* c, const zo_weights* w, const zo_lora* lora, c
     if (cf.arch == ZO_ARCH_OPT && (!W.norm1_b || !W.b_qkv || !W.b_o || !W.norm2_b || !W.b_fc1 || !W.b_fc2))
       return fail(c, ZO_ERR_INVALID_ARG, "OPT layers need every bias");
     if (c->nt && (!lora->A[l] || !lora->B[l])) return fail(c, ZO_ERR_INVALID_ARG, "null LoRA tensor");
+    if (cf.weight_format != ZO_W_NATIVE && (!W.s_qkv || !W.s_o || !W.s_fc1 || !W.s_fc2))
+      return fail(c, ZO_ERR_INVALID_ARG, "quantised weights need their scales");
   }
   return ZO_OK;
 }
@@ -716,6 +735,16 @@ zo_status zo_profile_read(zo_ctx* ctx, double* host_ms, double* host_flops, int3
 }
 
 const char* zo_last_error(const zo_ctx* ctx) { return ctx ? ctx->err : g_init_error; }
+
+zo_status zo_dequantize(void* cuda_stream, int32_t weight_format, int32_t precision, const void* codes,
+                        const float* scale, void* out, int32_t rows, int32_t k_in) {
+  if (!codes || !scale || !out || rows < 1 || k_in < 1) return ZO_ERR_INVALID_ARG;
+  if (weight_format != ZO_W_INT8 && weight_format != ZO_W_NF4) return ZO_ERR_INVALID_ARG;
+  if (precision != ZO_FP32 && precision != ZO_BF16) return ZO_ERR_INVALID_ARG;
+  if (k_in % (weight_format == ZO_W_NF4 ? 64 : 16)) return ZO_ERR_UNSUPPORTED;
+  launch_dequant((cudaStream_t)cuda_stream, precision == ZO_BF16, weight_format, codes, scale, out, rows, k_in);
+  return cudaGetLastError() == cudaSuccess ? ZO_OK : ZO_ERR_CUDA;
+}
 
 zo_status zo_perturbation(void* cuda_stream, uint64_t seed, uint32_t tensor_id, uint32_t query,
                           int64_t n, uint32_t* dev_u32, float* dev_z) {
