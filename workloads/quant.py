@@ -40,8 +40,8 @@ def quantize_nf4(w: np.ndarray):
     absmax = np.abs(blk).max(axis=2).astype(np.float32)
     safe = np.where(absmax > 0, absmax, np.float32(1.0))
     x = blk / safe[:, :, None]
-    codes = np.abs(x[..., None] - _NF4[None, None, None, :]).argmin(axis=-1).astype(np.uint8)
-    codes = codes.reshape(rows, K)
+    mid = (_NF4[:-1] + _NF4[1:]) * np.float32(0.5)           # nearest level; a tie goes to the lower one
+    codes = np.searchsorted(mid, x.reshape(-1), side="left").astype(np.uint8).reshape(rows, K)
     packed = ((codes[:, 0::2] << 4) | codes[:, 1::2]).astype(np.uint8)
     return packed, safe
 
