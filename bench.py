@@ -98,13 +98,17 @@ def whole_job_value(world, units_per_step, steps, ms):
     return world * units_per_step * steps / (ms * 1e-3)
 
 
-def load_problem(spec, seed=1234, b_std=0.01):
-    """Synthetic weights on the device, one decoder block in host memory at a time."""
+def load_problem(spec, seed=1234, b_std=0.01, weights=None):
+    """Synthetic weights on the device, one decoder block in host memory at a time; `weights` =
+    "int8" / "nf4" stores the four linear weights of every block in that weight-only format."""
     import paper_2409_15520_b200 as zo
+    from workloads import quantize_layer
     if spec.arch == ARCH_LINEAR:
         return zo.DeviceProblem(make_linear_problem(spec, seed=seed, b_std=b_std), spec.bf16)
     p = make_decoder_globals(spec, seed)
-    p["layers"] = (make_decoder_layer(spec, seed, l, b_std) for l in range(spec.n_layers))
+    mk = (lambda l: make_decoder_layer(spec, seed, l, b_std)) if not weights else \
+        (lambda l: quantize_layer(make_decoder_layer(spec, seed, l, b_std), weights))
+    p["layers"] = (mk(l) for l in range(spec.n_layers))
     return zo.DeviceProblem(p, spec.bf16, n_layers=spec.n_layers)
 
 
@@ -198,8 +202,8 @@ def run_ablation(args, spec):
     import paper_2409_15520_b200 as zo
     from workloads import next_token_labels
     big = spec.with_(q=16, E=16, S=256)
-    prob = load_problem(big)
-    est = zo.Estimator(zo.make_config(big, flags=args.flags))
+    prob = load_problem(big, weights=args.weights)
+    est = zo.Estimator(zo.make_config(big, flags=args.flags, weight_format=args.weights))
     rng = np.random.default_rng(7)
 
     def time_point(q, E, S, schedule):
@@ -221,8 +225,10 @@ def run_ablation(args, spec):
     for S in (64, 128, 256):
         for E in (1, 8, 16):
             par, seq = time_point(1, E, S, "full"), time_point(1, E, S, "sequential")
-            print(json.dumps({"table": "inner_loop", "q": 1, "seq": S, "batch": E, "ms_parallel_pair": round(par, 3),
+            print(json.dumps({"table": "inner_loop", "weights": args.weights or "bf16", "q": 1, "seq": S, "batch": E, "ms_parallel_pair": round(par, 3),
                               "ms_sequential_pair": round(seq, 3), "speedup": round(seq / par, 3)}), flush=True)
+    if args.weights:
+        return                      # the paper's quantisation figure is the inner-loop grid only
     for S in (64, 128, 256):
         for q, E in ((1, 16), (4, 4), (16, 1)):
             r = {"table": "outer_loop", "q": q, "E": E, "seq": S}
@@ -273,6 +279,8 @@ def main():
     ap.add_argument("--ablation", action="store_true", help="the paper's inner/outer-loop runtime grids on this GPU")
     ap.add_argument("--schedule", default="full", choices=["full", "outer_only", "inner_only", "sequential"],
                     help="how the step is cut into forward passes (the paper's ablation)")
+    ap.add_argument("--weights", default=None, choices=["int8", "nf4"],
+                    help="weight-only quantised storage of the frozen linear weights (decoded once per pass)")
     ap.add_argument("--E", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--S", type=int, default=0, help="override the sequence length")
     args = ap.parse_args()
@@ -308,8 +316,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    prob = load_problem(spec)
-    est = zo.Estimator(zo.make_config(spec, flags=args.flags))
+    prob = load_problem(spec, weights=args.weights)
+    est = zo.Estimator(zo.make_config(spec, flags=args.flags, weight_format=args.weights))
     est.set_schedule(args.schedule)
     E, S, q, eps, lr = spec.E, spec.S, spec.q, spec.eps, spec.lr
     tokens_per_step = 2 * q * E * S
@@ -378,7 +386,7 @@ def main():
                    "lora_rank": spec.lora_rank, "q": q, "E": E, "S": S, "replicas": 2 * q,
                    "token_rows_per_step": tokens_per_step, "eps": eps, "lr": lr,
                    "l2": "inputs larger than L2 (weights and activations of several GB stream every step)",
-                   "schedule": args.schedule,
+                   "schedule": args.schedule, "weights": args.weights or "bf16",
                    "parallelism": "replicas only" if world > 1 else "1 gpu"},
         "zo_steps_per_s": world * args.steps / (ms * 1e-3),
         "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,
