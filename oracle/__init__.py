@@ -11,7 +11,8 @@ into the weights; closed-form gradient of the linear+MSE problem; quadratic
 loss (exact central difference, variance slope in q); brute-force coordinate
 finite differences; q=1 equals sequential in-place MeZO; the stored-pair
 recurrences of the Mobile MP-LoRA module; batched MP-LoRA equals 2q
-independent forwards; eps=0 degeneracy.  No function here is left unpinned.
+independent forwards; eps=0 degeneracy; NF4 levels against their normal-quantile construction,
+INT8/NF4 round-trip bounds and hand-built packing.  No function here is left unpinned.
 """
 from .philox import philox4x32_10, perturbation_u32, perturbation  # noqa: F401
 from .model import replica_losses, mp_lora_linear  # noqa: F401
