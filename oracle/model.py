@@ -164,6 +164,14 @@ def replica_losses(spec, p, Bn, tokens, labels, return_rows=False):
                            p.get("bias"), p["A"], _f64(Bn), spec.lora_scale)
         per = ((Y - _f64(labels)[None]) ** 2).mean(-1)    # [n,T]
         return (per.mean(-1), per) if return_rows else per.mean(-1)
-    h = decoder_hidden(spec, p, [_f64(b) for b in Bn], np.asarray(tokens))
+    Bn = [_f64(b) for b in Bn]
+    if isinstance(tokens, (list, tuple)):
+        # ragged batch (no padding): every sequence is its own forward pass of its own length; the
+        # loss is still the mean over all labelled positions of the batch
+        parts = [row_losses(spec, p, decoder_hidden(spec, p, Bn, np.asarray(t)[None]), np.asarray(l)[None])
+                 for t, l in zip(tokens, labels)]
+        rl = np.concatenate(parts, axis=1)
+        return (rl.mean(-1), rl) if return_rows else rl.mean(-1)
+    h = decoder_hidden(spec, p, Bn, np.asarray(tokens))
     rl = row_losses(spec, p, h, np.asarray(labels))
     return (rl.mean(-1), rl) if return_rows else rl.mean(-1)

@@ -217,3 +217,24 @@ def test_replica_order_and_sign_convention():
         lm = oracle.replica_losses(spec, p, (p["B"] - eps * z)[None], p["X"], p["target"])[0]
         assert losses[2 * i] == lp and losses[2 * i + 1] == lm
         assert np.sign(g[i]) == np.sign(lp - lm)
+
+
+@pytest.mark.parametrize("arch", [ARCH_OPT, ARCH_LLAMA])
+def test_ragged_batch_equals_padded_batch_with_ignored_padding(arch):
+    """Causal attention: tokens appended after a sequence cannot change its earlier positions, so the
+    ragged (unpadded) evaluation equals the padded one with the padding positions left out of the loss."""
+    from workloads import make_ragged_batch
+    spec, p = _tiny(arch, E=3, S=8, max_seq=8, n_labelled=2)
+    toks, labs = make_ragged_batch(spec, seed=5)
+    assert len({len(t) for t in toks}) > 1 and all(2 <= len(t) <= 8 for t in toks)
+    pad_t = np.zeros((3, 8), np.int32)
+    pad_l = np.full((3, 8), -1, np.int32)
+    for b, (t, l) in enumerate(zip(toks, labs)):
+        pad_t[b, :len(t)] = t
+        pad_t[b, len(t):] = 7                      # arbitrary padding token
+        pad_l[b, :len(l)] = l
+    a = oracle.zo_step(spec, p, toks, labs, 3, 2, 1e-2, 1e-2)
+    b = oracle.zo_step(spec, p, pad_t, pad_l, 3, 2, 1e-2, 1e-2)
+    assert np.allclose(a[0], b[0], rtol=1e-12) and np.allclose(a[1], b[1], rtol=1e-9)
+    for x, y in zip(a[2], b[2]):
+        assert np.allclose(x, y, rtol=0, atol=1e-12)

@@ -8,6 +8,6 @@ own random generators.
 from .spec import ModelSpec, CONFIGS, config  # noqa: F401
 from .synth import (  # noqa: F401
     bf16_round, to_bf16_bits, from_bf16_bits, make_linear_problem,
-    make_decoder_problem, make_decoder_globals, make_decoder_layer, next_token_labels, label_word_labels,
+    make_decoder_problem, make_ragged_batch, make_decoder_globals, make_decoder_layer, next_token_labels, label_word_labels,
 )
 from .quant import quantize_int8, quantize_nf4, quantize_layer  # noqa: F401

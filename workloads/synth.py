@@ -136,3 +136,24 @@ def label_word_labels(spec: ModelSpec, seed: int) -> np.ndarray:
     lab = np.full((spec.E, spec.S), -1, np.int32)
     lab[:, spec.S - 1] = _rng(seed, 21).integers(0, 2, size=spec.E, dtype=np.int32)
     return lab
+
+
+def make_ragged_batch(spec: ModelSpec, seed: int = 1234, min_frac: float = 0.25):
+    """Variable-length stand-in for tokenised task prompts: E sequences with lengths uniform in
+    [max(2, min_frac*S), S], uniform random token ids; labels as for the fixed-length batches (the last
+    `n_labelled` predicting positions of each sequence, or the class id at its final position).
+    Returns (list of int32 token arrays, list of int32 label arrays)."""
+    rng = _rng(seed, 30)
+    lo = max(2, int(min_frac * spec.S))
+    lens = rng.integers(lo, spec.S + 1, size=spec.E)
+    toks, labs = [], []
+    for b, n in enumerate(lens):
+        t = rng.integers(0, spec.vocab, size=int(n), dtype=np.int32)
+        if spec.loss_kind == LOSS_CE_LABEL_WORDS:
+            l = np.full(int(n), -1, np.int32)
+            l[-1] = rng.integers(0, 2)
+        else:
+            l = next_token_labels(t[None], min(spec.n_labelled, int(n) - 1))[0]
+        toks.append(t)
+        labs.append(l)
+    return toks, labs
