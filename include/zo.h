@@ -178,6 +178,20 @@ ZO_API zo_status zo_step(zo_ctx* ctx, const zo_weights* weights, const zo_lora* 
                   const void* tokens, const void* labels, int32_t E, int32_t S,
                   uint64_t seed, int32_t q, float eps, float lr);
 
+/* The same step on a PACKED variable-length batch (no padding rows at all: the paper's second
+ * argument for small E is less padding; here there is none).  Decoders only.
+ *   tokens, labels : int32 [total_tokens], the E sequences back to back
+ *   cu_seqlens     : int32 [E + 1] device array, cu[0] = 0, cu[b+1] - cu[b] = length of sequence b
+ *                    (1 .. max_len), cu[E] = total_tokens
+ *   max_len        : upper bound of the lengths, <= max_seq; total_tokens <= max_E * max_seq
+ * Positions (learned or rotary) restart at 0 in every sequence; attention is causal inside a
+ * sequence; labels as in zo_step.  A malformed cu_seqlens is reported by zo_losses as
+ * ZO_ERR_INVALID_ARG. */
+ZO_API zo_status zo_step_varlen(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
+                                const int32_t* tokens, const int32_t* labels, const int32_t* cu_seqlens,
+                                int32_t E, int32_t total_tokens, int32_t max_len, uint64_t seed,
+                                int32_t q, float eps, float lr);
+
 /* Same step with tokens and labels in HOST memory (pinned or pageable): they are
  * copied to the device on the context's stream first.  The host buffers must stay
  * untouched until the stream has passed the copy (e.g. until zo_losses returns). */

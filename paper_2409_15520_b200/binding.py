@@ -71,6 +71,9 @@ _STEP_ARGS = [C.c_void_p, C.POINTER(ZoWeights), C.POINTER(ZoLora), C.c_void_p, C
               C.c_int32, C.c_int32, C.c_uint64, C.c_int32, C.c_float, C.c_float]
 zo_step = _sig("zo_step", C.c_int, _STEP_ARGS)
 zo_step_host = _sig("zo_step_host", C.c_int, _STEP_ARGS)
+zo_step_varlen = _sig("zo_step_varlen", C.c_int, [
+    C.c_void_p, C.POINTER(ZoWeights), C.POINTER(ZoLora), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+    C.c_int32, C.c_int32, C.c_uint64, C.c_int32, C.c_float, C.c_float])
 zo_losses = _sig("zo_losses", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p])
 zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)])
 zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
@@ -224,6 +227,13 @@ class Estimator:
         lab = prob.labels if labels is None else labels
         self._check(zo_step(self._h, C.byref(prob.weights), C.byref(prob.lora), _ptr(tok), _ptr(lab),
                             E, S, seed, q, eps, lr))
+        self.q = q
+
+    def step_varlen(self, prob: DeviceProblem, tokens, labels, cu_seqlens, max_len, seed, q, eps, lr):
+        """Packed variable-length batch: int32 device tensors tokens/labels [total], cu_seqlens [E+1]."""
+        E, total = cu_seqlens.numel() - 1, tokens.numel()
+        self._check(zo_step_varlen(self._h, C.byref(prob.weights), C.byref(prob.lora), _ptr(tokens), _ptr(labels),
+                                   _ptr(cu_seqlens), E, total, max_len, seed, q, eps, lr))
         self.q = q
 
     def step_host(self, prob: DeviceProblem, E, S, seed, q, eps, lr):

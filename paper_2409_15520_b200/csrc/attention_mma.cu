@@ -73,7 +73,7 @@ template <int N> __device__ __forceinline__ void cp_wait() {
 
 template <int DH>
 __global__ void __launch_bounds__(128, 3)
-attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E, int S, int Tp,
+attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, SeqLayout sl, int Tp,
                      int d) {
   extern __shared__ __align__(16) uint8_t sm_raw[];
   constexpr int LDS = DH + 8;
@@ -82,8 +82,10 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
   bf16* Vs = Ks + 64 * LDS;
   const int qt = gridDim.x - 1 - blockIdx.x;          // longest tiles first
   const int q0 = qt * 64, h = blockIdx.y, sq = blockIdx.z;
-  const int n = sq / E, b = sq % E;
-  const size_t row_base = (size_t)n * Tp + (size_t)b * S;
+  const int n = sq / sl.E, b = sq % sl.E;
+  const int S = sl.cu ? sl.cu[b + 1] - sl.cu[b] : sl.S;          // this sequence's length
+  if (q0 >= S) return;                                            // uniform over the CTA
+  const size_t row_base = (size_t)n * Tp + (size_t)(sl.cu ? sl.cu[b] : b * sl.S);
   const int ld = 3 * d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -231,22 +233,23 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, int E
 }
 
 template <int DH>
-void launch_t(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp, int d, int H) {
+void launch_t(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl, int Tp, int d, int H) {
+  const int S = sl.S, E = sl.E;
   const size_t smem = (size_t)3 * 64 * (DH + 8) * sizeof(bf16);
   cudaFuncSetAttribute(attention_mma_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   dim3 grid((S + 63) / 64, H, n * E);
-  attention_mma_kernel<DH><<<grid, 128, smem, st>>>((const bf16*)qkv, (bf16*)ctx, E, S, Tp, d);
+  attention_mma_kernel<DH><<<grid, 128, smem, st>>>((const bf16*)qkv, (bf16*)ctx, sl, Tp, d);
 }
 
 }  // namespace
 
 bool attention_mma_supported(int dh) { return dh == 64 || dh == 128; }
 
-void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp,
+void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl, int Tp,
                           int d, int H) {
   const int dh = d / H;
-  if (dh == 64) launch_t<64>(st, qkv, ctx, n, E, S, Tp, d, H);
-  else if (dh == 128) launch_t<128>(st, qkv, ctx, n, E, S, Tp, d, H);
+  if (dh == 64) launch_t<64>(st, qkv, ctx, n, sl, Tp, d, H);
+  else if (dh == 128) launch_t<128>(st, qkv, ctx, n, sl, Tp, d, H);
 }
 
 }  // namespace zo

@@ -71,6 +71,7 @@ struct Params {
   int act, swiglu;
   const float* rope_tab;    // non-null: rotate q and k (columns < rope_cols) in the epilogue
   int rope_cols, rope_dh, rope_s, rope_tp;
+  const int32_t* rope_pos;  // packed variable-length rows: position of row (m % rope_tp), else null
   int has_lora;
   int slab;                 // 1: the LoRA term is one or two extra k-blocks on the tensor cores
   int a_mod;                // > 0: the packed-U rows of tile row m are m % a_mod (input shared by all replicas)
@@ -722,7 +723,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (have2) add_res(col0 + po * 32, f2);
         if (rope_here) {
           const int dh = P.rope_dh, hd = dh >> 1;
-          const float* cs = P.rope_tab + (size_t)((row % P.rope_tp) % P.rope_s) * dh;   // cos[0..hd) | sin[0..hd)
+          const float* cs = P.rope_tab + (size_t)(P.rope_pos ? P.rope_pos[row % P.rope_tp] : (row % P.rope_tp) % P.rope_s) * dh;   // cos[0..hd) | sin[0..hd)
           if (po > 0) {
             const int h0 = col0 % dh;                  // head-local index of this chunk's first column (< hd)
 #pragma unroll
@@ -866,7 +867,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
   CUtensorMap tmU = tmA;
   P.a_mod = G.a_mod;
-  P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp;
+  P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp; P.rope_pos = G.rope_pos;
   if (P.slab) {
     e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)(G.a_mod > 0 ? G.a_mod : G.M), (uint64_t)G.pack_ld);
     if (e) return 10000 + e;

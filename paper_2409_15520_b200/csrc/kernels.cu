@@ -11,7 +11,7 @@ namespace zo {
 // =========================================================================================
 template <typename T>
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __restrict__ tok_emb,
-                             const T* __restrict__ pos_emb, T* __restrict__ out, int Tn, int S,
+                             const T* __restrict__ pos_emb, T* __restrict__ out, int Tn, SeqLayout sl,
                              int d, int vocab, uint32_t* status) {
   const int t = blockIdx.x;
   T* o = out + (size_t)t * d;
@@ -25,7 +25,7 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __rest
     id = 0;
   }
   const T* e = tok_emb + (size_t)id * d;
-  const T* p = pos_emb ? pos_emb + (size_t)(t % S) * d : nullptr;
+  const T* p = pos_emb ? pos_emb + (size_t)(sl.pos ? sl.pos[t] : t % sl.S) * d : nullptr;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     float v = to_f(e[c]);
     if (p) v += to_f(p[c]);
@@ -34,14 +34,14 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const T* __rest
 }
 
 void launch_embed(cudaStream_t st, int bf, const int32_t* tokens, const void* tok_emb,
-                  const void* pos_emb, void* out, int T, int Tp, int S, int d, int vocab,
+                  const void* pos_emb, void* out, int T, int Tp, SeqLayout sl, int d, int vocab,
                   uint32_t* status) {
   if (bf)
     embed_kernel<bf16><<<Tp, 128, 0, st>>>(tokens, (const bf16*)tok_emb, (const bf16*)pos_emb,
-                                           (bf16*)out, T, S, d, vocab, status);
+                                           (bf16*)out, T, sl, d, vocab, status);
   else
     embed_kernel<float><<<Tp, 128, 0, st>>>(tokens, (const float*)tok_emb, (const float*)pos_emb,
-                                            (float*)out, T, S, d, vocab, status);
+                                            (float*)out, T, sl, d, vocab, status);
 }
 
 // =========================================================================================
@@ -450,7 +450,7 @@ void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float t
 // In place on the q and k sections of the fused [rows, 3d] buffer.  Each thread rotates VEC
 // consecutive pairs (16-byte accesses).
 template <typename T>
-__global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S, int d, int H,
+__global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, SeqLayout sl, int d, int H,
                             const float* __restrict__ tab) {
   constexpr int VEC = 16 / sizeof(T);
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -463,7 +463,7 @@ __global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S,
   rest /= H;
   const int which = (int)(rest % 2);                  // 0 = q, 1 = k
   const long long row = rest / 2;
-  const int s = (int)((row % Tp) % S);
+  const int s = sl.pos ? sl.pos[row % Tp] : (int)((row % Tp) % sl.S);
   const float* cs = tab + (size_t)s * 2 * half + j;   // row s: cos[0..half) then sin[0..half)
   T* p = qkv + (size_t)row * 3 * d + (size_t)which * d + h * 2 * half + j;
   uint4 lo = *reinterpret_cast<const uint4*>(p), hi = *reinterpret_cast<const uint4*>(p + half);
@@ -481,7 +481,7 @@ __global__ void rope_kernel(T* __restrict__ qkv, long long total, int Tp, int S,
 }
 // Scalar variant for head dimensions whose half is not a multiple of the vector width.
 template <typename T>
-__global__ void rope_scalar_kernel(T* __restrict__ qkv, long long total, int Tp, int S, int d, int H,
+__global__ void rope_scalar_kernel(T* __restrict__ qkv, long long total, int Tp, SeqLayout sl, int d, int H,
                                    const float* __restrict__ tab) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= total) return;
@@ -492,7 +492,7 @@ __global__ void rope_scalar_kernel(T* __restrict__ qkv, long long total, int Tp,
   rest /= H;
   const int which = (int)(rest % 2);
   const long long row = rest / 2;
-  const int s = (int)((row % Tp) % S);
+  const int s = sl.pos ? sl.pos[row % Tp] : (int)((row % Tp) % sl.S);
   const float c = tab[(size_t)s * 2 * half + j], sn = tab[(size_t)s * 2 * half + half + j];
   T* p = qkv + (size_t)row * 3 * d + (size_t)which * d + h * 2 * half + j;
   const float x1 = to_f(p[0]), x2 = to_f(p[half]);
@@ -500,24 +500,24 @@ __global__ void rope_scalar_kernel(T* __restrict__ qkv, long long total, int Tp,
   p[half] = from_f<T>(x2 * c + x1 * sn);
 }
 template <typename T>
-static void rope_dispatch(cudaStream_t st, void* qkv, int rows, int Tp, int S, int d, int H,
+static void rope_dispatch(cudaStream_t st, void* qkv, int rows, int Tp, SeqLayout sl, int d, int H,
                           const float* tab) {
   constexpr int VEC = 16 / sizeof(T);
   const int half = d / H / 2;
   if (half % VEC == 0 && d % VEC == 0 && ((uintptr_t)qkv & 15) == 0) {
     const long long total = (long long)rows * 2 * H * (half / VEC);
     if (total > 0)
-      rope_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((T*)qkv, total, Tp, S, d, H, tab);
+      rope_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((T*)qkv, total, Tp, sl, d, H, tab);
   } else {
     const long long total = (long long)rows * 2 * H * half;
     if (total > 0)
-      rope_scalar_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((T*)qkv, total, Tp, S, d, H, tab);
+      rope_scalar_kernel<T><<<(unsigned)((total + 255) / 256), 256, 0, st>>>((T*)qkv, total, Tp, sl, d, H, tab);
   }
 }
-void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, int d, int H,
+void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, SeqLayout sl, int d, int H,
                  const float* tab) {
-  if (bf) rope_dispatch<bf16>(st, qkv, rows, Tp, S, d, H, tab);
-  else rope_dispatch<float>(st, qkv, rows, Tp, S, d, H, tab);
+  if (bf) rope_dispatch<bf16>(st, qkv, rows, Tp, sl, d, H, tab);
+  else rope_dispatch<float>(st, qkv, rows, Tp, sl, d, H, tab);
 }
 
 // =========================================================================================
@@ -527,18 +527,20 @@ void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, in
 // =========================================================================================
 template <typename T, int DH>
 __global__ void __launch_bounds__(256)
-attention_simt_kernel(const T* __restrict__ qkv, T* __restrict__ ctx, int E, int S, int Tp,
+attention_simt_kernel(const T* __restrict__ qkv, T* __restrict__ ctx, SeqLayout sl, int Tp,
                       int d) {
   extern __shared__ float sm[];
   constexpr int LDQ = DH + 1;
-  const int Sp = (S + 63) & ~63;
+  const int Sp = (sl.S + 63) & ~63;              // row pitch of the score tile (longest sequence)
   float* Qs = sm;                 // [64][LDQ]
   float* Ks = Qs + 64 * LDQ;      // [64][LDQ]  (K tile, later V tile)
   float* Ss = Ks + 64 * LDQ;      // [64][Sp + 1]
   const int LDS = Sp + 1;
   const int q0 = blockIdx.x * 64, h = blockIdx.y, sq = blockIdx.z;
-  const int n = sq / E, b = sq % E;
-  const size_t row_base = (size_t)n * Tp + (size_t)b * S;
+  const int n = sq / sl.E, b = sq % sl.E;
+  const int S = sl.cu ? sl.cu[b + 1] - sl.cu[b] : sl.S;          // this sequence's length
+  if (q0 >= S) return;
+  const size_t row_base = (size_t)n * Tp + (size_t)(sl.cu ? sl.cu[b] : b * sl.S);
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const float scale = rsqrtf((float)DH);
   const int ld = 3 * d;
@@ -639,23 +641,24 @@ attention_simt_kernel(const T* __restrict__ qkv, T* __restrict__ ctx, int E, int
 }
 
 template <typename T, int DH>
-static void attention_simt_launch(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S,
+static void attention_simt_launch(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl,
                                   int Tp, int d, int H) {
+  const int S = sl.S, E = sl.E;
   const int Sp = (S + 63) & ~63;
   const size_t smem = (size_t)(2 * 64 * (DH + 1) + 64 * (Sp + 1)) * sizeof(float);
   cudaFuncSetAttribute(attention_simt_kernel<T, DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                        (int)smem);
   dim3 grid((S + 63) / 64, H, n * E);
-  attention_simt_kernel<T, DH><<<grid, 256, smem, st>>>((const T*)qkv, (T*)ctx, E, S, Tp, d);
+  attention_simt_kernel<T, DH><<<grid, 256, smem, st>>>((const T*)qkv, (T*)ctx, sl, Tp, d);
 }
 
-void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, int E,
-                           int S, int Tp, int d, int H) {
+void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, SeqLayout sl,
+                           int Tp, int d, int H) {
   const int dh = d / H;
 #define ZO_ATT(DH)                                                             \
   if (dh == DH) {                                                              \
-    if (bf) attention_simt_launch<bf16, DH>(st, qkv, ctx, n, E, S, Tp, d, H);  \
-    else attention_simt_launch<float, DH>(st, qkv, ctx, n, E, S, Tp, d, H);    \
+    if (bf) attention_simt_launch<bf16, DH>(st, qkv, ctx, n, sl, Tp, d, H);    \
+    else attention_simt_launch<float, DH>(st, qkv, ctx, n, sl, Tp, d, H);      \
     return;                                                                    \
   }
   ZO_ATT(16) ZO_ATT(32) ZO_ATT(64) ZO_ATT(128)
@@ -684,23 +687,50 @@ void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows,
 }
 
 // =========================================================================================
+// Packed variable-length batch: position of every packed row inside its sequence.
+__global__ void varlen_index_kernel(const int32_t* __restrict__ cu, int E, int Tn, int Tp, int max_len,
+                                    int32_t* __restrict__ pos, uint32_t* status) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= Tp) return;
+  if (t >= Tn) { pos[t] = 0; return; }
+  int lo = 0, hi = E;                               // largest b with cu[b] <= t
+  while (hi - lo > 1) {
+    const int mid = (lo + hi) >> 1;
+    if (cu[mid] <= t) lo = mid; else hi = mid;
+  }
+  const int p = t - cu[lo];
+  const int len = cu[lo + 1] - cu[lo];
+  if (p < 0 || len < 1 || len > max_len || p >= len || cu[0] != 0 || cu[E] != Tn) {
+    atomicOr(status, ST_BAD_LABELS);
+    pos[t] = 0;
+    return;
+  }
+  pos[t] = p;
+}
+void launch_varlen_index(cudaStream_t st, const int32_t* cu, int E, int T, int Tp, int max_len, int32_t* pos,
+                         uint32_t* status) {
+  varlen_index_kernel<<<(Tp + 255) / 256, 256, 0, st>>>(cu, E, T, Tp, max_len, pos, status);
+}
+
 // Labelled positions of each sequence, in order: lab_idx[b*P + p] = b*S + s (or -1),
 // lab_val = the label there.  One thread per sequence (S is small).
 // =========================================================================================
-__global__ void label_scan_kernel(const int32_t* __restrict__ labels, int E, int S, int P,
+__global__ void label_scan_kernel(const int32_t* __restrict__ labels, SeqLayout sl, int P,
                                   int n_classes, int32_t* lab_idx, int32_t* lab_val,
                                   int32_t* lab_cnt, uint32_t* status) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= E) return;
+  if (b >= sl.E) return;
+  const int start = sl.cu ? sl.cu[b] : b * sl.S;
+  const int S = sl.cu ? sl.cu[b + 1] - start : sl.S;
   int cnt = 0;
   for (int s = 0; s < S; ++s) {
-    const int v = labels[b * S + s];
+    const int v = labels[start + s];
     if (v < 0) continue;
     if (v >= n_classes || cnt >= P) {
       atomicOr(status, ST_BAD_LABELS);
       continue;
     }
-    lab_idx[b * P + cnt] = b * S + s;
+    lab_idx[b * P + cnt] = start + s;
     lab_val[b * P + cnt] = v;
     ++cnt;
   }
@@ -710,9 +740,9 @@ __global__ void label_scan_kernel(const int32_t* __restrict__ labels, int E, int
     lab_val[b * P + cnt] = -1;
   }
 }
-void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
+void launch_label_scan(cudaStream_t st, const int32_t* labels, SeqLayout sl, int P, int n_classes,
                        int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status) {
-  label_scan_kernel<<<(E + 63) / 64, 64, 0, st>>>(labels, E, S, P, n_classes, lab_idx, lab_val,
+  label_scan_kernel<<<(sl.E + 63) / 64, 64, 0, st>>>(labels, sl, P, n_classes, lab_idx, lab_val,
                                                   lab_cnt, status);
 }
 

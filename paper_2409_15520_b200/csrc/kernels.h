@@ -22,6 +22,15 @@ struct LoraDesc {
 
 enum { ACT_NONE = 0, ACT_RELU = 1 };
 
+// How the T token rows of one replica split into sequences.  Fixed length: E sequences of S rows
+// (cu = pos = null).  Packed variable length: sequence b is rows cu[b] .. cu[b+1]-1, S is the longest
+// allowed length, pos[t] the position of packed row t inside its sequence.
+struct SeqLayout {
+  int E, S;
+  const int32_t* cu;
+  const int32_t* pos;
+};
+
 struct GemmDesc {
   const void* A; int lda;       // [M, K] activations
   const void* W;                // [N, K] weights (K contiguous)
@@ -41,6 +50,7 @@ struct GemmDesc {
   const float* rope_tab;        // tensor-core kernel: rotate columns < rope_cols (q, k) in the epilogue; table
                                 // rows cos[0..dh/2) | sin[0..dh/2); position of row m = (m % rope_tp) % rope_s
   int rope_cols, rope_dh, rope_s, rope_tp;
+  const int32_t* rope_pos;      // packed variable-length rows: position of row (m % rope_tp), else null
   int a_mod;                    // > 0 with lora_slab: packed-U row of output row m is m % a_mod (shared input)
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
@@ -48,7 +58,7 @@ struct GemmDesc {
 
 // --- elementwise / reduction kernels (bf = 1: bfloat16 tensors, 0: float) -------------------
 void launch_embed(cudaStream_t st, int bf, const int32_t* tokens, const void* tok_emb,
-                  const void* pos_emb, void* out, int T, int Tp, int S, int d, int vocab,
+                  const void* pos_emb, void* out, int T, int Tp, SeqLayout sl, int d, int vocab,
                   uint32_t* status);
 // Row norm. kind 0 = LayerNorm (gain, bias), 1 = RMSNorm (gain).  When lab_idx != null the
 // source row of output row (n, j) with j < EP is n*Tp + lab_idx[j] (negative: zero row).
@@ -60,16 +70,20 @@ void launch_lora_down(cudaStream_t st, int bf, const void* X, int ldx, const voi
 void launch_lora_apply(cudaStream_t st, int bf, const void* base, int ldb, int base_shared,
                        void* out, int ldo, int n, int T, const LoraDesc& L, int nsec);
 void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float theta);
-void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, int S, int d, int H,
+void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, SeqLayout sl, int d, int H,
                  const float* tab);
-void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, int E,
-                           int S, int Tp, int d, int H);
+void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, int n, SeqLayout sl,
+                           int Tp, int d, int H);
 // Tensor-core causal attention for bf16 with head_dim 64 or 128 (q, k already rotated).
 bool attention_mma_supported(int dh);
-void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, int E, int S, int Tp,
+void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl, int Tp,
                           int d, int H);
 void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows, int ffn);
-void launch_label_scan(cudaStream_t st, const int32_t* labels, int E, int S, int P, int n_classes,
+// Positions of packed rows: pos[t] = t - cu[b] for the sequence b that holds row t (0 for pad rows);
+// flags sequences longer than max_len or a non-monotone cu.
+void launch_varlen_index(cudaStream_t st, const int32_t* cu, int E, int T, int Tp, int max_len, int32_t* pos,
+                         uint32_t* status);
+void launch_label_scan(cudaStream_t st, const int32_t* labels, SeqLayout sl, int P, int n_classes,
                        int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status);
 void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
                     int EP, int rows, double* row_loss);

@@ -18,7 +18,7 @@ char g_init_error[256] = "";
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
-      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, total;
+      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, pos, total;
 };
 
 inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -124,6 +124,7 @@ Plan make_plan(const zo_config& c) {
     p.lab_cnt = take(c.max_E * 4);
     p.tok_stage = take(Tm * 4);
     p.lab_stage = take(Tm * 4);
+    p.pos = take(Tp * 4);
     p.xh = take(Mh * d * es);
     if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
     p.rowloss = take(Mh * 8);
@@ -327,10 +328,11 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
 
 zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const int32_t* tokens,
                        const int32_t* labels, int E, int S, uint64_t seed, int q, float eps,
-                       float lr) {
+                       float lr, const int32_t* cu = nullptr, int total_tokens = 0) {
   const zo_config& cf = c->cfg;
   const int bf = c->bf, r = cf.lora_rank, d = cf.d_model, f = cf.d_ffn, H = cf.n_heads;
-  const int T = E * S, Tp = (int)up(T, row_pad(cf));
+  // packed variable-length batch: T = all tokens, S = longest allowed sequence
+  const int T = cu ? total_tokens : E * S, Tp = (int)up(T, row_pad(cf));
   const int nt = c->nt, J = nt * r;
   const bool opt = cf.arch == ZO_ARCH_OPT;
   const int nkind = opt ? 0 : 1;
@@ -358,7 +360,13 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
 
   const int P = cf.max_labelled, EP = E * P;
   const int n_classes = cf.loss_kind == ZO_LOSS_CE_LABEL_WORDS ? 2 : cf.vocab;
-  PROF(PC_MISC, 0.0, launch_label_scan(st, labels, E, S, P, n_classes, lab_idx, lab_val, lab_cnt, status));
+  SeqLayout sl{E, S, cu, nullptr};
+  if (cu) {
+    int32_t* pos = c->at<int32_t>(c->plan.pos);
+    PROF(PC_MISC, 0.0, launch_varlen_index(st, cu, E, T, Tp, S, pos, status));
+    sl.pos = pos;
+  }
+  PROF(PC_MISC, 0.0, launch_label_scan(st, labels, sl, P, n_classes, lab_idx, lab_val, lab_cnt, status));
 
   Pass passes[64];
   const int n_pass = make_passes(c->schedule, q, passes);
@@ -366,7 +374,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   const Pass ps = passes[pi];
   const int n = ps.count, M = n * Tp;          // replicas and token rows of this forward pass
   // shared prefix: embedding on the T shared tokens, once for all replicas of the pass
-  PROF(PC_MISC, 0.0, launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, S, d, cf.vocab, status));
+  PROF(PC_MISC, 0.0, launch_embed(st, bf, tokens, w->tok_emb, opt ? w->pos_emb : nullptr, h0, T, Tp, sl, d, cf.vocab, status));
 
   for (int l = 0; l < cf.n_layers; ++l) {
     const zo_layer_weights& W = w->layers[l];
@@ -399,7 +407,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     // The rotary embedding rides in the epilogue of whichever tensor-core GEMM writes q|k|v last.
     bool rope_done = opt;
     auto with_rope = [&](GemmDesc& D) {
-      D.rope_tab = rope; D.rope_cols = 2 * d; D.rope_dh = d / H; D.rope_s = S; D.rope_tp = Tp;
+      D.rope_tab = rope; D.rope_cols = 2 * d; D.rope_dh = d / H; D.rope_s = S; D.rope_tp = Tp; D.rope_pos = sl.pos;
       rope_done = true;
     };
     const bool tcore = bf && !(cf.flags & ZO_FLAG_SIMT_GEMM);
@@ -433,11 +441,11 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(G);
       if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
-    if (!rope_done) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, S, d, H, rope)); }
+    if (!rope_done) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, sl, d, H, rope)); }
     if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
-      PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, E, S, Tp, d, H));
+      PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, sl, Tp, d, H));
     } else {
-      PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, E, S, Tp, d, H));
+      PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, sl, Tp, d, H));
     }
     GemmDesc O{};
     O.A = x; O.lda = d; O.W = weight(W.w_o, W.s_o, d, d); O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
@@ -624,6 +632,27 @@ zo_status zo_step(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora, c
   zo_status s = check_step_args(ctx, weights, lora, tokens, labels, E, S, q, eps, lr);
   if (s) return s;
   return do_step(ctx, weights, lora, tokens, labels, E, S, seed, q, eps, lr);
+}
+
+zo_status zo_step_varlen(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora, const int32_t* tokens,
+                         const int32_t* labels, const int32_t* cu_seqlens, int32_t E, int32_t total_tokens,
+                         int32_t max_len, uint64_t seed, int32_t q, float eps, float lr) {
+  zo_status s = check_step_args(ctx, weights, lora, tokens, labels, E, max_len, q, eps, lr);
+  if (s) return s;
+  if (ctx->cfg.arch == ZO_ARCH_LINEAR) return fail(ctx, ZO_ERR_UNSUPPORTED, "variable-length batches are for decoders");
+  if (!cu_seqlens) return fail(ctx, ZO_ERR_INVALID_ARG, "cu_seqlens is NULL");
+  if (total_tokens < E || (long long)total_tokens > (long long)E * max_len ||
+      (long long)total_tokens > (long long)ctx->cfg.max_E * ctx->cfg.max_seq)
+    return fail(ctx, ZO_ERR_INVALID_ARG, "total_tokens outside E .. E*max_len");
+  ctx->launches = 0;
+  cudaError_t e = cudaMemsetAsync(ctx->at<uint32_t>(ctx->plan.status), 0, 4, ctx->st);
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  s = step_decoder(ctx, weights, lora, tokens, labels, E, max_len, seed, q, eps, lr, cu_seqlens, total_tokens);
+  if (s) return s;
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  ctx->stepped = 1; ctx->last_q = q; ctx->last_E = E; ctx->last_S = max_len;
+  return ZO_OK;
 }
 
 zo_status zo_step_host(zo_ctx* ctx, const zo_weights* weights, const zo_lora* lora,
