@@ -83,9 +83,9 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, SeqLa
   const int qt = gridDim.x - 1 - blockIdx.x;          // longest tiles first
   const int q0 = qt * 64, h = blockIdx.y, sq = blockIdx.z;
   const int n = sq / sl.E, b = sq % sl.E;
-  const int S = sl.cu ? sl.cu[b + 1] - sl.cu[b] : sl.S;          // this sequence's length
+  const int S = sl.len(b);                                        // this sequence's length
   if (q0 >= S) return;                                            // uniform over the CTA
-  const size_t row_base = (size_t)n * Tp + (size_t)(sl.cu ? sl.cu[b] : b * sl.S);
+  const size_t row_base = (size_t)n * Tp + (size_t)sl.start(b);
   const int ld = 3 * d;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;

@@ -538,9 +538,9 @@ attention_simt_kernel(const T* __restrict__ qkv, T* __restrict__ ctx, SeqLayout 
   const int LDS = Sp + 1;
   const int q0 = blockIdx.x * 64, h = blockIdx.y, sq = blockIdx.z;
   const int n = sq / sl.E, b = sq % sl.E;
-  const int S = sl.cu ? sl.cu[b + 1] - sl.cu[b] : sl.S;          // this sequence's length
+  const int S = sl.len(b);                          // this sequence's length
   if (q0 >= S) return;
-  const size_t row_base = (size_t)n * Tp + (size_t)(sl.cu ? sl.cu[b] : b * sl.S);
+  const size_t row_base = (size_t)n * Tp + (size_t)sl.start(b);
   const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
   const float scale = rsqrtf((float)DH);
   const int ld = 3 * d;
@@ -720,8 +720,8 @@ __global__ void label_scan_kernel(const int32_t* __restrict__ labels, SeqLayout 
                                   int32_t* lab_cnt, uint32_t* status) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= sl.E) return;
-  const int start = sl.cu ? sl.cu[b] : b * sl.S;
-  const int S = sl.cu ? sl.cu[b + 1] - start : sl.S;
+  const int start = sl.start(b);
+  const int S = sl.len(b);
   int cnt = 0;
   for (int s = 0; s < S; ++s) {
     const int v = labels[start + s];

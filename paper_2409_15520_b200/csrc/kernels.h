@@ -29,6 +29,21 @@ struct SeqLayout {
   int E, S;
   const int32_t* cu;
   const int32_t* pos;
+  int T;   // token rows of one replica (bounds every cu-derived index)
+  // first row and length of sequence b, clamped so that a malformed cu cannot index outside the batch
+  __host__ __device__ int start(int b) const {
+    if (!cu) return b * S;
+    const int s0 = cu[b];
+    return s0 < 0 ? 0 : (s0 > T ? T : s0);
+  }
+  __host__ __device__ int len(int b) const {
+    if (!cu) return S;
+    const int s0 = start(b);
+    int l = cu[b + 1] - s0;
+    if (l > S) l = S;
+    if (l > T - s0) l = T - s0;
+    return l < 0 ? 0 : l;
+  }
 };
 
 struct GemmDesc {

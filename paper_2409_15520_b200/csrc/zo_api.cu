@@ -360,7 +360,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
 
   const int P = cf.max_labelled, EP = E * P;
   const int n_classes = cf.loss_kind == ZO_LOSS_CE_LABEL_WORDS ? 2 : cf.vocab;
-  SeqLayout sl{E, S, cu, nullptr};
+  SeqLayout sl{E, S, cu, nullptr, T};
   if (cu) {
     int32_t* pos = c->at<int32_t>(c->plan.pos);
     PROF(PC_MISC, 0.0, launch_varlen_index(st, cu, E, T, Tp, S, pos, status));
