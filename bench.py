@@ -238,6 +238,48 @@ def run_ablation(args, spec):
             print(json.dumps(r), flush=True)
 
 
+def run_varlen(args, spec):
+    """Padding study (the paper's second argument for small E): the same E variable-length sequences
+    (lengths uniform in [S/4, S]) run (a) padded to S in the fixed-length step and (b) packed back to
+    back through zo_step_varlen, which spends nothing on padding rows.  One JSON line."""
+    import torch
+    import paper_2409_15520_b200 as zo
+    from workloads import make_ragged_batch
+    prob = load_problem(spec, weights=args.weights)
+    est = zo.Estimator(zo.make_config(spec, flags=args.flags, weight_format=args.weights))
+    toks, labs = make_ragged_batch(spec, seed=77)
+    E, S, q = spec.E, spec.S, spec.q
+    pad_t = np.zeros((E, S), np.int32)
+    pad_l = np.full((E, S), -1, np.int32)
+    for b, (t, l) in enumerate(zip(toks, labs)):
+        pad_t[b, :len(t)], pad_l[b, :len(l)] = t, l
+    dev = lambda a: torch.tensor(np.ascontiguousarray(a), dtype=torch.int32, device="cuda")
+    d_pt, d_pl = dev(pad_t), dev(pad_l)
+    d_t, d_l = dev(np.concatenate(toks)), dev(np.concatenate(labs))
+    d_cu = dev(np.concatenate([[0], np.cumsum([len(t) for t in toks])]))
+    real = int(sum(len(t) for t in toks))
+
+    def timed(fn):
+        ts = []
+        for i in range(args.warmup + args.steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn(i)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1))
+        return float(np.median(ts[args.warmup:])), est.losses()[0]
+
+    ms_pad, l_pad = timed(lambda i: est.step(prob, E, S, 7, q, spec.eps, 0.0, tokens=d_pt, labels=d_pl))
+    ms_pack, l_pack = timed(lambda i: est.step_varlen(prob, d_t, d_l, d_cu, S, 7, q, spec.eps, 0.0))
+    print(json.dumps({"study": "padding", "workload": args.workload, "E": E, "S": S, "q": q, "real_tokens": real,
+                      "padded_tokens": E * S, "padding_fraction": round(1 - real / (E * S), 4),
+                      "ms_padded": round(ms_pad, 3), "ms_packed": round(ms_pack, 3),
+                      "speedup": round(ms_pad / ms_pack, 3),
+                      "real_tokens_per_s_packed": round(2 * q * real / (ms_pack * 1e-3)),
+                      "max_rel_loss_diff": float(np.max(np.abs(l_pad - l_pack) / np.abs(l_pad)))}))
+
+
 def run_reference(args, spec):
     """The CPU oracle as it stands, timed on the host cores (rank 0 only)."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -277,6 +319,7 @@ def main():
     ap.add_argument("--rank", type=int, default=0, help="override the LoRA rank")
     ap.add_argument("--sweep", action="store_true", help="MP-LoRA linear micro-benchmark grid (rank x q)")
     ap.add_argument("--ablation", action="store_true", help="the paper's inner/outer-loop runtime grids on this GPU")
+    ap.add_argument("--varlen", action="store_true", help="padded vs packed variable-length batch (padding study)")
     ap.add_argument("--schedule", default="full", choices=["full", "outer_only", "inner_only", "sequential"],
                     help="how the step is cut into forward passes (the paper's ablation)")
     ap.add_argument("--weights", default=None, choices=["int8", "nf4"],
@@ -303,6 +346,8 @@ def main():
         return run_reference(args, spec)
     if args.ablation:
         return run_ablation(args, spec)
+    if args.varlen:
+        return run_varlen(args, spec)
 
     import torch
     import torch.distributed as dist
