@@ -950,6 +950,10 @@ __constant__ float c_nf4[16] = {-1.0f, -0.6961928009986877f, -0.5250730514526367
 template <typename T>
 __global__ void dequant_kernel(int fmt, const uint8_t* __restrict__ codes, const float* __restrict__ scale,
                                T* __restrict__ out, long long total16, int K) {
+  // the 16 levels go to shared memory: lanes look up different codes, which constant memory serialises
+  __shared__ float tab[16];
+  if (threadIdx.x < 16) tab[threadIdx.x] = c_nf4[threadIdx.x];
+  __syncthreads();
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;   // group of 16 elements
   if (i >= total16) return;
   const long long e0 = i * 16;
@@ -968,8 +972,8 @@ __global__ void dequant_kernel(int fmt, const uint8_t* __restrict__ codes, const
     const float s = scale[row * (K / 64) + col / 64];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-      w[2 * j] = c_nf4[c[j] >> 4] * s;
-      w[2 * j + 1] = c_nf4[c[j] & 15] * s;
+      w[2 * j] = tab[c[j] >> 4] * s;
+      w[2 * j + 1] = tab[c[j] & 15] * s;
     }
   }
   __align__(16) T o[16];
