@@ -86,6 +86,8 @@ enum { ZO_FLAG_SIMT_GEMM = 1,
         * from fp32 U and fp32 (B + k eps z), never as the extra tensor-core k-block (which rounds
         * U, B and k eps z to bfloat16).  A/B switch. */
        ZO_FLAG_LORA_EPILOGUE = 4 };
+/* Bits 8..15 of flags, when non-zero, override the tensor-core GEMM's raster group (128-row tiles that
+ * sweep the weight panels together; default 16).  Tuning aid; results do not depend on it. */
 
 typedef struct zo_ctx zo_ctx; /* opaque; owned by the library; released by zo_free */
 

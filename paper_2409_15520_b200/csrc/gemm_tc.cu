@@ -72,6 +72,7 @@ struct Params {
   const float* rope_tab;    // non-null: rotate q and k (columns < rope_cols) in the epilogue
   int rope_cols, rope_dh, rope_s, rope_tp;
   const int32_t* rope_pos;  // packed variable-length rows: position of row (m % rope_tp), else null
+  int group_m;              // 128-row tiles per raster group
   int has_lora;
   int slab;                 // 1: the LoRA term is one or two extra k-blocks on the tensor cores
   int a_mod;                // > 0: the packed-U rows of tile row m are m % a_mod (input shared by all replicas)
@@ -293,7 +294,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int STAGES = PAIR ? Cfg<PAIR>::STAGES : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0);
   constexpr uint32_t STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
   constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
-  constexpr int GROUP_M = PAIR ? 8 : 16;             // 16 row tiles of 128 per raster group
+  const int GROUP_M = PAIR ? (P.group_m + 1) / 2 : P.group_m;   // row tiles of a raster group
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   float* lbuf = (float*)(smem + STAGES * STAGE_BYTES);
@@ -867,6 +868,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
   CUtensorMap tmU = tmA;
   P.a_mod = G.a_mod;
+  P.group_m = G.group_m > 0 ? G.group_m : 16;
   P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp; P.rope_pos = G.rope_pos;
   if (P.slab) {
     e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)(G.a_mod > 0 ? G.a_mod : G.M), (uint64_t)G.pack_ld);

@@ -66,6 +66,7 @@ struct GemmDesc {
                                 // rows cos[0..dh/2) | sin[0..dh/2); position of row m = (m % rope_tp) % rope_s
   int rope_cols, rope_dh, rope_s, rope_tp;
   const int32_t* rope_pos;      // packed variable-length rows: position of row (m % rope_tp), else null
+  int group_m;                  // 128-row tiles per raster group of the tensor-core kernel (0 = default 16)
   int a_mod;                    // > 0 with lora_slab: packed-U row of output row m is m % a_mod (shared input)
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile

@@ -213,6 +213,7 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
   if (tcore) {
     GemmDesc Gt = G;
     Gt.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
+    Gt.group_m = (int)((flags >> 8) & 0xFF);     // diagnostic: raster group override in bits 8..15
     const int e = launch_gemm_tc(st, Gt, status, n_sms);
     if (e) {
       snprintf(err, errn, "tensor-core GEMM launch failed (code %d: %s)", e,

@@ -35,7 +35,9 @@ def test_packed_variable_length_step(arch, bf16, loss):
     rows per replica not a multiple of anything): positions restart per sequence, attention stays inside
     a sequence, the loss is the mean over all labelled positions of the batch."""
     spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=bf16, loss_kind=loss, label_words=(3, 99),
-                     **{**BASE, "n_labelled": 1 if loss == LOSS_CE_LABEL_WORDS else 4})
+                     **{**BASE, "n_labelled": 1 if loss == LOSS_CE_LABEL_WORDS else 4,
+                        # five labelled rows only: a larger eps keeps the loss difference above fp32 noise
+                        "eps": 5e-2 if loss == LOSS_CE_LABEL_WORDS else 1e-2})
     p = make_decoder_problem(spec, seed=4, b_std=0.05)
     toks, labs = make_ragged_batch(spec, seed=6)
     assert len({len(t) for t in toks}) > 1
