@@ -73,6 +73,7 @@ struct Params {
   int rope_cols, rope_dh, rope_s, rope_tp;
   const int32_t* rope_pos;  // packed variable-length rows: position of row (m % rope_tp), else null
   int group_m;              // 128-row tiles per raster group
+  int run_order;            // 1: contiguous runs of tiles, row tile fastest inside (replica, column tile)
   int has_lora;
   int slab;                 // 1: the LoRA term is one or two extra k-blocks on the tensor cores
   int a_mod;                // > 0: the packed-U rows of tile row m are m % a_mod (input shared by all replicas)
@@ -310,6 +311,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_n = (P.N + ncol_tile - 1) / ncol_tile;
   const int num_tiles = tiles_m * tiles_n;
   const int num_kb = (P.K + BK - 1) / BK;
+  // Tile schedule of this CTA (pair).  Default: tiles unit, unit + n_units, ... of the grouped raster.
+  // Run order (expansion launches, whose cost is the generated operand): a contiguous run of tiles
+  // ordered row tile fastest inside (replica, column tile), so consecutive tiles reuse one operand.
+  const int run_chunk = (num_tiles + n_units - 1) / n_units;
+  const int t_first = P.run_order ? unit * run_chunk : unit;
+  const int t_step = P.run_order ? 1 : n_units;
+  const int t_end = P.run_order ? min(num_tiles, t_first + run_chunk) : num_tiles;
+  auto coords = [&](int t, int& tm, int& tn) {
+    if (P.run_order) {
+      const int tpr = P.L.rows_per_replica / TILE_M;     // row tiles per replica
+      const int rest = t / tpr;
+      tn = rest % tiles_n;
+      tm = (rest / tiles_n) * tpr + (t - rest * tpr);
+    } else {
+      tile_coords(t, tiles_m, tiles_n, GROUP_M, tm, tn);
+    }
+  };
+  // The generated LoRA operand depends on (replica, column tile) only: -1 = tile without LoRA term.
+  auto slab_key = [&](int tm, int tn) -> int {
+    if (tile_slot(P, tn * ncol_tile) < 0) return -1;
+    return ((tm * TILE_M) / P.L.rows_per_replica) * tiles_n + tn;
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < MAX_STAGES; ++s) {
@@ -353,9 +376,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0) {
       uint32_t issued = 0;
       bool ok = true;
-      for (int tile = unit; tile < num_tiles && ok; tile += n_units) {
+      for (int tile = t_first; tile < t_end && ok; tile += t_step) {
         int tm, tn;
-        tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+        coords(tile, tm, tn);
         const int m0 = tm * TILE_M + (int)rank * BM;
         const int brow0 = tn * ncol_tile;
         const int brow1 = P.swiglu ? P.N + brow0 : brow0 + 128;
@@ -399,8 +422,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
       uint32_t consumed = 0, titer = 0, ltiles = 0;
+      int cur_key = -2;                              // key of the operand the slab holds
       bool ok = true;
-      for (int tile = unit; tile < num_tiles && ok; tile += n_units, ++titer) {
+      for (int tile = t_first; tile < t_end && ok; tile += t_step, ++titer) {
         const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
         if (!mbar_wait(smem_u32(&ctrl->tempty[a]), aph ^ 1u, ctrl, P.status)) { ok = false; break; }
         tc_fence_after();
@@ -426,12 +450,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         if (!PAIR && ok) {
           int tm, tn;
-          tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
-          if (tile_slot(P, tn * ncol_tile) >= 0) {
+          coords(tile, tm, tn);
+          const int key = slab_key(tm, tn);
+          if (key >= 0) {
+            const bool fresh = key != cur_key;        // a newly generated operand to wait for
             for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++consumed) {
               const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
               if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
-                  (lkb == 0 && !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status))) { ok = false; break; }
+                  (lkb == 0 && fresh && !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status))) { ok = false; break; }
               tc_fence_after();
               const uint64_t ad = smem_desc(tiles_base + s * STAGE_BYTES);
               const uint64_t bd = smem_desc(tiles_base + STAGES * STAGE_BYTES + lkb * SLAB_BYTES);
@@ -442,7 +468,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               tc_commit(smem_u32(&ctrl->empty[s]));
             }
             if (!ok) break;
-            ++ltiles;
+            if (fresh) { ++ltiles; cur_key = key; }
           }
         }
         if (ok) {
@@ -468,7 +494,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // (B part) and K = khalf + k (perturbation part); all other K positions stay zero.
     auto gen_slab = [&](int g_tile) {
       int tm, tn;
-      tile_coords(g_tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+      coords(g_tile, tm, tn);
       const int n0g = tn * ncol_tile;
       const int slot = tile_slot(P, n0g);
       if (slot < 0) return;                         // uniform over the CTA
@@ -513,10 +539,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int i = et; i < (int)(SLAB_BYTES / 16) * (P.kslot / BK); i += EP_THREADS)
         reinterpret_cast<uint4*>(slab)[i] = make_uint4(0, 0, 0, 0);
       ep_bar();
-      if (unit < num_tiles) gen_slab(unit);
     }
+    int cur_key = -2;                                // key of the operand the slab holds
+    auto gen_if_new = [&](int t) {                   // same decision sequence as the MMA warp's
+      int tm, tn;
+      coords(t, tm, tn);
+      const int key = slab_key(tm, tn);
+      if (key >= 0 && key != cur_key) {
+        gen_slab(t);
+        cur_key = key;
+      }
+    };
+    if (!PAIR && P.slab && t_first < t_end) gen_if_new(t_first);
     uint32_t titer = 0;
-    for (int tile = unit; tile < num_tiles; tile += n_units, ++titer) {
+    for (int tile = t_first; tile < t_end; tile += t_step, ++titer) {
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
       if (et == 0) ctrl->ep_go = mbar_wait(smem_u32(&ctrl->tfull[a]), aph, ctrl, P.status) ? 1u : 0u;
       ep_bar();
@@ -525,9 +561,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!go) break;
       tc_fence_after();
       // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
-      if (!PAIR && P.slab && tile + n_units < num_tiles) gen_slab(tile + n_units);
+      if (!PAIR && P.slab && tile + t_step < t_end) gen_if_new(tile + t_step);
       int tm, tn;
-      tile_coords(tile, tiles_m, tiles_n, GROUP_M, tm, tn);
+      coords(tile, tm, tn);
       const int m0 = tm * TILE_M + (int)rank * BM, n0 = tn * ncol_tile;
       const int row = m0 + wq * 32 + lane;
       const bool row_ok = row < P.M;
@@ -869,6 +905,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   CUtensorMap tmU = tmA;
   P.a_mod = G.a_mod;
   P.group_m = G.group_m > 0 ? G.group_m : 16;
+  P.run_order = (P.slab && G.K == 0) ? 1 : 0;     // expansion only: amortise the generated operand
   P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp; P.rope_pos = G.rope_pos;
   if (P.slab) {
     e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)(G.a_mod > 0 ? G.a_mod : G.M), (uint64_t)G.pack_ld);
