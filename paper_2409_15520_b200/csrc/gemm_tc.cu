@@ -73,10 +73,8 @@ struct Params {
   int rope_cols, rope_dh, rope_s, rope_tp;
   const int32_t* rope_pos;  // packed variable-length rows: position of row (m % rope_tp), else null
   int group_m;              // 128-row tiles per raster group
-  int run_order;            // 1: contiguous runs of tiles, row tile fastest inside (replica, column tile)
   int has_lora;
   int slab;                 // 1: the LoRA term is one or two extra k-blocks on the tensor cores
-  int a_mod;                // > 0: the packed-U rows of tile row m are m % a_mod (input shared by all replicas)
   int kslot, khalf;         // K extent of one slot in the packed bf16 U, offset of its second copy
   bf16* pack_out; int pack_ld;  // down-projection: also write the packed bf16 U here (or null)
   int pack_r;
@@ -311,28 +309,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_n = (P.N + ncol_tile - 1) / ncol_tile;
   const int num_tiles = tiles_m * tiles_n;
   const int num_kb = (P.K + BK - 1) / BK;
-  // Tile schedule of this CTA (pair).  Default: tiles unit, unit + n_units, ... of the grouped raster.
-  // Run order (expansion launches, whose cost is the generated operand): a contiguous run of tiles
-  // ordered row tile fastest inside (replica, column tile), so consecutive tiles reuse one operand.
-  const int run_chunk = (num_tiles + n_units - 1) / n_units;
-  const int t_first = P.run_order ? unit * run_chunk : unit;
-  const int t_step = P.run_order ? 1 : n_units;
-  const int t_end = P.run_order ? min(num_tiles, t_first + run_chunk) : num_tiles;
-  auto coords = [&](int t, int& tm, int& tn) {
-    if (P.run_order) {
-      const int tpr = P.L.rows_per_replica / TILE_M;     // row tiles per replica
-      const int rest = t / tpr;
-      tn = rest % tiles_n;
-      tm = (rest / tiles_n) * tpr + (t - rest * tpr);
-    } else {
-      tile_coords(t, tiles_m, tiles_n, GROUP_M, tm, tn);
-    }
-  };
-  // The generated LoRA operand depends on (replica, column tile) only: -1 = tile without LoRA term.
-  auto slab_key = [&](int tm, int tn) -> int {
-    if (tile_slot(P, tn * ncol_tile) < 0) return -1;
-    return ((tm * TILE_M) / P.L.rows_per_replica) * tiles_n + tn;
-  };
+  // Tile schedule of this CTA (pair): tiles unit, unit + n_units, ... of the grouped raster.
+  const int t_first = unit, t_step = n_units, t_end = num_tiles;
+  auto coords = [&](int t, int& tm, int& tn) { tile_coords(t, tiles_m, tiles_n, GROUP_M, tm, tn); };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < MAX_STAGES; ++s) {
@@ -407,7 +386,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const uint32_t bar = smem_u32(&ctrl->full[s]);
           mbar_expect_tx(bar, A_BYTES);
           tma_load_2d(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot + lkb * BK,
-                      P.a_mod > 0 ? m0 % P.a_mod : m0, bar);
+                      m0, bar);
         }
         if (!ok) break;
       }
@@ -422,7 +401,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0) {
       uint32_t consumed = 0, titer = 0, ltiles = 0;
-      int cur_key = -2;                              // key of the operand the slab holds
       bool ok = true;
       for (int tile = t_first; tile < t_end && ok; tile += t_step, ++titer) {
         const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -451,24 +429,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!PAIR && ok) {
           int tm, tn;
           coords(tile, tm, tn);
-          const int key = slab_key(tm, tn);
-          if (key >= 0) {
-            const bool fresh = key != cur_key;        // a newly generated operand to wait for
+          if (tile_slot(P, tn * ncol_tile) >= 0) {
             for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++consumed) {
               const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
               if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
-                  (lkb == 0 && fresh && !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status))) { ok = false; break; }
+                  (lkb == 0 && !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status))) { ok = false; break; }
               tc_fence_after();
               const uint64_t ad = smem_desc(tiles_base + s * STAGE_BYTES);
               const uint64_t bd = smem_desc(tiles_base + STAGES * STAGE_BYTES + lkb * SLAB_BYTES);
 #pragma unroll
               for (int k = 0; k < BK / 16; ++k)
-                tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC,
-                       (uint32_t)((num_kb | lkb | k) != 0));
+                tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC, 1u);
               tc_commit(smem_u32(&ctrl->empty[s]));
             }
             if (!ok) break;
-            if (fresh) { ++ltiles; cur_key = key; }
+            ++ltiles;
           }
         }
         if (ok) {
@@ -540,17 +515,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         reinterpret_cast<uint4*>(slab)[i] = make_uint4(0, 0, 0, 0);
       ep_bar();
     }
-    int cur_key = -2;                                // key of the operand the slab holds
-    auto gen_if_new = [&](int t) {                   // same decision sequence as the MMA warp's
-      int tm, tn;
-      coords(t, tm, tn);
-      const int key = slab_key(tm, tn);
-      if (key >= 0 && key != cur_key) {
-        gen_slab(t);
-        cur_key = key;
-      }
-    };
-    if (!PAIR && P.slab && t_first < t_end) gen_if_new(t_first);
+    if (!PAIR && P.slab && t_first < t_end) gen_slab(t_first);
     uint32_t titer = 0;
     for (int tile = t_first; tile < t_end; tile += t_step, ++titer) {
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -561,7 +526,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!go) break;
       tc_fence_after();
       // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
-      if (!PAIR && P.slab && tile + t_step < t_end) gen_if_new(tile + t_step);
+      if (!PAIR && P.slab && tile + t_step < t_end) gen_slab(tile + t_step);
       int tm, tn;
       coords(tile, tm, tn);
       const int m0 = tm * TILE_M + (int)rank * BM, n0 = tn * ncol_tile;
@@ -577,7 +542,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int nchunk = ncol_tile / 32;
       const int po = P.rope_tab ? (P.rope_dh >> 6) : 0;          // 128 -> 2, 64 -> 1, <= 32 -> 0 (same chunk)
       const int pshift = po == 1 ? 1 : 0;                      // keep both chunks of a pair with one warp
-      const bool acc_valid = num_kb > 0 || tile_slot(P, n0) >= 0;
       // The perturbed B columns are staged G columns at a time (the whole 256-column tile for
       // rank <= 16): one generation phase, two barriers, then barrier-free chunks.
       const int G = P.has_lora ? lora_phase_cols(P.L.r) : 256;
@@ -682,12 +646,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool rope_here = P.rope_tab != nullptr && col0 < P.rope_cols;
         if (rope_here && po > 0 && (c % (2 * po)) >= po) continue;   // done with its low partner
         uint32_t v[32];
-        if (acc_valid) {
-          tc_ld32(taddr + c * 32, v);
-        } else {                                     // no k-block at all fed this tile: the sum is empty
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = 0u;
-        }
+        tc_ld32(taddr + c * 32, v);
         float f[32];
         if (P.swiglu) {
           uint32_t up[32];
@@ -742,13 +701,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool have2 = rope_here && po > 0;
         if (have2) {
           uint32_t v2[32];
-          if (acc_valid) {
-            tc_ld32(taddr + (c + po) * 32, v2);
-            tc_ld_wait();
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v2[j] = 0u;
-          }
+          tc_ld32(taddr + (c + po) * 32, v2);
+          tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             f2[j] = __uint_as_float(v2[j]);
@@ -876,19 +830,17 @@ static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, 
 }
 
 int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_sms) {
-  if (G.M <= 0 || G.N <= 0 || G.K < 0 || (G.K == 0 && !(G.lora && G.lora_slab))) return 0;
+  if (G.M <= 0 || G.N <= 0) return 0;
+  if (G.K <= 0) return (int)cudaErrorInvalidValue;   // every tile needs at least one base k-block
   if (!g_encode) {
     const int e = gemm_tc_init();
     if (e) return e;
   }
   CUtensorMap tmA, tmB;
-  int e = 0;
-  if (G.K > 0) {
-    e = make_map(&tmA, G.A, (uint64_t)G.K, (uint64_t)G.M, (uint64_t)G.lda);
-    if (e) return 10000 + e;
-    e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
-    if (e) return 10000 + e;
-  }
+  int e = make_map(&tmA, G.A, (uint64_t)G.K, (uint64_t)G.M, (uint64_t)G.lda);
+  if (e) return 10000 + e;
+  e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
+  if (e) return 10000 + e;
   tc::Params P;
   P.M = G.M;
   P.N = G.swiglu ? G.N / 2 : G.N;
@@ -903,18 +855,15 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.kslot = G.kslot; P.khalf = G.khalf;
   P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
   CUtensorMap tmU = tmA;
-  P.a_mod = G.a_mod;
   P.group_m = G.group_m > 0 ? G.group_m : 16;
-  P.run_order = (P.slab && G.K == 0) ? 1 : 0;     // expansion only: amortise the generated operand
   P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp; P.rope_pos = G.rope_pos;
   if (P.slab) {
-    e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)(G.a_mod > 0 ? G.a_mod : G.M), (uint64_t)G.pack_ld);
+    e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)G.M, (uint64_t)G.pack_ld);
     if (e) return 10000 + e;
-    if (G.K == 0) tmA = tmB = tmU;                   // expansion only: no base product in this launch
   }
   P.status = status;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
-  if (G.cta_pair && P.M > tc::BM && G.K > 0) {
+  if (G.cta_pair && P.M > tc::BM) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
     static int max_clusters = 0;                       // co-resident pairs on this device
     cudaLaunchConfig_t cfg = {};

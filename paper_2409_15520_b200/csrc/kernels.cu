@@ -88,16 +88,17 @@ __global__ void norm_kernel(int kind, const T* __restrict__ x, T* __restrict__ o
   }
 }
 
-// Vectorised variant: 16-byte accesses, the row is read once and kept in registers.
-// Requires d % VEC == 0 and d <= blockDim.x * VEC * NV.
+// One block per row: 16-byte accesses, the row is read once and kept packed in registers (NV vectors
+// per thread), one shared-memory exchange per reduction.  Few registers per thread, so many rows are
+// in flight per SM.  Requires d % VEC == 0 and d <= TPB * VEC * NV with TPB = blockDim.x <= 256.
 template <typename T, int NV>
 __global__ void __launch_bounds__(256)
 norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
                 const T* __restrict__ b, int d, float eps, const int32_t* __restrict__ lab_idx,
                 int EP, int Tp) {
   constexpr int VEC = 16 / sizeof(T);
-  __shared__ float red[32];
-  const int row = blockIdx.x;
+  __shared__ float red[2][8];
+  const int row = blockIdx.x, tpb = blockDim.x, nw = tpb >> 5;
   long long src = row;
   if (lab_idx) {
     const int n = row / EP, j = row % EP;
@@ -107,64 +108,71 @@ norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T*
   T* o = out + (size_t)row * d;
   const int nvec = d / VEC;
   if (src < 0) {
-    for (int v = threadIdx.x; v < nvec; v += blockDim.x)
+    for (int v = threadIdx.x; v < nvec; v += tpb)
       *reinterpret_cast<uint4*>(o + v * VEC) = make_uint4(0, 0, 0, 0);
     return;
   }
   const T* xr = x + (size_t)src * d;
-  float val[NV][VEC];
+  uint4 raw[NV];
+#pragma unroll
+  for (int i = 0; i < NV; ++i) {
+    const int v = threadIdx.x + i * tpb;
+    raw[i] = v < nvec ? *reinterpret_cast<const uint4*>(xr + v * VEC) : make_uint4(0, 0, 0, 0);
+  }
   float s = 0.f;
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
-    const int v = threadIdx.x + i * blockDim.x;
-    if (v < nvec) {
-      const uint4 raw = *reinterpret_cast<const uint4*>(xr + v * VEC);
-      const T* e = reinterpret_cast<const T*>(&raw);
+    const T* e = reinterpret_cast<const T*>(&raw[i]);
 #pragma unroll
-      for (int j = 0; j < VEC; ++j) {
-        val[i][j] = to_f(e[j]);
-        s += kind == 0 ? val[i][j] : val[i][j] * val[i][j];
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < VEC; ++j) val[i][j] = 0.f;
+    for (int j = 0; j < VEC; ++j) {
+      const float t = to_f(e[j]);
+      s += kind == 0 ? t : t * t;
     }
   }
+  // block sum: one exchange through shared memory, every thread adds the warp partials itself
+  auto all_sum = [&](float v, float* r) {
+    v = warp_sum(v);
+    if ((threadIdx.x & 31) == 0) r[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float tot = 0.f;
+    for (int w = 0; w < nw; ++w) tot += r[w];
+    return tot;
+  };
+  s = all_sum(s, red[0]);
   float mu = 0.f, rstd;
   if (kind == 0) {
-    mu = block_sum(s, red) / d;
+    mu = s / d;
     float q = 0.f;
 #pragma unroll
     for (int i = 0; i < NV; ++i) {
-      const int v = threadIdx.x + i * blockDim.x;
-      if (v < nvec) {
+      if (threadIdx.x + i * tpb < nvec) {
+        const T* e = reinterpret_cast<const T*>(&raw[i]);
 #pragma unroll
         for (int j = 0; j < VEC; ++j) {
-          const float t = val[i][j] - mu;
+          const float t = to_f(e[j]) - mu;
           q += t * t;
         }
       }
     }
-    rstd = rsqrtf(block_sum(q, red) / d + eps);
+    rstd = rsqrtf(all_sum(q, red[1]) / d + eps);
   } else {
-    rstd = rsqrtf(block_sum(s, red) / d + eps);
+    rstd = rsqrtf(s / d + eps);
   }
 #pragma unroll
   for (int i = 0; i < NV; ++i) {
-    const int v = threadIdx.x + i * blockDim.x;
+    const int v = threadIdx.x + i * tpb;
     if (v < nvec) {
       const uint4 graw = *reinterpret_cast<const uint4*>(g + v * VEC);
       const T* ge = reinterpret_cast<const T*>(&graw);
       uint4 braw = make_uint4(0, 0, 0, 0);
       if (kind == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
       const T* be = reinterpret_cast<const T*>(&braw);
+      const T* e = reinterpret_cast<const T*>(&raw[i]);
       uint4 oraw;
       T* oe = reinterpret_cast<T*>(&oraw);
 #pragma unroll
-      for (int j = 0; j < VEC; ++j) {
-        const float y = (val[i][j] - mu) * rstd * to_f(ge[j]) + ((kind == 0 && b) ? to_f(be[j]) : 0.f);
-        oe[j] = from_f<T>(y);
-      }
+      for (int j = 0; j < VEC; ++j)
+        oe[j] = from_f<T>((to_f(e[j]) - mu) * rstd * to_f(ge[j]) + ((kind == 0 && b) ? to_f(be[j]) : 0.f));
       *reinterpret_cast<uint4*>(o + v * VEC) = oraw;
     }
   }
@@ -256,28 +264,28 @@ static void norm_dispatch(cudaStream_t st, int kind, const void* x, void* out, c
                           int Tp) {
   constexpr int VEC = 16 / sizeof(T);
   const bool aligned = (((uintptr_t)x | (uintptr_t)out | (uintptr_t)g | (uintptr_t)b) & 15) == 0;
-  if (aligned && d % VEC == 0 && d <= 32 * VEC * 16) {
-    const int nv = (d / VEC + 31) / 32;
+  const int nvec = d / VEC;
+  if (aligned && d % VEC == 0 && nvec <= 64) {
+    // short rows: one warp per row, four rows per block
+    const int nv = (nvec + 31) / 32;
     const int grid = (rows + 3) / 4;
-#define ZO_NW(NV) norm_warp_kernel<T, NV><<<grid, 128, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp)
-    if (nv <= 1) ZO_NW(1);
-    else if (nv <= 2) ZO_NW(2);
-    else if (nv <= 4) ZO_NW(4);
-    else if (nv <= 8) ZO_NW(8);
-    else ZO_NW(16);
-#undef ZO_NW
+    if (nv <= 1)
+      norm_warp_kernel<T, 1><<<grid, 128, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp);
+    else
+      norm_warp_kernel<T, 2><<<grid, 128, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp);
     return;
   }
-  if (aligned && d % VEC == 0 && d <= 256 * VEC * 4) {
-    const int nvec = d / VEC;
-    int th = nvec < 256 ? ((nvec + 31) / 32) * 32 : 256;
+  if (aligned && d % VEC == 0 && nvec <= 256 * 4) {
+    // two vectors per thread up to 256 threads, then more vectors per thread
+    int th = ((nvec + 1) / 2 + 31) / 32 * 32;
+    if (th > 256) th = 256;
     const int nv = (nvec + th - 1) / th;
-    if (nv <= 1)
-      norm_vec_kernel<T, 1><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
-    else if (nv == 2)
-      norm_vec_kernel<T, 2><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
-    else
-      norm_vec_kernel<T, 4><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp);
+#define ZO_NV(NV) norm_vec_kernel<T, NV><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp)
+    if (nv <= 1) ZO_NV(1);
+    else if (nv == 2) ZO_NV(2);
+    else if (nv == 3) ZO_NV(3);
+    else ZO_NV(4);
+#undef ZO_NV
     return;
   }
   const int th = d >= 2048 ? 256 : 128;

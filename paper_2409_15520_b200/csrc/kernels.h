@@ -67,7 +67,6 @@ struct GemmDesc {
   int rope_cols, rope_dh, rope_s, rope_tp;
   const int32_t* rope_pos;      // packed variable-length rows: position of row (m % rope_tp), else null
   int group_m;                  // 128-row tiles per raster group of the tensor-core kernel (0 = default 16)
-  int a_mod;                    // > 0 with lora_slab: packed-U row of output row m is m % a_mod (shared input)
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
 };
@@ -85,6 +84,13 @@ void launch_lora_down(cudaStream_t st, int bf, const void* X, int ldx, const voi
                       int rows, int K, int J);
 void launch_lora_apply(cudaStream_t st, int bf, const void* base, int ldb, int base_shared,
                        void* out, int ldo, int n, int T, const LoraDesc& L, int nsec);
+// Shared-input expansion on the bf16 path: out[j, t, :] = base[t, :] + s U[t, :] (B + k eps z) for the n
+// replicas of a pass (base and U on the T shared rows; out rows j * rows_per_replica + t), written with
+// full-line stores.  Supported when every section is a multiple of 128 columns, r <= 64 and rows are
+// 16-byte aligned.
+bool lora_expand_supported(const void* base, int ldb, const void* out, int ldo, const LoraDesc& L);
+void launch_lora_expand(cudaStream_t st, const void* base, int ldb, void* out, int ldo, int n, int T,
+                        const LoraDesc& L, int nsec, int n_sms);
 void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float theta);
 void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, SeqLayout sl, int d, int H,
                  const float* tab);

@@ -316,7 +316,11 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
   L.rep_base = ps.base; L.rep_stride = ps.stride;
-  PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
+  if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && lora_expand_supported(base, ko, Y, ko, L)) {
+    PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, base, ko, Y, ko, n, T, L, 1, c->n_sms));
+  } else {
+    PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
+  }
   PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss_pass));
   PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, nullptr, n, T, ps.base, ps.stride, rowloss, losses, losses_d, status));
   }
@@ -395,7 +399,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     void* ub = c->at<uint8_t>(c->plan.ub);
     if (J) {
       s = run_lora_down(c, st, bf, cf.flags, xn, d, lora->A[l], U, rows, d, J, status, c->n_sms,
-                        &c->launches, c->err, sizeof(c->err), slab ? ub : nullptr, nt * kslot, r, kslot);
+                        &c->launches, c->err, sizeof(c->err), (slab && !first) ? ub : nullptr, nt * kslot, r, kslot);
       if (s) return s;
     }
     // quantised storage: decode each weight right before its GEMM, once for all replicas of the pass
@@ -419,15 +423,9 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       // first perturbed layer: one base product on the shared block, expanded to 2q outputs
       G.out = qkv0; G.ldo = 3 * d;
       GEMM(G);
-      if (slab) {
-        // expansion on the tensor cores: no base k-blocks, only the LoRA block(s), base added as a
-        // residual that every replica shares
-        GemmDesc X{};
-        X.M = M; X.N = 3 * d; X.K = 0; X.out = qkv; X.ldo = 3 * d; X.res = qkv0; X.ldr = 3 * d; X.res_mod = Tp;
-        X.lora = &L; X.lora_slab = 1; X.pack_u = ub; X.pack_ld = nt * kslot; X.pack_r = r; X.kslot = kslot;
-        X.khalf = kslot / 2; X.a_mod = Tp; X.prof_class = PC_LORA_APPLY;
-        if (!opt) with_rope(X);
-        GEMM(X);
+      if (tcore && lora_expand_supported(qkv0, 3 * d, qkv, 3 * d, L)) {
+        // expansion to the 2q outputs of the pass: bound by the output stream, full-line stores
+        PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, qkv0, 3 * d, qkv, 3 * d, n, T, L, 3, c->n_sms));
       } else {
         PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
       }
@@ -823,7 +821,12 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   void* base = sp + 256 + up(rows * r * 4, 256);   // shared input: base product X W^T
   void* pack = (uint8_t*)base + (x_replicated ? 0 : up((size_t)T * k_out * (bf ? 2 : 4), 256));
   if (cudaMemsetAsync(status, 0, 4, st) != cudaSuccess) return ZO_ERR_CUDA;
-  const bool slab = slab_lora_ok(bf, flags, T, k_out, r);
+  LoraDesc L{};
+  L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
+  L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
+  L.scale = scale; L.eps = eps; L.seed = seed; L.tensor_base = tensor_id; L.rows_per_replica = T;
+  L.rep_base = 0; L.rep_stride = 1;
+  const bool slab = x_replicated && slab_lora_ok(bf, flags, T, k_out, r);
   const int kslot = r > 32 ? 128 : 64;
   if (slab && cudaMemsetAsync(pack, 0, rows * kslot * 2, st) != cudaSuccess) return ZO_ERR_CUDA;
   int launches = 0;
@@ -831,11 +834,6 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   zo_status s = run_lora_down(nullptr, st, bf, flags, X, k_in, A, U, (int)rows, k_in, r, status, sms,
                               &launches, err, sizeof(err), slab ? pack : nullptr, kslot, r, kslot);
   if (s) return s;
-  LoraDesc L{};
-  L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
-  L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
-  L.scale = scale; L.eps = eps; L.seed = seed; L.tensor_base = tensor_id; L.rows_per_replica = T;
-  L.rep_base = 0; L.rep_stride = 1;
   GemmDesc G{};
   G.A = X; G.lda = k_in; G.W = W; G.M = (int)rows; G.N = k_out; G.K = k_in; G.bias = bias;
   G.ldo = k_out;
@@ -843,13 +841,8 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
     G.out = base;
     s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
     if (s) return s;
-    if (slab) {
-      GemmDesc X{};
-      X.M = n * T; X.N = k_out; X.K = 0; X.out = Y; X.ldo = k_out; X.res = base; X.ldr = k_out; X.res_mod = T;
-      X.lora = &L; X.lora_slab = 1; X.pack_u = pack; X.pack_ld = kslot; X.pack_r = r; X.kslot = kslot;
-      X.khalf = kslot / 2; X.a_mod = T;
-      s = run_gemm(nullptr, st, bf, flags, X, status, sms, &launches, err, sizeof(err));
-      if (s) return s;
+    if (bf && !(flags & ZO_FLAG_SIMT_GEMM) && lora_expand_supported(base, k_out, Y, k_out, L)) {
+      launch_lora_expand(st, base, k_out, Y, k_out, n, T, L, 1, sms);
     } else {
       launch_lora_apply(st, bf, base, k_out, 1, Y, k_out, n, T, L, 1);
     }

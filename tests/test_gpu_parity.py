@@ -120,7 +120,7 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
     assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
 
 
-@pytest.mark.parametrize("arch,S", [(ARCH_LLAMA, 100), (ARCH_OPT, 64), (ARCH_LLAMA, 1)])
+@pytest.mark.parametrize("arch,S", [(ARCH_LLAMA, 100), (ARCH_OPT, 64), (ARCH_LLAMA, 1), (ARCH_LLAMA, 300)])
 def test_decoder_bf16_head_dim_128(arch, S):
     """Tensor-core attention with head_dim 128 (rotary embedding applied while staging), ragged
     and single-token sequences; compared with the oracle and with the CUDA-core attention."""
@@ -139,15 +139,15 @@ def test_decoder_bf16_head_dim_128(arch, S):
     assert np.allclose(got["losses"], simt["losses"], rtol=2e-3, atol=0), (got["losses"], simt["losses"])
 
 
-@pytest.mark.parametrize("x_replicated", [0, 1])
-@pytest.mark.parametrize("r", [8, 16, 64])
-def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
-    """The MP-LoRA layer equation on its own, both input modes, against the oracle's layer."""
+def _mp_lora_linear_case(x_replicated, r, T, ki, ko, q, pair_identical=True):
+    """Runs the MP-LoRA layer on its own through every GEMM implementation and checks it against the
+    oracle's layer: the outputs, and the difference of every +/- replica pair (which isolates the
+    perturbation term: its sign, its query index and its scale)."""
     import torch
     import paper_2409_15520_b200 as zo
     from workloads import bf16_round
     rng = np.random.default_rng(r + x_replicated)
-    T, ki, ko, q, eps, scale, seed, tid = 256, 328, 544, 2, 1e-2, 2.0, 77, 3
+    eps, scale, seed, tid = 1e-2, 2.0, 77, 3
     n = 2 * q
     X = bf16_round(rng.standard_normal((n if x_replicated else 1, T, ki)).astype(np.float32))
     W = bf16_round(0.05 * rng.standard_normal((ko, ki)).astype(np.float32))
@@ -167,11 +167,42 @@ def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
         outs[flags] = Y.float().cpu().numpy().astype(np.float64)
         err = np.max(np.abs(outs[flags] - ref))
         assert err < 2e-2 * np.max(np.abs(ref)), (flags, err, np.max(np.abs(ref)))
-    assert np.array_equal(outs[0], outs[PAIR])
-    # the perturbation must be visible in the outputs: replicas 0 and 1 differ as the oracle's do
-    d_gpu, d_ref = outs[0][0] - outs[0][1], ref[0] - ref[1]
-    assert np.max(np.abs(d_ref)) > 0
-    assert np.max(np.abs(d_gpu - d_ref)) < 0.1 * np.max(np.abs(d_ref)) + 2 * 2.0 ** -8 * np.max(np.abs(ref))
+    if pair_identical:     # CTA-pair and single-CTA kernels accumulate in the same order
+        assert np.array_equal(outs[0], outs[PAIR])
+    # the perturbation must be visible in the outputs: replicas 2i and 2i+1 differ as the oracle's do
+    for i in range(q):
+        d_gpu, d_ref = outs[0][2 * i] - outs[0][2 * i + 1], ref[2 * i] - ref[2 * i + 1]
+        assert np.max(np.abs(d_ref)) > 0
+        assert np.max(np.abs(d_gpu - d_ref)) < 0.1 * np.max(np.abs(d_ref)) + 2 * 2.0 ** -8 * np.max(np.abs(ref))
+    return outs
+
+
+@pytest.mark.parametrize("x_replicated", [0, 1])
+@pytest.mark.parametrize("r", [8, 16, 64])
+def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
+    """The MP-LoRA layer equation on its own, both input modes, against the oracle's layer (k_out is
+    not a multiple of the column tiles: the low-rank term runs in the GEMM epilogue or in the
+    CUDA-core expansion)."""
+    _mp_lora_linear_case(x_replicated, r, T=256, ki=328, ko=544, q=2)
+
+
+@pytest.mark.parametrize("r", [5, 8, 16, 32, 64])
+def test_mp_lora_linear_shared_input_expansion(r):
+    """Shared input with k_out a multiple of 128: the expansion kernel (operand generated once per
+    replica and column tile, warp-level tensor-core product, staged full-line stores) for every rank
+    class, a rank that is not a multiple of 4 or 8, and a ragged last row tile (T = 200)."""
+    outs = _mp_lora_linear_case(0, r, T=200, ki=328, ko=384, q=3)
+    # the CUDA-core expansion computes the same sums in fp32 from unrounded operands: the two agree to bf16 rounding
+    assert np.max(np.abs(outs[0] - outs[SIMT])) < 2.0 ** -6 * np.max(np.abs(outs[SIMT]))
+
+
+@pytest.mark.parametrize("r", [8, 64])
+def test_mp_lora_linear_replicated_input_slab(r):
+    """Replicated input with k_out a multiple of 256 and T of 128: the low-rank term as generated
+    tensor-core k-blocks (one for r <= 32, two above).  The CTA-pair kernel keeps the low-rank term in
+    its epilogue (fp32 from unrounded operands), so the two agree to bf16 rounding only."""
+    outs = _mp_lora_linear_case(1, r, T=256, ki=328, ko=512, q=2, pair_identical=False)
+    assert np.max(np.abs(outs[0] - outs[PAIR])) < 2.0 ** -6 * np.max(np.abs(outs[PAIR]))
 
 
 @pytest.mark.parametrize("bf16", [False, True])
