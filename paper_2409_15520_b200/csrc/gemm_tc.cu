@@ -59,6 +59,7 @@ struct Ctrl {
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
+  volatile uint32_t ep_last;
 };
 constexpr uint32_t SLAB_BYTES = BN * BK * 2;     // generated B operand of the LoRA k-block (aliases the fp32 staging)
 constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + SLAB_BYTES + sizeof(Ctrl);  // both variants: 192 KiB of stages
@@ -80,6 +81,9 @@ struct Params {
   int pack_r;
   LoraDesc L;
   uint32_t* status;
+  int ksplit;               // > 1: the K range of every tile is cut into ksplit units of work
+  float4* part;             // ksplit > 1: fp32 partial accumulators, [unit][64 column quads][128 rows]
+  int* tile_count;          // ksplit > 1: units of each tile that have delivered (returns to zero)
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -285,7 +289,7 @@ __device__ __forceinline__ int tile_slot(const Params& P, int n0) {
   return P.slab ? P.L.slot_of_sec[n0 / P.L.width] : -1;
 }
 
-template <bool PAIR>
+template <bool PAIR, bool SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmU, const Params P) {
@@ -309,9 +313,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_n = (P.N + ncol_tile - 1) / ncol_tile;
   const int num_tiles = tiles_m * tiles_n;
   const int num_kb = (P.K + BK - 1) / BK;
-  // Tile schedule of this CTA (pair): tiles unit, unit + n_units, ... of the grouped raster.
-  const int t_first = unit, t_step = n_units, t_end = num_tiles;
-  auto coords = [&](int t, int& tm, int& tn) { tile_coords(t, tiles_m, tiles_n, GROUP_M, tm, tn); };
+  // Work schedule of this CTA (pair): units unit, unit + n_units, ...  A unit is a tile of the grouped
+  // raster, or with split K (few tiles, long K: the weight stream has to be spread over all SMs) one of
+  // the ksplit K ranges of a tile.
+  const int ksplit = SPLIT ? P.ksplit : 1;            // (its own instantiation: the common case pays nothing)
+  const int t_first = unit, t_step = n_units, t_end = num_tiles * ksplit;
+  auto coords = [&](int t, int& tm, int& tn) { tile_coords(t / ksplit, tiles_m, tiles_n, GROUP_M, tm, tn); };
+  auto kb_range = [&](int t, int& ks, int& kb0, int& kb1) {
+    ks = t % ksplit;
+    kb0 = (int)((long long)ks * num_kb / ksplit);
+    kb1 = (int)((long long)(ks + 1) * num_kb / ksplit);
+  };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < MAX_STAGES; ++s) {
@@ -361,7 +373,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int m0 = tm * TILE_M + (int)rank * BM;
         const int brow0 = tn * ncol_tile;
         const int brow1 = P.swiglu ? P.N + brow0 : brow0 + 128;
-        for (int kb = 0; kb < num_kb; ++kb, ++issued) {
+        int ks, kb0, kb1;
+        kb_range(tile, ks, kb0, kb1);
+        for (int kb = kb0; kb < kb1; ++kb, ++issued) {
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
@@ -378,7 +392,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
           }
         }
-        const int lslot = PAIR ? -1 : tile_slot(P, brow0);
+        const int lslot = (PAIR || ks != 0) ? -1 : tile_slot(P, brow0);   // the LoRA block rides with the first K range
         for (int lkb = 0; ok && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued) {
           // LoRA k-blocks: only the A operand (packed U) travels through the ring
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
@@ -407,7 +421,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!mbar_wait(smem_u32(&ctrl->tempty[a]), aph ^ 1u, ctrl, P.status)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + a * BN;
-        for (int kb = 0; kb < num_kb; ++kb, ++consumed) {
+        int ks, kb0, kb1;
+        kb_range(tile, ks, kb0, kb1);
+        for (int kb = kb0; kb < kb1; ++kb, ++consumed) {
           const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status)) { ok = false; break; }
           tc_fence_after();
@@ -417,10 +433,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           for (int k = 0; k < BK / 16; ++k) {
             if (PAIR)
               tc_mma_pair(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC_PAIR,
-                          (uint32_t)((kb | k) != 0));
+                          (uint32_t)(((kb - kb0) | k) != 0));
             else
               tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC,
-                     (uint32_t)((kb | k) != 0));
+                     (uint32_t)(((kb - kb0) | k) != 0));
           }
           // frees the stage (in both CTAs of a pair) once these MMAs retire
           if (PAIR) tc_commit_pair(smem_u32(&ctrl->empty[s]));
@@ -429,7 +445,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!PAIR && ok) {
           int tm, tn;
           coords(tile, tm, tn);
-          if (tile_slot(P, tn * ncol_tile) >= 0) {
+          if (ks == 0 && tile_slot(P, tn * ncol_tile) >= 0) {
             for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++consumed) {
               const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
               if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
@@ -472,7 +488,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       coords(g_tile, tm, tn);
       const int n0g = tn * ncol_tile;
       const int slot = tile_slot(P, n0g);
-      if (slot < 0) return;                         // uniform over the CTA
+      if (slot < 0 || g_tile % ksplit != 0) return;  // uniform over the CTA (same decision as the MMA warp's)
       const int sec = n0g / P.L.width, cs = n0g - sec * P.L.width;
       const int repg = P.L.rep_base + P.L.rep_stride * ((tm * TILE_M) / P.L.rows_per_replica);
       const float sz = ((repg & 1) ? -P.L.eps : P.L.eps) * P.L.scale;
@@ -533,6 +549,61 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int row = m0 + wq * 32 + lane;
       const bool row_ok = row < P.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + a * BN;
+      constexpr bool split = SPLIT;
+      if (split) {
+        // Split K: deliver this unit's partial accumulator (all 256 columns; lanes = rows are contiguous
+        // in the scratch layout, so every access is a full 512-byte segment), hand the accumulator
+        // buffer back, and count the delivery.  The CTA that delivers a tile's last part runs the
+        // epilogue on the sum of the parts, taken in K order whichever CTA that is.
+        float4* pu = P.part + (size_t)tile * 64 * 128 + wq * 32 + lane;
+        for (int c = half; c < 8; c += 2) {
+          uint32_t v[32];
+          tc_ld32(taddr + c * 32, v);
+          tc_ld_wait();
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4)
+            pu[(size_t)(c * 8 + j4) * 128] =
+                make_float4(__uint_as_float(v[4 * j4]), __uint_as_float(v[4 * j4 + 1]),
+                            __uint_as_float(v[4 * j4 + 2]), __uint_as_float(v[4 * j4 + 3]));
+        }
+        __threadfence();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[a]));
+        ep_bar();
+        if (et == 0) {
+          int* cnt = P.tile_count + tile / ksplit;
+          const bool last = atomicAdd(cnt, 1) == ksplit - 1;
+          if (last) *cnt = 0;                      // every part has arrived: ready for the next launch
+          __threadfence();
+          ctrl->ep_last = last ? 1u : 0u;
+        }
+        ep_bar();
+        const bool last = ctrl->ep_last != 0u;
+        ep_bar();                                  // ep_last may be rewritten after this point
+        if (!last) continue;
+      }
+      // accumulator chunk `cchunk` (32 columns) of this thread's row: from tensor memory, or the sum of
+      // the tile's parts
+      auto load_acc = [&](int cchunk, uint32_t (&v)[32]) {
+        if (!split) {
+          tc_ld32(taddr + cchunk * 32, v);
+          return;
+        }
+        const float4* pp = P.part + (size_t)(tile - tile % ksplit) * 64 * 128 + (size_t)cchunk * 8 * 128 + wq * 32 + lane;
+        float sacc[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sacc[j] = 0.f;
+        for (int s2 = 0; s2 < ksplit; ++s2, pp += 64 * 128) {
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4) {
+            const float4 t4 = __ldcg(pp + j4 * 128);
+            sacc[4 * j4] += t4.x; sacc[4 * j4 + 1] += t4.y; sacc[4 * j4 + 2] += t4.z; sacc[4 * j4 + 3] += t4.w;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(sacc[j]);
+      };
       const int rrow = P.res ? (P.res_mod > 0 ? row % P.res_mod : row) : 0;
       // per-tile LoRA constants: all rows of the tile belong to one replica
       const int rep = P.has_lora ? P.L.rep_base + P.L.rep_stride * (m0 / P.L.rows_per_replica) : 0;
@@ -646,11 +717,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool rope_here = P.rope_tab != nullptr && col0 < P.rope_cols;
         if (rope_here && po > 0 && (c % (2 * po)) >= po) continue;   // done with its low partner
         uint32_t v[32];
-        tc_ld32(taddr + c * 32, v);
+        load_acc(c, v);
         float f[32];
         if (P.swiglu) {
           uint32_t up[32];
-          tc_ld32(taddr + 128 + c * 32, up);
+          load_acc(4 + c, up);
           tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -701,7 +772,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool have2 = rope_here && po > 0;
         if (have2) {
           uint32_t v2[32];
-          tc_ld32(taddr + (c + po) * 32, v2);
+          load_acc(c + po, v2);
           tc_ld_wait();
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -765,10 +836,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         emit(col0, f);
         if (have2) emit(col0 + po * 32, f2);
       }
-      // accumulator buffer drained: hand it back to the MMA warp
+      // accumulator buffer drained: hand it back to the MMA warp (split K did so when it delivered)
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) {
+      if (lane == 0 && !split) {
         if (PAIR) mbar_arrive_leader(smem_u32(&ctrl->tempty[a]));   // the leader waits for both CTAs
         else mbar_arrive(smem_u32(&ctrl->tempty[a]));
       }
@@ -809,10 +880,13 @@ int gemm_tc_init() {
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return e ? (int)e : 999;
   g_encode = (EncodeTiledFn)fn;
-  e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)tc::SMEM_BYTES);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
   return (int)e;
 }
@@ -862,6 +936,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     if (e) return 10000 + e;
   }
   P.status = status;
+  P.ksplit = 1; P.part = nullptr; P.tile_count = nullptr;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
   if (G.cta_pair && P.M > tc::BM) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
@@ -875,7 +950,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     if (max_clusters == 0) {
       cfg.gridDim = dim3(2 * (n_sms / 2));
       int mc = 0;
-      if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true>, &cfg) != cudaSuccess || mc < 1) {
+      if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true, false>, &cfg) != cudaSuccess || mc < 1) {
         cudaGetLastError();
         mc = n_sms / 2;
       }
@@ -885,12 +960,25 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     const int pairs = (int)(tiles < max_clusters ? tiles : max_clusters);
     cfg.gridDim = dim3(2 * pairs);
     P.slab = 0;
-    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true>, tmA, tmB, tmU, P);
+    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true, false>, tmA, tmB, tmU, P);
   }
   const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
   const long long tiles = (long long)tiles_m * tiles_n;
-  const int grid = (int)(tiles < n_sms ? tiles : n_sms);
-  tc::gemm_tc_kernel<false><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+  // Few tiles and a long K (small batches: the GEMM is a stream of weights): cut K so that the units
+  // of work cover the SMs, at least four k-blocks per unit.
+  const int num_kb = (G.K + tc::BK - 1) / tc::BK;
+  const int unit_cap = n_sms < G.split_units ? n_sms : G.split_units;
+  if (G.split_ws && G.split_cnt && tiles * 2 <= unit_cap && num_kb >= 8) {
+    int ks = (int)(unit_cap / tiles);
+    if (ks > num_kb / 4) ks = num_kb / 4;
+    if (ks >= 2) { P.ksplit = ks; P.part = (float4*)G.split_ws; P.tile_count = G.split_cnt; }
+  }
+  const long long units = tiles * P.ksplit;
+  const int grid = (int)(units < n_sms ? units : n_sms);
+  if (P.ksplit > 1)
+    tc::gemm_tc_kernel<false, true><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+  else
+    tc::gemm_tc_kernel<false, false><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
   return (int)cudaGetLastError();
 }
 

@@ -3,10 +3,11 @@
 // where base = X W^T (+ bias) and U = X A^T were computed once on the shared rows.  The op writes
 // n*T*k_out outputs from T*k_out inputs: it is bound by the output stream, so everything is arranged
 // for full-line accesses.  One CTA owns a (replica, 128-column tile) pair, generates that pair's
-// operand [s B ; s k eps z] (bf16, rank index along K) once, and sweeps row tiles of 128 tokens:
-// the base tile arrives through cp.async (double-buffered), the rank-2r product U'[U|U] x operand runs
-// on warp-level tensor-core MMAs (m16n8k16, fp32 accumulate), the sum is rounded once to bf16 and
-// leaves through shared memory as 16 bytes per lane on contiguous row segments.  Sections that carry
+// operand [s B ; s k eps z] (bf16, rank index along K) once, and sweeps row tiles of 128 tokens.
+// Inside a tile every warp runs a private pipeline on its 16 rows: the base rows arrive through
+// cp.async (double-buffered, one tile ahead), the rank-2r product [U|U] x operand runs on warp-level
+// tensor-core MMAs (m16n8k16, fp32 accumulate), the sum is rounded once to bf16 and leaves through
+// shared memory as 16 bytes per lane on contiguous row segments.  Sections that carry
 // no adapter are copied through the same pipeline.
 #include "kernels.h"
 #include "mma.cuh"
@@ -36,14 +37,19 @@ lora_expand_kernel(const bf16* __restrict__ base, int ldb, bf16* __restrict__ ou
   const int tile0 = blockIdx.z * tiles_per_cta, tile1 = min(ntile, tile0 + tiles_per_cta);
   if (tile0 >= tile1) return;
 
+  // Every warp runs its own pipeline over its 16 rows of each row tile: it stages those rows itself,
+  // so after the operand is built no CTA-wide barrier is needed.
+  bf16* Cw0 = Cs + warp * 16 * LDC;                    // the warp's rows in buffer 0 (buffer 1: + XT * LDC)
   auto stage_base = [&](int tile, int buf) {
-    bf16* dst = Cs + buf * XT * LDC;
+    const int wrow0 = tile * XT + warp * 16;
+    const int j0 = (lane & 15) * 8;
+    const bf16* src0 = base + col0 + j0;
+    const uint32_t d0 = (uint32_t)__cvta_generic_to_shared(Cw0 + buf * XT * LDC + (lane >> 4) * LDC + j0);
 #pragma unroll
-    for (int i = threadIdx.x; i < XT * (XT / 8); i += 256) {
-      const int rr = i >> 4, j0 = (i & 15) * 8;
-      const int row = tile * XT + rr;
-      const bf16* src = base + (size_t)min(row, T - 1) * ldb + col0 + j0;
-      cp_async16((uint32_t)__cvta_generic_to_shared(dst + rr * LDC + j0), src, row < T ? 16 : 0);
+    for (int k = 0; k < 8; ++k) {                      // two rows of 256 bytes per pass
+      const int row = wrow0 + 2 * k + (lane >> 4);
+      const bool ok = row < T;
+      cp_async16(d0 + 2 * k * LDC * 2, ok ? src0 + (size_t)row * ldb : src0, ok ? 16 : 0);
     }
   };
   stage_base(tile0, 0);
@@ -71,11 +77,35 @@ lora_expand_kernel(const bf16* __restrict__ base, int ldb, bf16* __restrict__ ou
         Bs[(c4 + j) * LDB + r + k] = __float2bfloat16_rn(zz[j] * sz);
       }
     }
+    __syncthreads();                                   // operand complete: the only CTA-wide hand-over
   }
+
+  // A = [U | U | 0] of the warp's 16 rows of a tile, rounded to bf16 as it is loaded (fragment order of
+  // the m16n8k16 A operand).  Short operands are fetched one tile ahead.
+  constexpr int NKS = KT / 16;
+  constexpr bool PREFETCH_A = KT <= 32;
+  auto load_a = [&](int tile, uint32_t (&af)[NKS][4]) {
+    const int ra = tile * XT + warp * 16 + g, rb = ra + 8;
+    const float* ua = L.U + (size_t)min(ra, T - 1) * L.ldu + slot * r;
+    const float* ub = L.U + (size_t)min(rb, T - 1) * L.ldu + slot * r;
+    auto aval = [&](const float* u, bool ok, int kk) -> float {
+      return (ok && kk < 2 * r) ? u[kk < r ? kk : kk - r] : 0.f;
+    };
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks) {
+      const int k0 = ks * 16 + 2 * t;
+      af[ks][0] = pack2(aval(ua, ra < T, k0), aval(ua, ra < T, k0 + 1));
+      af[ks][1] = pack2(aval(ub, rb < T, k0), aval(ub, rb < T, k0 + 1));
+      af[ks][2] = pack2(aval(ua, ra < T, k0 + 8), aval(ua, ra < T, k0 + 9));
+      af[ks][3] = pack2(aval(ub, rb < T, k0 + 8), aval(ub, rb < T, k0 + 9));
+    }
+  };
+  uint32_t af[NKS][4];
+  if (slot >= 0 && PREFETCH_A) load_a(tile0, af);
 
   for (int tile = tile0; tile < tile1; ++tile) {
     const int buf = (tile - tile0) & 1;
-    __syncthreads();                                   // operand written; everyone is done with the other buffer
+    __syncwarp();                                      // every lane is done with the other buffer
     if (tile + 1 < tile1) stage_base(tile + 1, buf ^ 1);
     cp_commit();                                       // (possibly empty: keeps the group count uniform)
     const int wrow0 = tile * XT + warp * 16;           // first token row of this warp
@@ -85,36 +115,26 @@ lora_expand_kernel(const bf16* __restrict__ base, int ldb, bf16* __restrict__ ou
 #pragma unroll
       for (int i = 0; i < 4; ++i) acc[j][i] = 0.f;
     if (slot >= 0 && wrow0 < T) {
-      // A = [U | U | 0] of the warp's 16 rows, rounded to bf16 as it is loaded
-      const int ra = wrow0 + g, rb = ra + 8;
-      const float* ua = L.U + (size_t)min(ra, T - 1) * L.ldu + slot * r;
-      const float* ub = L.U + (size_t)min(rb, T - 1) * L.ldu + slot * r;
-      auto aval = [&](const float* u, bool ok, int kk) -> float {
-        return (ok && kk < 2 * r) ? u[kk < r ? kk : kk - r] : 0.f;
-      };
+      if (!PREFETCH_A) load_a(tile, af);
 #pragma unroll
-      for (int ks = 0; ks < KT / 16; ++ks) {
+      for (int ks = 0; ks < NKS; ++ks) {
         if (ks * 16 >= 2 * r) break;                   // nothing but zeros from here on
-        const int k0 = ks * 16 + 2 * t;
-        const uint32_t a0 = pack2(aval(ua, ra < T, k0), aval(ua, ra < T, k0 + 1));
-        const uint32_t a1 = pack2(aval(ub, rb < T, k0), aval(ub, rb < T, k0 + 1));
-        const uint32_t a2 = pack2(aval(ua, ra < T, k0 + 8), aval(ua, ra < T, k0 + 9));
-        const uint32_t a3 = pack2(aval(ub, rb < T, k0 + 8), aval(ub, rb < T, k0 + 9));
 #pragma unroll
         for (int jp = 0; jp < XT / 16; ++jp) {          // two 8-column tiles per ldmatrix
           uint32_t b0, b1, b2, b3;
           const int col = jp * 16 + (lane & 7) + (lane >> 4) * 8;
           const int c = ks * 16 + ((lane >> 3) & 1) * 8;
           ldsm_x4((uint32_t)__cvta_generic_to_shared(Bs + col * LDB + c), b0, b1, b2, b3);
-          mma_bf16(acc[2 * jp], a0, a1, a2, a3, b0, b1);
-          mma_bf16(acc[2 * jp + 1], a0, a1, a2, a3, b2, b3);
+          mma_bf16(acc[2 * jp], af[ks][0], af[ks][1], af[ks][2], af[ks][3], b0, b1);
+          mma_bf16(acc[2 * jp + 1], af[ks][0], af[ks][1], af[ks][2], af[ks][3], b2, b3);
         }
       }
+      if (PREFETCH_A && tile + 1 < tile1) load_a(tile + 1, af);   // lands under the stores below
     }
-    cp_wait<1>();                                      // this tile's base rows have landed
-    __syncthreads();
-    if (wrow0 >= T) continue;                          // (the barriers above stay uniform)
-    bf16* Cw = Cs + buf * XT * LDC + warp * 16 * LDC;  // the warp's 16 rows
+    cp_wait<1>();                                      // this lane's share of the tile's base rows has landed
+    __syncwarp();                                      // ... and so has every other lane's
+    if (wrow0 >= T) continue;
+    bf16* Cw = Cw0 + buf * XT * LDC;
     if (slot >= 0) {
 #pragma unroll
       for (int h = 0; h < 2; ++h) {

@@ -120,6 +120,27 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
     assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
 
 
+@pytest.mark.parametrize("arch,q", [(ARCH_LLAMA, 1), (ARCH_OPT, 2)])
+def test_decoder_bf16_small_batch_split_k(arch, q):
+    """One short sequence (a single 128-row tile per replica) with k_in = 512 and 1024: too few tiles
+    for the SMs, so the tensor-core GEMMs cut K into units of work and the CTA that delivers a tile's
+    last part sums the parts in K order and runs the fused epilogue (bias, residual, rotary embedding,
+    LoRA k-block with the first part).  Checked against the oracle and the CUDA-core GEMM, and for
+    run-to-run bit-identity (the sum order does not depend on which CTA finishes last)."""
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
+                     **{**TINY, "d_model": 512, "n_heads": 4, "d_ffn": 1024, "vocab": 517, "S": 40,
+                        "E": 1, "max_seq": 40, "q": q, "n_layers": 2, "lora_rank": 8})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 47)
+    got = run_gpu(spec, p, 47)
+    again = run_gpu(spec, p, 47)
+    simt = run_gpu(spec, p, 47, flags=SIMT)
+    assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
+    assert np.allclose(got["losses"], simt["losses"], rtol=3e-3, atol=0), (got["losses"], simt["losses"])
+    assert np.array_equal(got["losses"], again["losses"]) and np.array_equal(got["rows"], again["rows"])
+    assert np.array_equal(got["B"][0], again["B"][0])
+
+
 @pytest.mark.parametrize("arch,S", [(ARCH_LLAMA, 100), (ARCH_OPT, 64), (ARCH_LLAMA, 1), (ARCH_LLAMA, 300)])
 def test_decoder_bf16_head_dim_128(arch, S):
     """Tensor-core attention with head_dim 128 (rotary embedding applied while staging), ragged
