@@ -87,7 +87,10 @@ enum { ZO_FLAG_SIMT_GEMM = 1,
         * U, B and k eps z to bfloat16).  A/B switch. */
        ZO_FLAG_LORA_EPILOGUE = 4 };
 /* Bits 8..15 of flags, when non-zero, override the tensor-core GEMM's raster group (128-row tiles that
- * sweep the weight panels together; default 16).  Tuning aid; results do not depend on it. */
+ * sweep the weight panels together; default 16).  Tuning aid; results do not depend on it.
+ * Bits 16..20, when non-zero, bound the number of K ranges the tensor-core GEMM cuts a tile into when a
+ * launch has fewer tiles than SMs (small batches; 1 = never split).  Tuning aid; the sum order, and
+ * with it the last bits of the result, depends on the number of ranges, not on the run. */
 
 typedef struct zo_ctx zo_ctx; /* opaque; owned by the library; released by zo_free */
 

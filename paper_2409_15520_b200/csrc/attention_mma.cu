@@ -179,8 +179,8 @@ attention_mma_kernel(const bf16* __restrict__ qkv, bf16* __restrict__ ctx, SeqLa
         }
       }
     }
-    __syncthreads();                                            // every warp is done with this buffer
-    if (kt + 2 < n_kt) {
+    if (kt + 2 < n_kt) {                                        // uniform over the CTA
+      __syncthreads();                                          // every warp is done with this buffer
       stage_tile_async<DH, 64>(Ks + (kt & 1) * TILE, seq, ld, d + h * DH, k0 + 128, S);
       stage_tile_async<DH, 64>(Vs + (kt & 1) * TILE, seq, ld, 2 * d + h * DH, k0 + 128, S);
     }

@@ -24,6 +24,9 @@
 //     the weight tile, so the shared-memory traffic per SM drops by a third; 6 stages.  The
 //     leader CTA issues the MMAs and releases stages/accumulators in both CTAs with multicast
 //     commits; the peer's TMA completes on the leader's barrier.
+//   * split K for small batches (far fewer tiles than SMs, cost = the stream of weights): a first
+//     launch computes one K range of a tile per CTA and stores fp32 parts, a second launch of the
+//     same template sums them in K order and runs the fused epilogue; no CTA waits for another.
 //   * every mbarrier wait is bounded; on expiry the kernel raises ST_TIMEOUT in the status
 //     word, drains its copies and MMAs, frees its tensor memory and returns.
 #include <cuda.h>
@@ -59,7 +62,6 @@ struct Ctrl {
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
-  volatile uint32_t ep_last;
 };
 constexpr uint32_t SLAB_BYTES = BN * BK * 2;     // generated B operand of the LoRA k-block (aliases the fp32 staging)
 constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + SLAB_BYTES + sizeof(Ctrl);  // both variants: 192 KiB of stages
@@ -83,7 +85,6 @@ struct Params {
   uint32_t* status;
   int ksplit;               // > 1: the K range of every tile is cut into ksplit units of work
   float4* part;             // ksplit > 1: fp32 partial accumulators, [unit][64 column quads][128 rows]
-  int* tile_count;          // ksplit > 1: units of each tile that have delivered (returns to zero)
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -289,7 +290,13 @@ __device__ __forceinline__ int tile_slot(const Params& P, int n0) {
   return P.slab ? P.L.slot_of_sec[n0 / P.L.width] : -1;
 }
 
-template <bool PAIR, bool SPLIT>
+// SPLIT 0: every CTA (pair) computes whole tiles.  Split K, for launches with far fewer tiles than SMs
+// whose cost is the stream of weights (small batches), takes two launches of this kernel: SPLIT 1
+// computes one K range of a tile per unit of work and stores the fp32 accumulator to scratch; SPLIT 2
+// runs no MMA at all: its CTAs take a quarter of a tile's column chunks each, sum the parts in K order
+// (so the result does not depend on timing) and run the same fused epilogue as SPLIT 0.
+constexpr int FIN_GROUPS = 4;
+template <bool PAIR, int SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmU, const Params P) {
@@ -314,9 +321,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int num_tiles = tiles_m * tiles_n;
   const int num_kb = (P.K + BK - 1) / BK;
   // Work schedule of this CTA (pair): units unit, unit + n_units, ...  A unit is a tile of the grouped
-  // raster, or with split K (few tiles, long K: the weight stream has to be spread over all SMs) one of
-  // the ksplit K ranges of a tile.
-  const int ksplit = SPLIT ? P.ksplit : 1;            // (its own instantiation: the common case pays nothing)
+  // raster, or with split K one of the ksplit K ranges of a tile.
+  const int ksplit = SPLIT ? P.ksplit : 1;
   const int t_first = unit, t_step = n_units, t_end = num_tiles * ksplit;
   auto coords = [&](int t, int& tm, int& tn) { tile_coords(t / ksplit, tiles_m, tiles_n, GROUP_M, tm, tn); };
   auto kb_range = [&](int t, int& ks, int& kb0, int& kb1) {
@@ -341,7 +347,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {
+  if (warp == 1 && SPLIT != 2) {
     if (PAIR) {
       asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
                        smem_u32(&ctrl->tmem_base)),
@@ -364,7 +370,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && SPLIT != 2) {
       uint32_t issued = 0;
       bool ok = true;
       for (int tile = t_first; tile < t_end && ok; tile += t_step) {
@@ -413,7 +419,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && rank == 0) {
+    if (lane == 0 && rank == 0 && SPLIT != 2) {
       uint32_t consumed = 0, titer = 0, ltiles = 0;
       bool ok = true;
       for (int tile = t_first; tile < t_end && ok; tile += t_step, ++titer) {
@@ -526,37 +532,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&ctrl->lfull));
     };
-    if (!PAIR && P.slab) {
+    if (!PAIR && P.slab && SPLIT != 2) {
       for (int i = et; i < (int)(SLAB_BYTES / 16) * (P.kslot / BK); i += EP_THREADS)
         reinterpret_cast<uint4*>(slab)[i] = make_uint4(0, 0, 0, 0);
       ep_bar();
     }
-    if (!PAIR && P.slab && t_first < t_end) gen_slab(t_first);
+    if (!PAIR && P.slab && SPLIT != 2 && t_first < t_end) gen_slab(t_first);
     uint32_t titer = 0;
-    for (int tile = t_first; tile < t_end; tile += t_step, ++titer) {
+    // iteration space: the units of this CTA; in the summing launch (tile, chunk group) pairs
+    const int e_first = SPLIT == 2 ? (int)blockIdx.x : t_first;
+    const int e_step = SPLIT == 2 ? (int)gridDim.x : t_step;
+    const int e_end = SPLIT == 2 ? num_tiles * FIN_GROUPS : t_end;
+    for (int it = e_first; it < e_end; it += e_step, ++titer) {
+      const int tile = SPLIT == 2 ? (it / FIN_GROUPS) * ksplit : it;   // (summing launch: first unit of the tile)
+      const int grp = SPLIT == 2 ? it % FIN_GROUPS : -1;
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
-      if (et == 0) ctrl->ep_go = mbar_wait(smem_u32(&ctrl->tfull[a]), aph, ctrl, P.status) ? 1u : 0u;
-      ep_bar();
-      const bool go = ctrl->ep_go != 0u;
-      ep_bar();                                    // ep_go may be rewritten after this point
-      if (!go) break;
-      tc_fence_after();
-      // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
-      if (!PAIR && P.slab && tile + t_step < t_end) gen_slab(tile + t_step);
+      if (SPLIT != 2) {
+        if (et == 0) ctrl->ep_go = mbar_wait(smem_u32(&ctrl->tfull[a]), aph, ctrl, P.status) ? 1u : 0u;
+        ep_bar();
+        const bool go = ctrl->ep_go != 0u;
+        ep_bar();                                    // ep_go may be rewritten after this point
+        if (!go) break;
+        tc_fence_after();
+        // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
+        if (!PAIR && P.slab && tile + t_step < t_end) gen_slab(tile + t_step);
+      }
       int tm, tn;
       coords(tile, tm, tn);
       const int m0 = tm * TILE_M + (int)rank * BM, n0 = tn * ncol_tile;
       const int row = m0 + wq * 32 + lane;
       const bool row_ok = row < P.M;
       const uint32_t taddr = tmem_base + ((uint32_t)(wq * 32) << 16) + a * BN;
-      constexpr bool split = SPLIT;
-      if (split) {
-        // Split K: deliver this unit's partial accumulator (all 256 columns; lanes = rows are contiguous
-        // in the scratch layout, so every access is a full 512-byte segment), hand the accumulator
-        // buffer back, and count the delivery.  The CTA that delivers a tile's last part runs the
-        // epilogue on the sum of the parts, taken in K order whichever CTA that is.
+      constexpr bool split = SPLIT != 0;
+      if (SPLIT == 1) {
+        // deliver this unit's partial accumulator (the chunks that hold output columns; lanes = rows are
+        // contiguous in the scratch layout, so every access is a full 512-byte segment) and hand the
+        // accumulator buffer back
         float4* pu = P.part + (size_t)tile * 64 * 128 + wq * 32 + lane;
-        for (int c = half; c < 8; c += 2) {
+        const int cvalid = P.swiglu ? 8 : min(8, (P.N - n0 + 31) / 32);   // chunks that hold output columns
+        for (int c = half; c < cvalid; c += 2) {
           uint32_t v[32];
           tc_ld32(taddr + c * 32, v);
           tc_ld_wait();
@@ -566,22 +580,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 make_float4(__uint_as_float(v[4 * j4]), __uint_as_float(v[4 * j4 + 1]),
                             __uint_as_float(v[4 * j4 + 2]), __uint_as_float(v[4 * j4 + 3]));
         }
-        __threadfence();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->tempty[a]));
-        ep_bar();
-        if (et == 0) {
-          int* cnt = P.tile_count + tile / ksplit;
-          const bool last = atomicAdd(cnt, 1) == ksplit - 1;
-          if (last) *cnt = 0;                      // every part has arrived: ready for the next launch
-          __threadfence();
-          ctrl->ep_last = last ? 1u : 0u;
-        }
-        ep_bar();
-        const bool last = ctrl->ep_last != 0u;
-        ep_bar();                                  // ep_last may be rewritten after this point
-        if (!last) continue;
+        continue;
       }
       // accumulator chunk `cchunk` (32 columns) of this thread's row: from tensor memory, or the sum of
       // the tile's parts
@@ -590,15 +592,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           tc_ld32(taddr + cchunk * 32, v);
           return;
         }
-        const float4* pp = P.part + (size_t)(tile - tile % ksplit) * 64 * 128 + (size_t)cchunk * 8 * 128 + wq * 32 + lane;
+        const float4* pp = P.part + (size_t)tile * 64 * 128 + (size_t)cchunk * 8 * 128 + wq * 32 + lane;
         float sacc[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) sacc[j] = 0.f;
-        for (int s2 = 0; s2 < ksplit; ++s2, pp += 64 * 128) {
+        // two parts per round: the loads of a round are all in flight before the first add, and the
+        // adds stay in K order
+        for (int s2 = 0; s2 < ksplit; s2 += 2, pp += 2 * 64 * 128) {
+          const bool two = s2 + 1 < ksplit;
+          float4 t0[8], t1[8];
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4) t0[j4] = __ldcg(pp + j4 * 128);
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4) t1[j4] = two ? __ldcg(pp + 64 * 128 + j4 * 128) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
           for (int j4 = 0; j4 < 8; ++j4) {
-            const float4 t4 = __ldcg(pp + j4 * 128);
-            sacc[4 * j4] += t4.x; sacc[4 * j4 + 1] += t4.y; sacc[4 * j4 + 2] += t4.z; sacc[4 * j4 + 3] += t4.w;
+            sacc[4 * j4] += t0[j4].x; sacc[4 * j4 + 1] += t0[j4].y; sacc[4 * j4 + 2] += t0[j4].z; sacc[4 * j4 + 3] += t0[j4].w;
+          }
+          if (two) {
+#pragma unroll
+            for (int j4 = 0; j4 < 8; ++j4) {
+              sacc[4 * j4] += t1[j4].x; sacc[4 * j4 + 1] += t1[j4].y; sacc[4 * j4 + 2] += t1[j4].z; sacc[4 * j4 + 3] += t1[j4].w;
+            }
           }
         }
 #pragma unroll
@@ -713,6 +728,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         } else if (((c >> pshift) & 1) != half) {
           continue;
         }
+        // summing launch: this CTA owns a quarter of the chunks (a rotary pair stays together)
+        if (SPLIT == 2 && (po == 2 ? (c & 1) + 2 * (c >> 2) : (c >> 1)) != grp) continue;
         // rotary embedding fused here: the pair (j, j + dh/2) of a head sits po chunks apart
         const bool rope_here = P.rope_tab != nullptr && col0 < P.rope_cols;
         if (rope_here && po > 0 && (c % (2 * po)) >= po) continue;   // done with its low partner
@@ -850,7 +867,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   tc_fence_before();
   __syncthreads();
   if (PAIR) cluster_sync();      // neither CTA leaves while the other may still signal or write into it
-  if (warp == 1) {
+  if (warp == 1 && SPLIT != 2) {
     __syncwarp();
     tc_fence_after();
     if (PAIR)
@@ -880,13 +897,16 @@ int gemm_tc_init() {
   cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
   if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return e ? (int)e : 999;
   g_encode = (EncodeTiledFn)fn;
-  e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            (int)tc::SMEM_BYTES);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
   return (int)e;
 }
@@ -936,7 +956,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     if (e) return 10000 + e;
   }
   P.status = status;
-  P.ksplit = 1; P.part = nullptr; P.tile_count = nullptr;
+  P.ksplit = 1; P.part = nullptr;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
   if (G.cta_pair && P.M > tc::BM) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
@@ -950,7 +970,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     if (max_clusters == 0) {
       cfg.gridDim = dim3(2 * (n_sms / 2));
       int mc = 0;
-      if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true, false>, &cfg) != cudaSuccess || mc < 1) {
+      if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true, 0>, &cfg) != cudaSuccess || mc < 1) {
         cudaGetLastError();
         mc = n_sms / 2;
       }
@@ -960,7 +980,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     const int pairs = (int)(tiles < max_clusters ? tiles : max_clusters);
     cfg.gridDim = dim3(2 * pairs);
     P.slab = 0;
-    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true, false>, tmA, tmB, tmU, P);
+    return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true, 0>, tmA, tmB, tmU, P);
   }
   const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
   const long long tiles = (long long)tiles_m * tiles_n;
@@ -968,17 +988,21 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   // of work cover the SMs, at least four k-blocks per unit.
   const int num_kb = (G.K + tc::BK - 1) / tc::BK;
   const int unit_cap = n_sms < G.split_units ? n_sms : G.split_units;
-  if (G.split_ws && G.split_cnt && tiles * 2 <= unit_cap && num_kb >= 8) {
+  if (G.split_ws && tiles * 2 <= unit_cap && num_kb >= 8) {
     int ks = (int)(unit_cap / tiles);
     if (ks > num_kb / 4) ks = num_kb / 4;
-    if (ks >= 2) { P.ksplit = ks; P.part = (float4*)G.split_ws; P.tile_count = G.split_cnt; }
+    if (G.split_cap > 0 && ks > G.split_cap) ks = G.split_cap;
+    if (ks >= 2) { P.ksplit = ks; P.part = (float4*)G.split_ws; }
   }
   const long long units = tiles * P.ksplit;
   const int grid = (int)(units < n_sms ? units : n_sms);
-  if (P.ksplit > 1)
-    tc::gemm_tc_kernel<false, true><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
-  else
-    tc::gemm_tc_kernel<false, false><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+  if (P.ksplit > 1) {
+    tc::gemm_tc_kernel<false, 1><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+    const long long fin = tiles * tc::FIN_GROUPS;
+    tc::gemm_tc_kernel<false, 2><<<(int)(fin < n_sms ? fin : n_sms), tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+    if (G.extra_launches) ++*G.extra_launches;
+  } else
+    tc::gemm_tc_kernel<false, 0><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
   return (int)cudaGetLastError();
 }
 

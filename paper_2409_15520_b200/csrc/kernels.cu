@@ -90,10 +90,11 @@ __global__ void norm_kernel(int kind, const T* __restrict__ x, T* __restrict__ o
 
 // One block per row: 16-byte accesses, the row is read once and kept packed in registers (NV vectors
 // per thread), one shared-memory exchange per reduction.  Few registers per thread, so many rows are
-// in flight per SM.  Requires d % VEC == 0 and d <= TPB * VEC * NV with TPB = blockDim.x <= 256.
-template <typename T, int NV>
+// in flight per SM.  KIND 0 = LayerNorm, 1 = RMSNorm (compiled apart: the kernel is close to its issue
+// limit, so the RMS path carries no mean or bias arithmetic).  Requires d % VEC == 0 and d <= TPB * VEC * NV with TPB = blockDim.x <= 256.
+template <typename T, int NV, int KIND>
 __global__ void __launch_bounds__(256)
-norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
+norm_vec_kernel(const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
                 const T* __restrict__ b, int d, float eps, const int32_t* __restrict__ lab_idx,
                 int EP, int Tp) {
   constexpr int VEC = 16 / sizeof(T);
@@ -126,7 +127,7 @@ norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T*
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
       const float t = to_f(e[j]);
-      s += kind == 0 ? t : t * t;
+      s += KIND == 0 ? t : t * t;
     }
   }
   // block sum: one exchange through shared memory, every thread adds the warp partials itself
@@ -140,7 +141,7 @@ norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T*
   };
   s = all_sum(s, red[0]);
   float mu = 0.f, rstd;
-  if (kind == 0) {
+  if (KIND == 0) {
     mu = s / d;
     float q = 0.f;
 #pragma unroll
@@ -165,14 +166,16 @@ norm_vec_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T*
       const uint4 graw = *reinterpret_cast<const uint4*>(g + v * VEC);
       const T* ge = reinterpret_cast<const T*>(&graw);
       uint4 braw = make_uint4(0, 0, 0, 0);
-      if (kind == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
+      if (KIND == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
       const T* be = reinterpret_cast<const T*>(&braw);
       const T* e = reinterpret_cast<const T*>(&raw[i]);
       uint4 oraw;
       T* oe = reinterpret_cast<T*>(&oraw);
 #pragma unroll
-      for (int j = 0; j < VEC; ++j)
-        oe[j] = from_f<T>((to_f(e[j]) - mu) * rstd * to_f(ge[j]) + ((kind == 0 && b) ? to_f(be[j]) : 0.f));
+      for (int j = 0; j < VEC; ++j) {
+        if (KIND == 0) oe[j] = from_f<T>((to_f(e[j]) - mu) * rstd * to_f(ge[j]) + (b ? to_f(be[j]) : 0.f));
+        else oe[j] = from_f<T>(to_f(e[j]) * rstd * to_f(ge[j]));
+      }
       *reinterpret_cast<uint4*>(o + v * VEC) = oraw;
     }
   }
@@ -280,7 +283,13 @@ static void norm_dispatch(cudaStream_t st, int kind, const void* x, void* out, c
     int th = ((nvec + 1) / 2 + 31) / 32 * 32;
     if (th > 256) th = 256;
     const int nv = (nvec + th - 1) / th;
-#define ZO_NV(NV) norm_vec_kernel<T, NV><<<rows, th, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp)
+#define ZO_NV(NV)                                                                                              \
+  do {                                                                                                         \
+    if (kind == 0)                                                                                             \
+      norm_vec_kernel<T, NV, 0><<<rows, th, 0, st>>>((const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp); \
+    else                                                                                                       \
+      norm_vec_kernel<T, NV, 1><<<rows, th, 0, st>>>((const T*)x, (T*)out, (const T*)g, (const T*)b, d, eps, lab_idx, EP, Tp); \
+  } while (0)
     if (nv <= 1) ZO_NV(1);
     else if (nv == 2) ZO_NV(2);
     else if (nv == 3) ZO_NV(3);

@@ -70,8 +70,9 @@ struct GemmDesc {
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
   int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
   float* split_ws;              // split-K scratch of the tensor-core kernel: split_units * 32768 floats, or null
-  int* split_cnt;               // split_units counters, zero before the first launch (the kernel restores zero)
   int split_units;
+  int* extra_launches;          // incremented when the GEMM took a second launch (split K), or null
+  int split_cap;                // > 0: upper bound on the number of K ranges per tile (1 = never split)
 };
 
 // --- elementwise / reduction kernels (bf = 1: bfloat16 tensors, 0: float) -------------------

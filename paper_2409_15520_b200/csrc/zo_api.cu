@@ -18,7 +18,7 @@ char g_init_error[256] = "";
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
-      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, pos, split_cnt, split_ws, total;
+      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, pos, split_ws, total;
 };
 
 inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -142,7 +142,6 @@ Plan make_plan(const zo_config& c) {
   p.g = take((size_t)c.max_q * 4);
   p.status = take(256);
   if (c.precision == ZO_BF16) {             // split-K scratch of the tensor-core GEMM (small batches)
-    p.split_cnt = take(SPLIT_UNITS * 4);
     p.split_ws = take((size_t)SPLIT_UNITS * 128 * 256 * 4);
   }
   p.total = off;
@@ -219,8 +218,9 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
     GemmDesc Gt = G;
     Gt.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
     Gt.group_m = (int)((flags >> 8) & 0xFF);     // diagnostic: raster group override in bits 8..15
+    Gt.split_cap = (int)((flags >> 16) & 0x1F);  // diagnostic: bound on the split-K factor in bits 16..20
     if (c && c->plan.split_ws) {
-      Gt.split_ws = c->at<float>(c->plan.split_ws); Gt.split_cnt = c->at<int>(c->plan.split_cnt); Gt.split_units = SPLIT_UNITS;
+      Gt.split_ws = c->at<float>(c->plan.split_ws); Gt.split_units = SPLIT_UNITS; Gt.extra_launches = launches;
     }
     const int e = launch_gemm_tc(st, Gt, status, n_sms);
     if (e) {
@@ -247,7 +247,7 @@ zo_status run_lora_down(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, cons
     G.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
     G.pack_out = pack_out; G.pack_ld = pack_ld; G.pack_r = pack_r; G.kslot = kslot; G.khalf = kslot / 2;
     if (c && c->plan.split_ws) {
-      G.split_ws = c->at<float>(c->plan.split_ws); G.split_cnt = c->at<int>(c->plan.split_cnt); G.split_units = SPLIT_UNITS;
+      G.split_ws = c->at<float>(c->plan.split_ws); G.split_units = SPLIT_UNITS; G.extra_launches = launches;
     }
     ProfScope ps(c, PC_LORA_DOWN, 2.0 * rows * (double)J * K);
     const int e = launch_gemm_tc(st, G, status, n_sms);

@@ -123,10 +123,10 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
 @pytest.mark.parametrize("arch,q", [(ARCH_LLAMA, 1), (ARCH_OPT, 2)])
 def test_decoder_bf16_small_batch_split_k(arch, q):
     """One short sequence (a single 128-row tile per replica) with k_in = 512 and 1024: too few tiles
-    for the SMs, so the tensor-core GEMMs cut K into units of work and the CTA that delivers a tile's
-    last part sums the parts in K order and runs the fused epilogue (bias, residual, rotary embedding,
-    LoRA k-block with the first part).  Checked against the oracle and the CUDA-core GEMM, and for
-    run-to-run bit-identity (the sum order does not depend on which CTA finishes last)."""
+    for the SMs, so the tensor-core GEMMs cut K into units of work that store fp32 parts, and a second
+    launch sums the parts in K order and runs the fused epilogue (bias, residual, rotary embedding;
+    the LoRA k-block rides with the first part).  Checked against the oracle and the CUDA-core GEMM,
+    and for run-to-run bit-identity."""
     spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
                      **{**TINY, "d_model": 512, "n_heads": 4, "d_ffn": 1024, "vocab": 517, "S": 40,
                         "E": 1, "max_seq": 40, "q": q, "n_layers": 2, "lora_rank": 8})
