@@ -80,7 +80,8 @@ enum { ZO_W_NATIVE = 0, ZO_W_INT8 = 1, ZO_W_NF4 = 2 };
  * CUDA-core validation kernels instead of the tensor-core ones (cross-checking only). */
 enum { ZO_FLAG_SIMT_GEMM = 1,
        /* ZO_FLAG_GEMM_PAIR: tensor-core GEMMs run CTA pairs (tcgen05 cta_group::2) on 256-row
-        * tiles instead of the default one CTA per 128-row tile (A/B switch; bit-identical results). */
+        * tiles instead of the default one CTA per 128-row tile (A/B switch; bit-identical results
+        * when the low-rank term runs in the epilogue in both and no launch is split along K). */
        ZO_FLAG_GEMM_PAIR = 2,
        /* ZO_FLAG_LORA_EPILOGUE: the MP-LoRA term is always added on CUDA cores in the GEMM epilogue
         * from fp32 U and fp32 (B + k eps z), never as the extra tensor-core k-block (which rounds
@@ -214,8 +215,13 @@ ZO_API zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g);
  * ZO_ARCH_LINEAR: one value per token row (mean over k_out).  Synchronises the stream. */
 ZO_API zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_rows);
 
-/* How a step is cut into forward passes (the paper's ablation of its two parallelisations; the
- * results of a step do not depend on it, only its cost does):
+/* How a step is cut into forward passes (the paper's ablation of its two parallelisations; only the
+ * cost of a step depends on it.  Results are bit-identical across schedules as long as no GEMM of the
+ * pass is small enough to be split along K, i.e. has fewer than half as many 128x256 tiles as the
+ * device has SMs; a split launch sums its K ranges in a fixed order that depends on the number of
+ * ranges, so there the schedules agree to fp32 summation order.  Every pass of one step has the same
+ * shape, so the + and - losses of a query always see the same summation order.  flags bits 16..20 = 1
+ * switch the split off):
  *   ZO_SCHEDULE_FULL        one pass over all 2q replicas (outer and inner loop in parallel; default)
  *   ZO_SCHEDULE_OUTER_ONLY  two passes of q replicas: every +eps path, then every -eps path
  *   ZO_SCHEDULE_INNER_ONLY  q passes of 2 replicas: the +/- pair of one query at a time

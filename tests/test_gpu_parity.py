@@ -120,6 +120,24 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
     assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
 
 
+@pytest.mark.parametrize("arch,bf16,d,heads", [(ARCH_OPT, True, 768, 12), (ARCH_OPT, False, 384, 6),
+                                               (ARCH_LLAMA, False, 384, 3), (ARCH_LLAMA, True, 1536, 12),
+                                               (ARCH_LLAMA, True, 5120, 40)])
+def test_decoder_wide_rows_block_norm(arch, bf16, d, heads):
+    """Rows wider than one warp's 64 vectors: the one-block-per-row norm (LayerNorm with bias and
+    RMSNorm, both precisions, two and three vectors per thread) instead of the warp-per-row kernel."""
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=bf16,
+                     **{**TINY, "d_model": d, "n_heads": heads, "d_ffn": 256, "vocab": 211, "S": 24,
+                        "E": 2, "max_seq": 24, "q": 2, "n_layers": 1 if d > 2048 else 2, "lora_rank": 4})
+    if not bf16:
+        _check_fp32(spec, seed=19, b_std=0.05)
+        return
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 19)
+    got = run_gpu(spec, p, 19)
+    assert np.allclose(got["losses"], ref["losses"], rtol=2e-2, atol=0), (got["losses"], ref["losses"])
+
+
 @pytest.mark.parametrize("arch,q", [(ARCH_LLAMA, 1), (ARCH_OPT, 2)])
 def test_decoder_bf16_small_batch_split_k(arch, q):
     """One short sequence (a single 128-row tile per replica) with k_in = 512 and 1024: too few tiles
