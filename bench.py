@@ -27,10 +27,10 @@ from workloads.spec import ARCH_LINEAR, ARCH_OPT  # noqa: E402
 METRIC, UNIT = "perturbed_fwd_tokens_per_s", "tokens/s"
 
 # DRAM bytes (read + write) of one gate|up GEMM launch of gemm_tc_kernel<false>, from the ncu capture
-# summarised in profiles/kernels_llama7b_q1_2layers.md: 962.1 MB at 8192 token rows.  Traffic
+# summarised in profiles/kernels_llama7b_q1_2layers.md: 959.1 MB at 8192 token rows.  Traffic
 # grows in proportion to the rows (activations, outputs and one weight-panel read per 2048 rows), so
 # the full launch is scaled by rows.  Set to None whenever that kernel changes after the capture.
-GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 962.1e6 / 8192}
+GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 959.1e6 / 8192}
 
 
 def _peaks():

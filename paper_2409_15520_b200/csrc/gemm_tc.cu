@@ -988,7 +988,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   // of work cover the SMs, at least four k-blocks per unit.
   const int num_kb = (G.K + tc::BK - 1) / tc::BK;
   const int unit_cap = n_sms < G.split_units ? n_sms : G.split_units;
-  if (G.split_ws && tiles * 2 <= unit_cap && num_kb >= 8) {
+  if (G.split_ws && tiles * 3 <= unit_cap && num_kb >= 8) {
     int ks = (int)(unit_cap / tiles);
     if (ks > num_kb / 4) ks = num_kb / 4;
     if (G.split_cap > 0 && ks > G.split_cap) ks = G.split_cap;
