@@ -217,8 +217,8 @@ ZO_API zo_status zo_row_losses(zo_ctx* ctx, float* host_rows, int32_t* host_n_ro
 
 /* How a step is cut into forward passes (the paper's ablation of its two parallelisations; only the
  * cost of a step depends on it.  Results are bit-identical across schedules as long as no GEMM of the
- * pass is small enough to be split along K, i.e. has at most a third as many 128x256 tiles as the
- * device has SMs; a split launch sums its K ranges in a fixed order that depends on the number of
+ * pass is small enough to be split along K, i.e. has at most 256 rows and at most a third as many
+ * 128x256 tiles as the device has SMs; a split launch sums its K ranges in a fixed order that depends on the number of
  * ranges, so there the schedules agree to fp32 summation order.  Every pass of one step has the same
  * shape, so the + and - losses of a query always see the same summation order.  flags bits 16..20 = 1
  * switch the split off):

@@ -18,8 +18,8 @@
 //     expects, one tile ahead.  Keeping B and k eps z in separate K ranges keeps the
 //     perturbation's resolution in bf16 whatever the magnitude of B.  Otherwise the term is
 //     added on CUDA cores in the epilogue from fp32 U and fp32 (B + k eps z).
-//   * PAIR variant (opt-in; measured slower under the 1 kW power cap than one CTA per tile, see
-//     the design notes): two CTAs of a cluster work on one 256 x 256 tile with
+//   * PAIR variant (opt-in; measured slower under the 1 kW power cap than one CTA per tile: it keeps
+//     the tensor pipe busier per clock, and the cap then lowers the clock by more): two CTAs of a cluster work on one 256 x 256 tile with
 //     tcgen05.mma.cta_group::2 - each CTA stages its own 128 rows of A and its 128-row half of
 //     the weight tile, so the shared-memory traffic per SM drops by a third; 6 stages.  The
 //     leader CTA issues the MMAs and releases stages/accumulators in both CTAs with multicast
@@ -65,6 +65,7 @@ struct Ctrl {
 };
 constexpr uint32_t SLAB_BYTES = BN * BK * 2;     // generated B operand of the LoRA k-block (aliases the fp32 staging)
 constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + SLAB_BYTES + sizeof(Ctrl);  // both variants: 192 KiB of stages
+constexpr size_t SMEM_BYTES_SUM = 1024 + SLAB_BYTES + sizeof(Ctrl);          // summing launch of split K: no ring
 
 struct Params {
   int M, N, K;              // N: accumulator columns (swiglu: d_ffn, the number of OUTPUT columns)
@@ -307,8 +308,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int GROUP_M = PAIR ? (P.group_m + 1) / 2 : P.group_m;   // row tiles of a raster group
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  float* lbuf = (float*)(smem + STAGES * STAGE_BYTES);
-  Ctrl* ctrl = (Ctrl*)(smem + Cfg<PAIR>::STAGES * STAGE_BYTES + SLAB_BYTES);
+  // the summing launch of split K stages nothing: its shared memory starts at the LoRA staging area
+  float* lbuf = (float*)(smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES));
+  Ctrl* ctrl = (Ctrl*)(smem + (SPLIT == 2 ? 0 : Cfg<PAIR>::STAGES * STAGE_BYTES) + SLAB_BYTES);
   const uint32_t tiles_base = smem_u32(smem);
   const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -485,7 +487,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int half = (warp - 2) >> 2;              // which of the quarter's two warps: even or odd chunks
     const bool out_vec_ok = ((uintptr_t)P.out & 15) == 0 && (P.ldo % (P.out_f32 ? 4 : 8)) == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
-    uint8_t* slab = smem + STAGES * STAGE_BYTES;
+    uint8_t* slab = smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES);
     // Slab mode: build the B operand [s B ; s k eps z] of a tile's LoRA k-block: 256 rows (output
     // columns) x 64 K-elements, K-major with the 128-byte swizzle.  Rank index k sits at K = k
     // (B part) and K = khalf + k (perturbation part); all other K positions stay zero.
@@ -984,11 +986,12 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   }
   const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
   const long long tiles = (long long)tiles_m * tiles_n;
-  // Few tiles and a long K (small batches: the GEMM is a stream of weights): cut K so that the units
-  // of work cover the SMs, at least four k-blocks per unit.
+  // At most 256 rows, few tiles and a long K (the small-batch regime: the GEMM is a stream of weights):
+  // cut K so that the units of work cover the SMs, at least four k-blocks per unit.  Larger launches
+  // are never split, so their sums do not depend on the batch shape.
   const int num_kb = (G.K + tc::BK - 1) / tc::BK;
   const int unit_cap = n_sms < G.split_units ? n_sms : G.split_units;
-  if (G.split_ws && tiles * 3 <= unit_cap && num_kb >= 8) {
+  if (G.split_ws && tiles_m <= 2 && tiles * 3 <= unit_cap && num_kb >= 8) {
     int ks = (int)(unit_cap / tiles);
     if (ks > num_kb / 4) ks = num_kb / 4;
     if (G.split_cap > 0 && ks > G.split_cap) ks = G.split_cap;
@@ -999,7 +1002,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   if (P.ksplit > 1) {
     tc::gemm_tc_kernel<false, 1><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
     const long long fin = tiles * tc::FIN_GROUPS;
-    tc::gemm_tc_kernel<false, 2><<<(int)(fin < n_sms ? fin : n_sms), tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+    tc::gemm_tc_kernel<false, 2><<<(int)(fin < n_sms ? fin : n_sms), tc::THREADS, tc::SMEM_BYTES_SUM, st>>>(tmA, tmB, tmU, P);
     if (G.extra_launches) ++*G.extra_launches;
   } else
     tc::gemm_tc_kernel<false, 0><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);

@@ -249,6 +249,7 @@ zo_status run_lora_down(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, cons
     if (c && c->plan.split_ws) {
       G.split_ws = c->at<float>(c->plan.split_ws); G.split_units = SPLIT_UNITS; G.extra_launches = launches;
     }
+    G.split_cap = (int)((flags >> 16) & 0x1F);
     ProfScope ps(c, PC_LORA_DOWN, 2.0 * rows * (double)J * K);
     const int e = launch_gemm_tc(st, G, status, n_sms);
     if (e) {
