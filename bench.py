@@ -126,7 +126,7 @@ def algorithmic_flops_per_step(spec):
 
 def oracle_sample(spec, seed=1234):
     """Bounded CPU sample of the same workload: the oracle's zo_step with q = 1 (one +/- pair) on up to
-    four sequences of the batch through a 2-block copy of the model.  Returns (seconds, token-forwards done,
+    eight sequences of the batch through a 2-block copy of the model.  Returns (seconds, token-forwards done,
     scale to full depth)."""
     import oracle
     if spec.arch == ARCH_LINEAR:
@@ -136,7 +136,7 @@ def oracle_sample(spec, seed=1234):
         oracle.zo_step(small, p, p["X"], p["target"], 1, 1, spec.eps, spec.lr)
         return time.perf_counter() - t0, 2 * small.E * small.S, 1.0, "q=1 on the full token block"
     L = min(2, spec.n_layers)
-    Es = min(4, spec.E)                      # sized for 10-30 s of CPU work at the 7B shape
+    Es = min(8, spec.E)                      # sized for 10-30 s of CPU work at the 7B shape
     small = spec.with_(n_layers=L, E=Es, q=1)
     p = make_decoder_globals(small, seed)
     p["layers"] = [make_decoder_layer(small, seed, l, 0.01) for l in range(L)]

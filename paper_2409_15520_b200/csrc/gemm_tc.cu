@@ -84,6 +84,7 @@ struct Params {
   int pack_r;
   LoraDesc L;
   uint32_t* status;
+  int n_half;               // 1: at most 128 output columns in all: one weight box per stage, MMAs of N = 128
   int ksplit;               // > 1: the K range of every tile is cut into ksplit units of work
   float4* part;             // ksplit > 1: fp32 partial accumulators, [unit][64 column quads][128 rows]
 };
@@ -238,6 +239,9 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                            ((uint32_t)(BM >> 4) << 24);
 // The pair instruction spans both CTAs: M = 256.
+// The same with N = 128 (launches with at most 128 output columns, e.g. the LoRA down-projection).
+constexpr uint32_t IDESC_N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) |
+                                ((uint32_t)(BM >> 4) << 24);
 constexpr uint32_t IDESC_PAIR = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                 ((uint32_t)((2 * BM) >> 4) << 24);
 
@@ -394,10 +398,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             tma_load_2d_pair(sa, &tmA, kb * BK, m0, bar);
             tma_load_2d_pair(sa + A_BYTES, &tmB, kb * BK, rank == 0 ? brow0 : brow1, bar);
           } else {
-            mbar_expect_tx(bar, Cfg<PAIR>::TX_BYTES);
+            mbar_expect_tx(bar, P.n_half ? A_BYTES + BOX_BYTES : Cfg<PAIR>::TX_BYTES);
             tma_load_2d(sa, &tmA, kb * BK, m0, bar);
             tma_load_2d(sa + A_BYTES, &tmB, kb * BK, brow0, bar);
-            tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
+            if (!P.n_half) tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
           }
         }
         const int lslot = (PAIR || ks != 0) ? -1 : tile_slot(P, brow0);   // the LoRA block rides with the first K range
@@ -443,7 +447,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               tc_mma_pair(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC_PAIR,
                           (uint32_t)(((kb - kb0) | k) != 0));
             else
-              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC,
+              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), P.n_half ? IDESC_N128 : IDESC,
                      (uint32_t)(((kb - kb0) | k) != 0));
           }
           // frees the stage (in both CTAs of a pair) once these MMAs retire
@@ -959,6 +963,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   }
   P.status = status;
   P.ksplit = 1; P.part = nullptr;
+  P.n_half = (!G.cta_pair && !G.swiglu && !P.slab && P.N <= 128) ? 1 : 0;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
   if (G.cta_pair && P.M > tc::BM) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
