@@ -305,16 +305,19 @@ template <bool PAIR, int SPLIT>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmU, const Params P) {
-  // ring depth: one stage is given up when the LoRA term needs two generated k-blocks (rank > 32)
-  const int STAGES = PAIR ? Cfg<PAIR>::STAGES : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0);
-  constexpr uint32_t STAGE_BYTES = Cfg<PAIR>::STAGE_BYTES;
+  // ring depth: one stage is given up when the LoRA term needs two generated k-blocks (rank > 32);
+  // narrow-output launches stage one weight box, so the same 192 KiB hold six stages of 32 KiB
+  const bool narrow = !PAIR && P.n_half;
+  const int STAGES = PAIR ? Cfg<PAIR>::STAGES
+                          : (narrow ? 6 : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0));
+  const uint32_t STAGE_BYTES = narrow ? A_BYTES + BOX_BYTES : Cfg<PAIR>::STAGE_BYTES;
   constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
   const int GROUP_M = PAIR ? (P.group_m + 1) / 2 : P.group_m;   // row tiles of a raster group
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   // the summing launch of split K stages nothing: its shared memory starts at the LoRA staging area
   float* lbuf = (float*)(smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES));
-  Ctrl* ctrl = (Ctrl*)(smem + (SPLIT == 2 ? 0 : Cfg<PAIR>::STAGES * STAGE_BYTES) + SLAB_BYTES);
+  Ctrl* ctrl = (Ctrl*)(smem + (SPLIT == 2 ? 0 : Cfg<PAIR>::STAGES * Cfg<PAIR>::STAGE_BYTES) + SLAB_BYTES);
   const uint32_t tiles_base = smem_u32(smem);
   const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
