@@ -326,6 +326,9 @@ def main():
                     help="how the step is cut into forward passes (the paper's ablation)")
     ap.add_argument("--weights", default=None, choices=["int8", "nf4"],
                     help="weight-only quantised storage of the frozen linear weights (decoded once per pass)")
+    ap.add_argument("--shard-queries", action="store_true",
+                    help="N > 1: spread the q queries of ONE step over the ranks (all-reduce of the 2q losses, "
+                         "identical update everywhere; strong scaling) instead of N independent replicas")
     ap.add_argument("--E", type=int, default=0, help="override the number of sequences")
     ap.add_argument("--S", type=int, default=0, help="override the sequence length")
     args = ap.parse_args()
@@ -368,6 +371,20 @@ def main():
     est.set_schedule(args.schedule)
     E, S, q, eps, lr = spec.E, spec.S, spec.q, spec.eps, spec.lr
     tokens_per_step = 2 * q * E * S
+    sharded = args.shard_queries
+    jobs = 1 if sharded else world            # independent steps in flight across the ranks
+
+    def one_step(seed, host=False):
+        if not sharded:
+            return (est.step_host if host else est.step)(prob, E, S, seed, q, eps, lr)
+        begin, count = zo.query_shard(q, world, rank)
+        est.set_query_shard(begin, count)
+        (est.step_host if host else est.step)(prob, E, S, seed, q, eps, 0.0)
+        zo.exchange_losses(est.loss_buffer(), q)
+        est.apply_update(prob, seed, q, eps, lr)
+
+    if sharded and world > q:
+        raise SystemExit("--shard-queries needs at least one query per rank")
 
     def barrier():
         if world > 1:
@@ -375,7 +392,7 @@ def main():
         torch.cuda.synchronize()
 
     for i in range(max(args.warmup, 3)):
-        est.step(prob, E, S, 100 + i, q, eps, lr)
+        one_step(100 + i)
     est.losses()
     sampler = ClockSampler(local)
     est.profile_enable(True)
@@ -385,7 +402,7 @@ def main():
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev0.record()
     for i in range(args.steps):
-        est.step(prob, E, S, 1000 + i, q, eps, lr)
+        one_step(1000 + i)
     ev1.record()
     barrier()
     clocks = sampler.stop()
@@ -401,7 +418,7 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(args.steps):
-        est.step_host(prob, E, S, 2000 + i, q, eps, lr)
+        one_step(2000 + i, host=True)
         est.losses()
     e1.record()
     barrier()
@@ -424,9 +441,9 @@ def main():
     peak = peaks["tflops_sustained"] if inside_long_step else peaks["tflops"]
     total_prof = sum(v[0] for v in prof.values())
     line = {
-        "metric": METRIC, "value": whole_job_value(world, tokens_per_step, args.steps, ms), "unit": UNIT,
+        "metric": METRIC, "value": whole_job_value(jobs, tokens_per_step, args.steps, ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if sharded else "weak", "vs_baseline": None,
         "dtype": "bf16" if spec.bf16 else "f32", "data": "synthetic",
         "config": {"workload": args.workload, "arch": {0: "linear", 1: "opt", 2: "llama"}[spec.arch],
                    "n_layers": spec.n_layers, "d_model": spec.d_model, "d_ffn": spec.d_ffn, "vocab": spec.vocab,
@@ -434,11 +451,12 @@ def main():
                    "token_rows_per_step": tokens_per_step, "eps": eps, "lr": lr,
                    "l2": "inputs larger than L2 (weights and activations of several GB stream every step)",
                    "schedule": args.schedule, "weights": args.weights or "bf16",
-                   "parallelism": "replicas only" if world > 1 else "1 gpu"},
-        "zo_steps_per_s": world * args.steps / (ms * 1e-3),
+                   "parallelism": (f"queries of one step sharded over {world} gpu(s), all-reduce of 2q losses" if sharded
+                                   else "replicas only" if world > 1 else "1 gpu")},
+        "zo_steps_per_s": jobs * args.steps / (ms * 1e-3),
         "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,
         "clocks": clocks,
-        "e2e": {"value": whole_job_value(world, tokens_per_step, args.steps, ms_e2e), "unit": UNIT,
+        "e2e": {"value": whole_job_value(jobs, tokens_per_step, args.steps, ms_e2e), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
         "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tflops, "peak": peak,

@@ -232,6 +232,42 @@ enum { ZO_SCHEDULE_FULL = 0, ZO_SCHEDULE_OUTER_ONLY = 1, ZO_SCHEDULE_INNER_ONLY 
        ZO_SCHEDULE_SEQUENTIAL = 3 };
 ZO_API zo_status zo_set_schedule(zo_ctx* ctx, int32_t schedule);
 
+/* Replica sharding over several devices.  The 2q replicas of a step are independent forward passes
+ * (Algorithm 1: every query i has its own seed s_i and its own pair of losses), so a step can be
+ * spread over devices that each hold the frozen weights and a copy of the trainable B tensors:
+ * device k runs the queries [q_begin, q_begin + q_count) of the step, the devices exchange the 2q
+ * loss scalars, and every device regenerates all z_i and applies the same update to its copy of B.
+ * No parameter or activation ever crosses between devices.
+ *
+ *   zo_set_query_shard(ctx, q_begin, q_count)
+ *       From now on zo_step / zo_step_host / zo_step_varlen run only the replicas 2*q_begin ..
+ *       2*(q_begin + q_count) - 1 of the q-query step they are given (same seed, same replica
+ *       numbering, so the perturbations are those of the whole step), write their losses at those
+ *       positions of the loss array, zero the other positions and stop there: no g, no update
+ *       (lr is ignored).  q_begin + q_count must not exceed the step's q (ZO_ERR_INVALID_ARG
+ *       from the step otherwise).  q_count = 0 (with q_begin = 0) switches sharding off.  The
+ *       schedule set by zo_set_schedule applies inside the shard.
+ *   zo_loss_buffer(ctx, &dev_losses, &capacity)
+ *       Device address of the step's float64 loss array (replica order, `capacity` = 2*max_q
+ *       entries, inside the caller's workspace).  After a sharded step it holds this shard's
+ *       losses and zeros elsewhere, so a sum over devices (an all-reduce of 2q doubles, exact
+ *       since every entry has one non-zero contributor) or an all-gather of the shards completes
+ *       it.  The exchange itself is the caller's: enqueue it on the context's stream, or order it
+ *       with the stream by events.
+ *   zo_apply_update(ctx, lora, seed, q, eps, lr)
+ *       g_i = (l_{2i} - l_{2i+1}) / (2 eps) from the loss array as it then stands, and
+ *       B <- B - lr (1/q) sum_i g_i z_i on this device's B.  Asynchronous on the context's stream.
+ *       A non-finite loss from any device leaves B untouched on every device (all see the same
+ *       array); zo_losses afterwards returns all 2q losses and g and the deferred status.
+ *       Also valid after an unsharded step with lr = 0 (apply the step later).
+ * A device-side fault on ONE device (ZO_ERR_TIMEOUT, bad token or label) skips that device's update
+ * only: check zo_losses on every device before the next step.  zo_row_losses after a sharded step
+ * holds this shard's rows only. */
+ZO_API zo_status zo_set_query_shard(zo_ctx* ctx, int32_t q_begin, int32_t q_count);
+ZO_API zo_status zo_loss_buffer(zo_ctx* ctx, double** dev_losses, int32_t* host_capacity);
+ZO_API zo_status zo_apply_update(zo_ctx* ctx, const zo_lora* lora, uint64_t seed, int32_t q,
+                                 float eps, float lr);
+
 /* Number of kernels the last zo_step enqueued. */
 ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 

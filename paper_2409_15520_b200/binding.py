@@ -78,6 +78,10 @@ zo_losses = _sig("zo_losses", C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p])
 zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTER(C.c_int32)])
 zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
 zo_set_schedule = _sig("zo_set_schedule", C.c_int, [C.c_void_p, C.c_int32])
+zo_set_query_shard = _sig("zo_set_query_shard", C.c_int, [C.c_void_p, C.c_int32, C.c_int32])
+zo_loss_buffer = _sig("zo_loss_buffer", C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32)])
+zo_apply_update = _sig("zo_apply_update", C.c_int, [C.c_void_p, C.POINTER(ZoLora), C.c_uint64, C.c_int32,
+                                                    C.c_float, C.c_float])
 SCHEDULES = {"full": 0, "outer_only": 1, "inner_only": 2, "sequential": 3}
 zo_free = _sig("zo_free", None, [C.c_void_p])
 zo_profile_enable = _sig("zo_profile_enable", C.c_int, [C.c_void_p, C.c_int32])
@@ -257,6 +261,22 @@ class Estimator:
 
     def set_schedule(self, name):
         self._check(zo_set_schedule(self._h, SCHEDULES[name]))
+
+    def set_query_shard(self, q_begin, q_count):
+        """Later steps run only the queries [q_begin, q_begin + q_count) and stop at their losses
+        (q_count = 0: whole steps again)."""
+        self._check(zo_set_query_shard(self._h, q_begin, q_count))
+
+    def loss_buffer(self):
+        """The step's float64 loss array [2 * max_q] as a tensor aliasing the workspace."""
+        ptr, cap = C.c_void_p(), C.c_int32()
+        self._check(zo_loss_buffer(self._h, C.byref(ptr), C.byref(cap)))
+        off = ptr.value - self.workspace.data_ptr()
+        assert off % 8 == 0 and 0 <= off and off + 8 * cap.value <= self.workspace.numel()
+        return self.workspace[off:off + 8 * cap.value].view(torch.float64)
+
+    def apply_update(self, prob: DeviceProblem, seed, q, eps, lr):
+        self._check(zo_apply_update(self._h, C.byref(prob.lora), seed, q, eps, lr))
 
     def profile_enable(self, on=True):
         self._check(zo_profile_enable(self._h, int(on)))

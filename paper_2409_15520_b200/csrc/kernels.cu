@@ -947,6 +947,20 @@ __global__ void zo_update_kernel(UpdateDesc D, const double* __restrict__ losses
     for (int j = 0; j < left; ++j) Bp[j] -= sc * a[j];
   }
 }
+// After the losses of other devices' queries have been written into the fp64 array: the fp32 copy
+// that zo_losses reads, and the finiteness check the local reduction did for its own entries.
+__global__ void losses_refresh_kernel(const double* __restrict__ losses_d, float* __restrict__ losses,
+                                      int n, uint32_t* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float l = (float)losses_d[i];
+  losses[i] = l;
+  if (!isfinite(l)) atomicOr(status, ST_NONFINITE);
+}
+void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n, uint32_t* status) {
+  losses_refresh_kernel<<<(n + 63) / 64, 64, 0, st>>>(losses_d, losses, n, status);
+}
+
 void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g) {
   const long long blks = (D.elems_per_slot + 3) / 4;

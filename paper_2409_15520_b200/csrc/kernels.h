@@ -138,6 +138,7 @@ struct UpdateDesc {
 // or lr == 0).  With write_g, block 0 also stores g[0..q).
 void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g);
+void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n, uint32_t* status);
 void launch_perturbation(cudaStream_t st, uint64_t seed, uint32_t tensor, uint32_t query,
                          long long n, uint32_t* u32, float* z);
 

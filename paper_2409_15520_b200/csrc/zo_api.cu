@@ -170,6 +170,7 @@ struct zo_ctx {
   int launches;
   int stepped, last_q, last_E, last_S;
   int schedule;
+  int shard_begin, shard_count;    // queries this context computes in a step (count 0 = all of them)
   char err[256];
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -285,6 +286,15 @@ inline int make_passes(int schedule, int q, Pass* out) {   // out holds up to 2q
   return np;
 }
 
+// Passes of a step on this context: with a query shard set, only the replicas of the queries
+// [shard_begin, shard_begin + shard_count) are run, at their positions in the whole step.
+inline int step_passes(const zo_ctx* c, int q, Pass* out) {
+  if (c->shard_count == 0) return make_passes(c->schedule, q, out);
+  const int np = make_passes(c->schedule, c->shard_count, out);
+  for (int i = 0; i < np; ++i) out[i].base += 2 * c->shard_begin;
+  return np;
+}
+
 // Can the MP-LoRA term ride in the tensor-core GEMM's epilogue?
 inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
   return bf && !(flags & ZO_FLAG_SIMT_GEMM) && Tp % 128 == 0 && width % 32 == 0;
@@ -294,6 +304,41 @@ inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
 inline bool slab_lora_ok(int bf, uint32_t flags, int Tp, int width, int r) {
   return fused_lora_ok(bf, flags, Tp, width) && !(flags & (ZO_FLAG_GEMM_PAIR | ZO_FLAG_LORA_EPILOGUE)) &&
          width % 256 == 0 && r <= 64;
+}
+
+// Projected gradients g_i from the step's 2q fp64 losses and the ZO-SGD update of every B tensor
+// (Algorithm 1, last line of the step).
+void enqueue_update(zo_ctx* c, const zo_lora* lora, uint64_t seed, int q, float eps, float lr) {
+  const zo_config& cf = c->cfg;
+  cudaStream_t st = c->st;
+  const uint32_t* status = c->at<uint32_t>(c->plan.status);
+  const double* losses_d = c->at<double>(c->plan.losses_d);
+  float* g = c->at<float>(c->plan.g);
+  const int r = cf.lora_rank;
+  if (cf.arch == ZO_ARCH_LINEAR) {
+    UpdateDesc D{};
+    D.B[0] = lora->B[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
+    D.elems_per_slot = (long long)r * cf.d_out;
+    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, lr, seed, status, 1));
+    return;
+  }
+  const int nt = c->nt, J = nt * r;
+  if (J == 0) {
+    UpdateDesc D{};
+    D.count = 0; D.n_slots = 0; D.elems_per_slot = 0;
+    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, 0.f, seed, status, 1));
+  }
+  for (int l0 = 0; l0 < cf.n_layers && J; l0 += UpdateDesc::MAX_T) {
+    UpdateDesc D{};
+    D.count = cf.n_layers - l0 < UpdateDesc::MAX_T ? cf.n_layers - l0 : UpdateDesc::MAX_T;
+    D.n_slots = nt;
+    D.elems_per_slot = (long long)r * cf.d_model;
+    for (int i = 0; i < D.count; ++i) {
+      D.B[i] = lora->B[l0 + i];
+      D.tensor_base[i] = (uint32_t)((l0 + i) * nt);
+    }
+    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, lr, seed, status, l0 == 0));
+  }
 }
 
 zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* X,
@@ -311,7 +356,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   float* losses = c->at<float>(c->plan.losses);
   double* losses_d = c->at<double>(c->plan.losses_d);
   Pass passes[64];
-  const int n_pass = make_passes(c->schedule, q, passes);
+  const int n_pass = step_passes(c, q, passes);
   for (int pi = 0; pi < n_pass; ++pi) {
   const Pass ps = passes[pi];
   const int n = ps.count;
@@ -336,10 +381,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss_pass));
   PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, nullptr, n, T, ps.base, ps.stride, rowloss, losses, losses_d, status));
   }
-  UpdateDesc D{};
-  D.B[0] = lora->B[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
-  D.elems_per_slot = (long long)r * ko;
-  PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, c->at<float>(c->plan.g), q, eps, lr, seed, status, 1));
+  if (c->shard_count == 0) enqueue_update(c, lora, seed, q, eps, lr);
   return ZO_OK;
 }
 
@@ -386,7 +428,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   PROF(PC_MISC, 0.0, launch_label_scan(st, labels, sl, P, n_classes, lab_idx, lab_val, lab_cnt, status));
 
   Pass passes[64];
-  const int n_pass = make_passes(c->schedule, q, passes);
+  const int n_pass = step_passes(c, q, passes);
   for (int pi = 0; pi < n_pass; ++pi) {
   const Pass ps = passes[pi];
   const int n = ps.count, M = n * Tp;          // replicas and token rows of this forward pass
@@ -500,24 +542,8 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, lab_val, n, EP, ps.base, ps.stride, rowloss, losses, losses_d, status));
   }  // passes
 
-  // projected gradients and ZO-SGD update of every B tensor
-  float* g = c->at<float>(c->plan.g);
-  if (J == 0) {
-    UpdateDesc D{};
-    D.count = 0; D.n_slots = 0; D.elems_per_slot = 0;
-    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, 0.f, seed, status, 1));
-  }
-  for (int l0 = 0; l0 < cf.n_layers && J; l0 += UpdateDesc::MAX_T) {
-    UpdateDesc D{};
-    D.count = cf.n_layers - l0 < UpdateDesc::MAX_T ? cf.n_layers - l0 : UpdateDesc::MAX_T;
-    D.n_slots = nt;
-    D.elems_per_slot = (long long)r * d;
-    for (int i = 0; i < D.count; ++i) {
-      D.B[i] = lora->B[l0 + i];
-      D.tensor_base[i] = (uint32_t)((l0 + i) * nt);
-    }
-    PROF(PC_UPDATE, 0.0, launch_zo_update(st, D, losses_d, g, q, eps, lr, seed, status, l0 == 0));
-  }
+  // projected gradients and ZO-SGD update of every B tensor (a sharded step stops at its losses)
+  if (c->shard_count == 0) enqueue_update(c, lora, seed, q, eps, lr);
 #undef GEMM
   return ZO_OK;
 }
@@ -554,12 +580,24 @@ zo_status check_step_args(zo_ctx* c, const zo_weights* w, const zo_lora* lora, c
   return ZO_OK;
 }
 
+// Start of every step: launch counter and device status word cleared; a sharded step also zeroes
+// the fp64 loss array so that the entries of the other shards' queries read 0 until the exchange.
+zo_status begin_step(zo_ctx* c, int q) {
+  c->launches = 0;
+  if (c->shard_count && c->shard_begin + c->shard_count > q)
+    return fail(c, ZO_ERR_INVALID_ARG, "query shard reaches past q");
+  cudaError_t e = cudaMemsetAsync(c->at<uint32_t>(c->plan.status), 0, 4, c->st);
+  if (e == cudaSuccess && c->shard_count)
+    e = cudaMemsetAsync(c->at<double>(c->plan.losses_d), 0, (size_t)2 * c->cfg.max_q * 8, c->st);
+  if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  return ZO_OK;
+}
+
 zo_status do_step(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* tokens,
                   const void* labels, int E, int S, uint64_t seed, int q, float eps, float lr) {
-  c->launches = 0;
-  cudaError_t e = cudaMemsetAsync(c->at<uint32_t>(c->plan.status), 0, 4, c->st);
-  if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
-  zo_status s;
+  zo_status s = begin_step(c, q);
+  if (s) return s;
+  cudaError_t e;
   if (c->cfg.arch == ZO_ARCH_LINEAR)
     s = step_linear(c, w, lora, tokens, labels, E * S, seed, q, eps, lr);
   else
@@ -655,12 +693,11 @@ zo_status zo_step_varlen(zo_ctx* ctx, const zo_weights* weights, const zo_lora* 
   if (total_tokens < E || (long long)total_tokens > (long long)E * max_len ||
       (long long)total_tokens > (long long)ctx->cfg.max_E * ctx->cfg.max_seq)
     return fail(ctx, ZO_ERR_INVALID_ARG, "total_tokens outside E .. E*max_len");
-  ctx->launches = 0;
-  cudaError_t e = cudaMemsetAsync(ctx->at<uint32_t>(ctx->plan.status), 0, 4, ctx->st);
-  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
+  s = begin_step(ctx, q);
+  if (s) return s;
   s = step_decoder(ctx, weights, lora, tokens, labels, E, max_len, seed, q, eps, lr, cu_seqlens, total_tokens);
   if (s) return s;
-  e = cudaGetLastError();
+  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
   ctx->stepped = 1; ctx->last_q = q; ctx->last_E = E; ctx->last_S = max_len;
   return ZO_OK;
@@ -735,6 +772,41 @@ zo_status zo_set_schedule(zo_ctx* ctx, int32_t schedule) {
   if (schedule < ZO_SCHEDULE_FULL || schedule > ZO_SCHEDULE_SEQUENTIAL)
     return fail(ctx, ZO_ERR_INVALID_ARG, "unknown schedule");
   ctx->schedule = schedule;
+  return ZO_OK;
+}
+
+zo_status zo_set_query_shard(zo_ctx* ctx, int32_t q_begin, int32_t q_count) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (q_begin < 0 || q_count < 0 || (q_count == 0 && q_begin != 0) || q_begin + q_count > ctx->cfg.max_q)
+    return fail(ctx, ZO_ERR_INVALID_ARG, "query shard outside 0..max_q");
+  ctx->shard_begin = q_begin;
+  ctx->shard_count = q_count;
+  return ZO_OK;
+}
+
+zo_status zo_loss_buffer(zo_ctx* ctx, double** dev_losses, int32_t* host_capacity) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (!dev_losses) return fail(ctx, ZO_ERR_INVALID_ARG, "dev_losses is NULL");
+  *dev_losses = ctx->at<double>(ctx->plan.losses_d);
+  if (host_capacity) *host_capacity = 2 * ctx->cfg.max_q;
+  return ZO_OK;
+}
+
+zo_status zo_apply_update(zo_ctx* ctx, const zo_lora* lora, uint64_t seed, int32_t q, float eps, float lr) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (!lora || !lora->B) return fail(ctx, ZO_ERR_INVALID_ARG, "lora is NULL");
+  if (!ctx->stepped) return fail(ctx, ZO_ERR_STATE, "zo_apply_update before any zo_step");
+  if (q != ctx->last_q) return fail(ctx, ZO_ERR_INVALID_ARG, "q differs from the step's");
+  if (!(eps >= 0.f) || !isfinite(eps) || !isfinite(lr)) return fail(ctx, ZO_ERR_INVALID_ARG, "eps or lr not finite");
+  const int n_b = ctx->cfg.arch == ZO_ARCH_LINEAR ? 1 : (ctx->nt ? ctx->cfg.n_layers : 0);
+  for (int l = 0; l < n_b; ++l)
+    if (!lora->B[l]) return fail(ctx, ZO_ERR_INVALID_ARG, "null LoRA tensor");
+  zo_ctx* c = ctx;
+  PROF(PC_LOSS, 0.0, launch_losses_refresh(ctx->st, ctx->at<double>(ctx->plan.losses_d), ctx->at<float>(ctx->plan.losses),
+                                           2 * q, ctx->at<uint32_t>(ctx->plan.status)));
+  enqueue_update(ctx, lora, seed, q, eps, lr);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
   return ZO_OK;
 }
 
