@@ -766,10 +766,21 @@ void launch_label_scan(cudaStream_t st, const int32_t* labels, SeqLayout sl, int
 // =========================================================================================
 // Fused log-softmax / label pick over the whole vocabulary, one block per labelled row:
 // row_loss = logsumexp(logits) - logits[label].
+// The row is read once: every thread keeps a running (max, sum of exp relative to that max) over
+// 16-byte loads, four of them in flight, and the block merges the 256 pairs at the end.  The
+// logits are streamed (read exactly once, by this kernel), so the loads bypass L1 allocation.
 // =========================================================================================
-__global__ void ce_rows_kernel(const float* __restrict__ logits, int ldl, int V,
-                               const int32_t* __restrict__ lab_val, int EP,
-                               double* __restrict__ row_loss) {
+__device__ __forceinline__ void lse_push4(float& m, float& s, const float4 v) {
+  const float mx = fmaxf(fmaxf(v.x, v.y), fmaxf(v.z, v.w));
+  if (mx > m) {                       // first chunk: m = -inf, s = 0, expf(-inf) = 0
+    s *= expf(m - mx);
+    m = mx;
+  }
+  s += (expf(v.x - m) + expf(v.y - m)) + (expf(v.z - m) + expf(v.w - m));
+}
+__global__ void __launch_bounds__(256)
+ce_rows_kernel(const float* __restrict__ logits, int ldl, int V, const int32_t* __restrict__ lab_val, int EP,
+               double* __restrict__ row_loss) {
   __shared__ float red[32];
   const int row = blockIdx.x;
   const int lab = lab_val[row % EP];
@@ -778,13 +789,39 @@ __global__ void ce_rows_kernel(const float* __restrict__ logits, int ldl, int V,
     return;
   }
   const float* p = logits + (size_t)row * ldl;
-  float m = -INFINITY;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) m = fmaxf(m, p[c]);
-  m = block_max(m, red);
-  float s = 0.f;
-  for (int c = threadIdx.x; c < V; c += blockDim.x) s += expf(p[c] - m);
-  s = block_sum(s, red);
-  if (threadIdx.x == 0) row_loss[row] = ((double)m - (double)p[lab]) + log((double)s);
+  float m = -INFINITY, s = 0.f;
+  // the vector path is taken for all rows or for none, so that a row's sum order (and with it the
+  // last bits of its loss) does not depend on where the row sits in the array
+  if ((((uintptr_t)logits) & 15) == 0 && (ldl & 3) == 0) {
+    const float4* p4 = reinterpret_cast<const float4*>(p);
+    const int n4 = V >> 2;
+    int c = threadIdx.x;
+    for (; c + 3 * 256 < n4; c += 4 * 256) {
+      const float4 a = __ldcs(p4 + c), b = __ldcs(p4 + c + 256);
+      const float4 d = __ldcs(p4 + c + 512), e = __ldcs(p4 + c + 768);
+      lse_push4(m, s, a);
+      lse_push4(m, s, b);
+      lse_push4(m, s, d);
+      lse_push4(m, s, e);
+    }
+    for (; c < n4; c += 256) lse_push4(m, s, __ldcs(p4 + c));
+    for (int t = (n4 << 2) + threadIdx.x; t < V; t += 256) {      // V % 4 leftovers
+      const float v = p[t];
+      if (v > m) { s *= expf(m - v); m = v; }
+      s += expf(v - m);
+    }
+  } else {
+    for (int t = threadIdx.x; t < V; t += 256) {
+      const float v = p[t];
+      if (v > m) { s *= expf(m - v); m = v; }
+      s += expf(v - m);
+    }
+  }
+  const float mb = block_max(m, red);
+  // a thread that saw no element has m = -inf, s = 0: expf(-inf) = 0 keeps it out (mb is finite
+  // unless the whole row is -inf or holds a NaN, which the replica mean reports as non-finite)
+  const float sb = block_sum(m == -INFINITY ? 0.f : s * expf(m - mb), red);
+  if (threadIdx.x == 0) row_loss[row] = ((double)mb - (double)p[lab]) + log((double)sb);
 }
 void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
                     int EP, int rows, double* row_loss) {

@@ -120,6 +120,23 @@ def test_decoder_bf16_tensor_core_multi_tile(arch):
     assert np.allclose(got["rows"], simt["rows"], rtol=0, atol=0.05)
 
 
+@pytest.mark.parametrize("vocab", [5000, 4100, 64])
+def test_full_vocab_loss_vector_path(vocab):
+    """Vocabularies that are a multiple of 4 take the 16-byte-load form of the log-softmax reduction:
+    5000 runs the four-loads-in-flight body once plus single chunks, 4100 the body and a one-chunk
+    tail in a few lanes only, 64 leaves most lanes of the block without any element.  fp32 mode, so
+    the 1e-4 loss tolerance applies; per-row losses are checked too."""
+    spec = ModelSpec(arch=ARCH_LLAMA, bf16=False, **{**TINY, "vocab": vocab, "q": 2})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 23)
+    got = run_gpu(spec, p, 23)
+    assert np.allclose(got["losses"], ref["losses"], rtol=1e-4, atol=0), (got["losses"], ref["losses"])
+    assert np.all(np.abs(got["g"] - ref["g"]) <= 1e-2 * np.abs(ref["g"]).max())
+    assert update_rel_err(spec, p, got["B"], ref["B"]) < 1e-3
+    seq = run_gpu(spec, p, 23, schedule="sequential")
+    assert np.array_equal(seq["losses"], got["losses"]) and np.array_equal(seq["rows"], got["rows"])
+
+
 @pytest.mark.parametrize("arch,bf16,d,heads", [(ARCH_OPT, True, 768, 12), (ARCH_OPT, False, 384, 6),
                                                (ARCH_LLAMA, False, 384, 3), (ARCH_LLAMA, True, 1536, 12),
                                                (ARCH_LLAMA, True, 5120, 40)])
