@@ -350,7 +350,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 2 * EP_WARPS : EP_WARPS);
     }
     mbar_init(smem_u32(&ctrl->drain), 1);
-    mbar_init(smem_u32(&ctrl->lfull), EP_WARPS);
+    mbar_init(smem_u32(&ctrl->lfull), PAIR ? 2 * EP_WARPS : EP_WARPS);
     ctrl->abort = 0u;
     ctrl->ep_go = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -407,15 +407,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (!P.n_half) tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
           }
         }
-        const int lslot = (PAIR || ks != 0) ? -1 : tile_slot(P, brow0);   // the LoRA block rides with the first K range
+        const int lslot = ks != 0 ? -1 : tile_slot(P, brow0);   // the LoRA block rides with the first K range
         for (int lkb = 0; ok && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued) {
           // LoRA k-blocks: only the A operand (packed U) travels through the ring
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
-          mbar_expect_tx(bar, A_BYTES);
-          tma_load_2d(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot + lkb * BK,
-                      m0, bar);
+          if (PAIR) {
+            if (rank == 0) mbar_expect_tx(bar, 2 * A_BYTES);     // each CTA brings the U rows of its half
+            tma_load_2d_pair(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot + lkb * BK, m0, bar);
+          } else {
+            mbar_expect_tx(bar, A_BYTES);
+            tma_load_2d(tiles_base + s * STAGE_BYTES, &tmU, lslot * P.kslot + lkb * BK, m0, bar);
+          }
         }
         if (!ok) break;
       }
@@ -457,7 +461,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           if (PAIR) tc_commit_pair(smem_u32(&ctrl->empty[s]));
           else tc_commit(smem_u32(&ctrl->empty[s]));
         }
-        if (!PAIR && ok) {
+        if (ok) {
           int tm, tn;
           coords(tile, tm, tn);
           if (ks == 0 && tile_slot(P, tn * ncol_tile) >= 0) {
@@ -469,9 +473,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               const uint64_t ad = smem_desc(tiles_base + s * STAGE_BYTES);
               const uint64_t bd = smem_desc(tiles_base + STAGES * STAGE_BYTES + lkb * SLAB_BYTES);
 #pragma unroll
-              for (int k = 0; k < BK / 16; ++k)
-                tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC, 1u);
-              tc_commit(smem_u32(&ctrl->empty[s]));
+              for (int k = 0; k < BK / 16; ++k) {
+                if (PAIR) tc_mma_pair(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC_PAIR, 1u);
+                else tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC, 1u);
+              }
+              if (PAIR) tc_commit_pair(smem_u32(&ctrl->empty[s]));
+              else tc_commit(smem_u32(&ctrl->empty[s]));
             }
             if (!ok) break;
             ++ltiles;
@@ -509,8 +516,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const float sz = ((repg & 1) ? -P.L.eps : P.L.eps) * P.L.scale;
       const float* Bm = P.L.B + (size_t)slot * P.L.r * P.L.width;
       const int kgroups = (P.L.r + 7) / 8;
-      for (int unit_i = et; unit_i < 64 * kgroups; unit_i += EP_THREADS) {
-        const int c4 = (unit_i & 63) * 4, k0 = (unit_i >> 6) * 8;
+      constexpr int CQ = PAIR ? 32 : 64;               // column quads of the operand rows this CTA holds
+      for (int unit_i = et; unit_i < CQ * kgroups; unit_i += EP_THREADS) {
+        const int c4l = (unit_i % CQ) * 4, k0 = (unit_i / CQ) * 8;
+        const int c4 = c4l + (PAIR ? (int)rank * 128 : 0);       // column inside the 256-column tile
         float bb[8][4], zz[8][4];
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {
@@ -526,7 +535,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const int n = c4 + j;                       // row of the operand tile = output column
+          const int n = c4l + j;                      // row of this CTA's operand tile = output column
           const uint4 vb = make_uint4(pack_bf16(bb[0][j], bb[1][j]), pack_bf16(bb[2][j], bb[3][j]),
                                       pack_bf16(bb[4][j], bb[5][j]), pack_bf16(bb[6][j], bb[7][j]));
           const uint4 vz = make_uint4(pack_bf16(zz[0][j], zz[1][j]), pack_bf16(zz[2][j], zz[3][j]),
@@ -539,14 +548,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&ctrl->lfull));
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_leader(smem_u32(&ctrl->lfull));        // the leader's MMA warp waits for both halves
+        else mbar_arrive(smem_u32(&ctrl->lfull));
+      }
     };
-    if (!PAIR && P.slab && SPLIT != 2) {
+    if (P.slab && SPLIT != 2) {
       for (int i = et; i < (int)(SLAB_BYTES / 16) * (P.kslot / BK); i += EP_THREADS)
         reinterpret_cast<uint4*>(slab)[i] = make_uint4(0, 0, 0, 0);
       ep_bar();
     }
-    if (!PAIR && P.slab && SPLIT != 2 && t_first < t_end) gen_slab(t_first);
+    if (P.slab && SPLIT != 2 && t_first < t_end) gen_slab(t_first);
     uint32_t titer = 0;
     // iteration space: the units of this CTA; in the summing launch (tile, chunk group) pairs
     const int e_first = SPLIT == 2 ? (int)blockIdx.x : t_first;
@@ -564,7 +576,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!go) break;
         tc_fence_after();
         // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
-        if (!PAIR && P.slab && tile + t_step < t_end) gen_slab(tile + t_step);
+        if (P.slab && tile + t_step < t_end) gen_slab(tile + t_step);
       }
       int tm, tn;
       coords(tile, tm, tn);
@@ -966,30 +978,45 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   }
   P.status = status;
   P.ksplit = 1; P.part = nullptr;
-  P.n_half = (!G.cta_pair && !G.swiglu && !P.slab && P.N <= 128) ? 1 : 0;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
-  if (G.cta_pair && P.M > tc::BM) {
-    // pairs of CTAs (clusters of 2) on 256-row tiles
-    static int max_clusters = 0;                       // co-resident pairs on this device
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-    cfg.blockDim = dim3(tc::THREADS); cfg.dynamicSmemBytes = tc::SMEM_BYTES; cfg.stream = st;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    if (max_clusters == 0) {
-      cfg.gridDim = dim3(2 * (n_sms / 2));
-      int mc = 0;
-      if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true, 0>, &cfg) != cudaSuccess || mc < 1) {
-        cudaGetLastError();
-        mc = n_sms / 2;
-      }
-      max_clusters = mc < n_sms / 2 ? mc : n_sms / 2;
+  const long long tiles2 = (long long)((P.M + 2 * tc::BM - 1) / (2 * tc::BM)) * tiles_n;   // 256-row tiles
+  static int max_clusters = 0;                       // co-resident CTA pairs on this device
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(tc::THREADS); cfg.dynamicSmemBytes = tc::SMEM_BYTES; cfg.stream = st;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  if (G.cta_pair && max_clusters == 0) {
+    cfg.gridDim = dim3(2 * (n_sms / 2));
+    int mc = 0;
+    if (cudaOccupancyMaxActiveClusters(&mc, tc::gemm_tc_kernel<true, 0>, &cfg) != cudaSuccess || mc < 1) {
+      cudaGetLastError();
+      mc = n_sms / 2;
     }
-    const long long tiles = (long long)((P.M + 2 * tc::BM - 1) / (2 * tc::BM)) * tiles_n;
-    const int pairs = (int)(tiles < max_clusters ? tiles : max_clusters);
+    max_clusters = mc < n_sms / 2 ? mc : n_sms / 2;
+  }
+  // cta_pair 1: pairs wherever the kernel allows; 2: pairs for the launches they were measured faster on:
+  // no low-rank term or its one-block tensor-core form (below), at least
+  // eight waves of 256-row tiles (the coarser tiles then cost no tail), and at most 3 TFLOP in the launch.
+  // The last bound separates the two regimes measured: at the OPT-1.3B shape (launches of 0.5-2.2 TFLOP,
+  // board below its power limit) pairs keep the tensor pipe 83 % busy against 70 % and the step gains
+  // 5 %; at the Llama-2-7B shape (4-24 TFLOP per launch, board at its 1 kW limit) the pair kernel's higher
+  // duty cycle only pulls the clock down, for every kernel of the step, and the step loses 3.5 %.
+  // A low-rank term rides along in the pair kernel only as the one-block tensor-core form, whose generated
+  // operand serves both 128-row halves of a tile: a replica must then be a whole number of 256-row tiles.
+  const bool pair_slab_ok = P.slab && P.kslot == tc::BK && P.L.rows_per_replica % (2 * tc::BM) == 0;
+  // (a down-projection that also packs bf16 U always runs single-CTA)
+  const bool pair = P.M > tc::BM && !G.pack_out &&
+                    (G.cta_pair == 1 || (G.cta_pair == 2 && (!G.lora || pair_slab_ok) && P.N >= tc::BN &&
+                                         tiles2 >= 8LL * max_clusters &&
+                                         2.0 * (double)G.M * (double)G.N * (double)G.K <= 3.0e12));
+  P.n_half = (!pair && !G.swiglu && !P.slab && P.N <= 128) ? 1 : 0;
+  if (pair) {
+    // pairs of CTAs (clusters of 2) on 256-row tiles
+    const int pairs = (int)(tiles2 < max_clusters ? tiles2 : max_clusters);
     cfg.gridDim = dim3(2 * pairs);
-    P.slab = 0;
+    if (!pair_slab_ok) P.slab = 0;
     return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true, 0>, tmA, tmB, tmU, P);
   }
   const int tiles_m = (P.M + tc::BM - 1) / tc::BM;

@@ -68,7 +68,7 @@ struct GemmDesc {
   const int32_t* rope_pos;      // packed variable-length rows: position of row (m % rope_tp), else null
   int group_m;                  // 128-row tiles per raster group of the tensor-core kernel (0 = default 16)
   int prof_class;               // profiling class of this launch (0: generic tensor-core GEMM)
-  int cta_pair;                 // 1: CTA pairs (cta_group::2) on 256-row tiles instead of one CTA per 128-row tile
+  int cta_pair;                 // CTA pairs (cta_group::2) on 256-row tiles: 0 never, 1 wherever possible, 2 where measured faster (large launches without a low-rank term)
   float* split_ws;              // split-K scratch of the tensor-core kernel: split_units * 32768 floats, or null
   int split_units;
   int* extra_launches;          // incremented when the GEMM took a second launch (split K), or null

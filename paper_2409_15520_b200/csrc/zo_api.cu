@@ -217,7 +217,7 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
                2.0 * G.M * (double)G.N * G.K);
   if (tcore) {
     GemmDesc Gt = G;
-    Gt.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : 0;
+    Gt.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : ((flags & ZO_FLAG_GEMM_SINGLE) ? 0 : 2);
     Gt.group_m = (int)((flags >> 8) & 0xFF);     // diagnostic: raster group override in bits 8..15
     Gt.split_cap = (int)((flags >> 16) & 0x1F);  // diagnostic: bound on the split-K factor in bits 16..20
     if (c && c->plan.split_ws) {
@@ -300,10 +300,13 @@ inline bool fused_lora_ok(int bf, uint32_t flags, int Tp, int width) {
   return bf && !(flags & ZO_FLAG_SIMT_GEMM) && Tp % 128 == 0 && width % 32 == 0;
 }
 // ... and as extra k-blocks on the tensor cores?  (rank <= 64; every 256-column tile inside one
-// section; single-CTA kernel)
+// section.  The CTA-pair kernel shares the generated operand between the two 128-row halves of its
+// 256-row tile, so there a replica must be a whole number of such tiles, and only the one-block
+// form, rank <= 32, is built.)
 inline bool slab_lora_ok(int bf, uint32_t flags, int Tp, int width, int r) {
-  return fused_lora_ok(bf, flags, Tp, width) && !(flags & (ZO_FLAG_GEMM_PAIR | ZO_FLAG_LORA_EPILOGUE)) &&
-         width % 256 == 0 && r <= 64;
+  if (!fused_lora_ok(bf, flags, Tp, width) || (flags & ZO_FLAG_LORA_EPILOGUE) || width % 256 != 0 || r > 64)
+    return false;
+  return !(flags & ZO_FLAG_GEMM_PAIR) || (Tp % 256 == 0 && r <= 32);
 }
 
 // Projected gradients g_i from the step's 2q fp64 losses and the ZO-SGD update of every B tensor

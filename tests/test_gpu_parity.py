@@ -17,6 +17,7 @@ pytestmark = pytest.mark.gpu
 
 SIMT = 1  # ZO_FLAG_SIMT_GEMM
 PAIR = 2  # ZO_FLAG_GEMM_PAIR
+SINGLE = 8  # ZO_FLAG_GEMM_SINGLE
 LORA_EPI = 4  # ZO_FLAG_LORA_EPILOGUE
 
 
@@ -259,6 +260,52 @@ def test_mp_lora_linear_replicated_input_slab(r):
     its epilogue (fp32 from unrounded operands), so the two agree to bf16 rounding only."""
     outs = _mp_lora_linear_case(1, r, T=256, ki=328, ko=512, q=2, pair_identical=False)
     assert np.max(np.abs(outs[0] - outs[PAIR])) < 2.0 ** -6 * np.max(np.abs(outs[PAIR]))
+    if r <= 32:
+        # a replica is a whole 256-row tile here, so the pair kernel runs the one-block tensor-core form
+        # too (each CTA generates the operand rows of its half): same operands, same order, same bits
+        assert np.array_equal(outs[0], outs[PAIR])
+
+
+@pytest.mark.parametrize("arch", [ARCH_LLAMA, ARCH_OPT])
+def test_decoder_pair_kernel_with_tensor_core_lora_block(arch):
+    """256 rows per replica and d = 256: under ZO_FLAG_GEMM_PAIR the q|k|v launch runs CTA pairs with the
+    low-rank term as a generated k-block and (Llama) the rotary embedding in its epilogue.  Same bits
+    as the single-CTA kernels; the oracle within the bf16 tolerance."""
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
+                     **{**TINY, "d_model": 256, "n_heads": 2, "d_ffn": 512, "vocab": 517, "S": 128, "E": 2,
+                        "max_seq": 128, "q": 2, "lora_rank": 8, "n_layers": 3, "n_labelled": 6})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 13)
+    got = run_gpu(spec, p, 13)
+    pair = run_gpu(spec, p, 13, flags=PAIR)
+    assert np.allclose(pair["losses"], ref["losses"], rtol=2e-2, atol=0), (pair["losses"], ref["losses"])
+    assert np.array_equal(got["losses"], pair["losses"]) and np.array_equal(got["rows"], pair["rows"])
+    assert all(np.array_equal(a, b) for a, b in zip(got["B"], pair["B"]))
+
+
+def test_automatic_tile_shape_matches_both_forced_shapes():
+    """A base product large enough for the default dispatch to pick CTA pairs (16384 shared rows x 2560
+    columns = 640 tiles of 256 x 256, more than eight waves of pairs): the default, the forced single-CTA
+    and the forced pair kernels return the same bits, and the oracle's layer within bf16 rounding on a
+    sample of rows (ragged K: 72 is not a multiple of the 64-deep k-block)."""
+    import torch
+    import paper_2409_15520_b200 as zo
+    from workloads import bf16_round
+    rng = np.random.default_rng(3)
+    T, ki, ko, r, q = 16384, 72, 2560, 8, 1
+    eps, scale, seed, tid = 1e-2, 1.0, 5, 2
+    X = bf16_round(rng.standard_normal((T, ki)).astype(np.float32))
+    W = bf16_round(0.05 * rng.standard_normal((ko, ki)).astype(np.float32))
+    A = bf16_round(0.05 * rng.standard_normal((r, ki)).astype(np.float32))
+    B = (0.05 * rng.standard_normal((r, ko))).astype(np.float32)
+    dev = lambda a: torch.tensor(a, device="cuda").to(torch.bfloat16).contiguous()
+    outs = {f: zo.mp_lora_linear(dev(X), dev(W), None, dev(A), torch.tensor(B, device="cuda"), T, q, scale, seed,
+                                 tid, eps, 0, flags=f).float().cpu().numpy() for f in (0, SINGLE, PAIR)}
+    assert np.array_equal(outs[0], outs[SINGLE]) and np.array_equal(outs[0], outs[PAIR])
+    rows = np.r_[0:3, 127:130, 255:258, 4095:4098, T - 3:T]
+    Bn = np.stack([B.astype(np.float64) + k * eps * perturbation(seed, tid, 0, (r, ko)) for k in (1, -1)])
+    ref = oracle.mp_lora_linear(np.broadcast_to(X[rows], (2, len(rows), ki)).astype(np.float64), W, None, A, Bn, scale)
+    assert np.max(np.abs(outs[0][:, rows] - ref)) < 2.0 ** -7 * np.max(np.abs(ref))
 
 
 @pytest.mark.parametrize("bf16", [False, True])
