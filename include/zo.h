@@ -81,12 +81,16 @@ enum { ZO_W_NATIVE = 0, ZO_W_INT8 = 1, ZO_W_NF4 = 2 };
 enum { ZO_FLAG_SIMT_GEMM = 1,
        /* Tensor-core GEMM tile shape.  Default: CTA pairs (tcgen05 cta_group::2) on 256-row tiles for
         * launches that have at least eight waves of such tiles and at most 3 TFLOP, and either no
-        * low-rank term or its one-block tensor-core form (projections and MLP at mid-size shapes: each CTA stages half of the weight tile,
-        * which cuts the L2 traffic per flop by a third), one CTA per 128-row tile for everything else
-        * (at the largest shapes the board sits at its power limit and pairs only lower the clock).  ZO_FLAG_GEMM_PAIR: pairs wherever the kernel allows (the low-rank term
-        * then runs in the epilogue unless rank <= 32 and a replica is a multiple of 256 rows).  ZO_FLAG_GEMM_SINGLE: never pairs.  A/B switches; the two tile
-        * shapes accumulate in the same order, so results are bit-identical when the low-rank term
-        * runs in the epilogue in both and no launch is split along K. */
+        * low-rank term or its one-block tensor-core form (projections and MLP at mid-size shapes:
+        * each CTA stages half of the weight tile, which cuts the L2 traffic per flop by a third);
+        * one CTA per 128-row tile for everything else (at the largest shapes the board sits at its
+        * power limit and pairs only lower the clock).
+        * ZO_FLAG_GEMM_PAIR: pairs wherever the kernel allows (the low-rank term then runs in the
+        * epilogue unless rank <= 32 and a replica is a multiple of 256 rows).
+        * ZO_FLAG_GEMM_SINGLE: never pairs.
+        * A/B switches: the two tile shapes accumulate in the same order, so results are
+        * bit-identical when the low-rank term takes the same form in both and no launch is split
+        * along K. */
        ZO_FLAG_GEMM_PAIR = 2,
        ZO_FLAG_GEMM_SINGLE = 8,
        /* ZO_FLAG_LORA_EPILOGUE: the MP-LoRA term is always added on CUDA cores in the GEMM epilogue
