@@ -27,10 +27,10 @@ from workloads.spec import ARCH_LINEAR, ARCH_OPT  # noqa: E402
 METRIC, UNIT = "perturbed_fwd_tokens_per_s", "tokens/s"
 
 # DRAM bytes (read + write) of one gate|up GEMM launch of gemm_tc_kernel<false>, from the ncu capture
-# summarised in profiles/kernels_llama7b_q1_2layers.md: 959.1 MB at 8192 token rows.  Traffic
+# summarised in profiles/kernels_llama7b_q1_2layers.md: 960.4 MB at 8192 token rows.  Traffic
 # grows in proportion to the rows (activations, outputs and one weight-panel read per 2048 rows), so
 # the full launch is scaled by rows.  Set to None whenever that kernel changes after the capture.
-GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 959.1e6 / 8192}
+GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 960.4e6 / 8192}
 
 
 def _peaks():
@@ -470,7 +470,7 @@ def main():
                      "traffic": (GEMM_FC1_DRAM_BYTES_PER_ROW[args.workload] * tokens_per_step
                                  if GEMM_FC1_DRAM_BYTES_PER_ROW.get(args.workload)
                                  and not (args.flags or args.rank or args.targets >= 0 or args.weights) else None),
-                     "traffic_note": "gate|up launch (37 % of the step), ncu capture at 8192 rows scaled by rows"},
+                     "traffic_note": "gate|up launch (41 % of the step), ncu capture of the same single-CTA kernel at 8192 rows scaled by rows"},
         "gemm_tflops_by_class": {k: round(prof[k][1] / (prof[k][0] * 1e-3) / 1e12, 1)
                                  for k in gemm_classes if prof[k][0] > 0},
         "kernel_time_share": {k: round(v[0] / total_prof, 4) for k, v in prof.items() if v[2]},
