@@ -18,12 +18,14 @@
 //     expects, one tile ahead.  Keeping B and k eps z in separate K ranges keeps the
 //     perturbation's resolution in bf16 whatever the magnitude of B.  Otherwise the term is
 //     added on CUDA cores in the epilogue from fp32 U and fp32 (B + k eps z).
-//   * PAIR variant (opt-in; measured slower under the 1 kW power cap than one CTA per tile: it keeps
-//     the tensor pipe busier per clock, and the cap then lowers the clock by more): two CTAs of a cluster work on one 256 x 256 tile with
-//     tcgen05.mma.cta_group::2 - each CTA stages its own 128 rows of A and its 128-row half of
-//     the weight tile, so the shared-memory traffic per SM drops by a third; 6 stages.  The
-//     leader CTA issues the MMAs and releases stages/accumulators in both CTAs with multicast
-//     commits; the peer's TMA completes on the leader's barrier.
+//   * PAIR variant: two CTAs of a cluster work on one 256 x 256 tile with tcgen05.mma.cta_group::2 -
+//     each CTA stages its own 128 rows of A and its 128-row half of the weight tile, so the L2
+//     traffic per flop drops by a third; 6 stages.  The leader CTA issues the MMAs and releases
+//     stages/accumulators in both CTAs with multicast commits; the peer's TMA completes on the
+//     leader's barrier.  The one-block LoRA form rides along (each CTA generates the operand rows
+//     it stages; the peer's epilogue warps arrive on the leader's barrier).  It keeps the tensor
+//     pipe busier per clock; under the 1 kW power cap of the largest shapes that only lowers the
+//     clock, so the host takes it for mid-size launches only (launch_gemm_tc).
 //   * split K for small batches (far fewer tiles than SMs, cost = the stream of weights): a first
 //     launch computes one K range of a tile per CTA and stores fp32 parts, a second launch of the
 //     same template sums them in K order and runs the fused epilogue; no CTA waits for another.
