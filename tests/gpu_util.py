@@ -22,7 +22,8 @@ def run_gpu(spec, p, seed, q=None, eps=None, lr=None, flags=0, host=False, sched
     lr = spec.lr if lr is None else lr
     cfg = zo.make_config(spec, flags=flags, max_q=max(q, spec.q), **cfg_kw)
     est = zo.Estimator(cfg)
-    prob = zo.DeviceProblem(p, spec.bf16)
+    # a precision override runs the same (bf16-representable) numbers through the other mode
+    prob = zo.DeviceProblem(p, spec.bf16 if cfg_kw.get("precision") is None else bool(cfg_kw["precision"]))
     if schedule:
         est.set_schedule(schedule)
     (est.step_host if host else est.step)(prob, spec.E, spec.S, seed, q, eps, lr)

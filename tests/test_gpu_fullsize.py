@@ -10,6 +10,7 @@ from oracle.zo import draw_z
 from workloads import config, make_decoder_problem
 
 from gpu_util import run_gpu
+from test_gpu_bf16_estimate import UPDATE_TOL, update_from_gpu_g
 
 pytestmark = pytest.mark.gpu
 
@@ -27,6 +28,8 @@ def test_sampled_row_losses_against_oracle(problem):
     q, E, P = spec.q, spec.E, spec.n_labelled
     rows = got["rows"].reshape(2 * q, E, P)
     assert np.isfinite(got["losses"]).all() and got["launches"] > 0
+    # the update line of Algorithm 1 alone: the oracle's formula fed the GPU's g
+    assert update_from_gpu_g(spec, p, seed, got) < UPDATE_TOL
     # replica means are the means of their rows
     assert np.allclose(rows.mean(axis=(1, 2)), got["losses"], rtol=1e-5)
     zs = {}
