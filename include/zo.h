@@ -168,8 +168,12 @@ typedef struct zo_lora {
 /* Bytes of device workspace zo_init needs for this configuration (0 on a bad config). */
 ZO_API size_t zo_workspace_bytes(const zo_config* cfg);
 
-/* Validates cfg, partitions the workspace, creates the context.  `cuda_stream` is a
+/* Set-up of the inputs Algorithm 1 lists before its loop (model, loss kind, bounds on q and the batch):
+ * validates cfg, partitions the workspace, creates the context.  `cuda_stream` is a
  * cudaStream_t (NULL = legacy default stream) on which every later call enqueues.
+ * Several devices in one process: call with the context's device current, here and in every later call
+ * on the context; per-device set-up of the kernels is done on first use and host threads may call in
+ * concurrently (one context is still one thread's at a time).
  * Unsupported (ZO_ERR_UNSUPPORTED): d_model % n_heads != 0; head_dim not in
  * {16, 32, 64, 128}; max_seq > 512; (r * k_out) % 4 != 0; ZO_BF16 with d_model, d_ffn or
  * d_out not a multiple of 8 (16-byte row pitch needed by the tensor-memory-accelerator loads). */
@@ -215,8 +219,10 @@ ZO_API zo_status zo_step_host(zo_ctx* ctx, const zo_weights* weights, const zo_l
                        const void* host_tokens, const void* host_labels, int32_t E, int32_t S,
                        uint64_t seed, int32_t q, float eps, float lr);
 
-/* Synchronises the stream and copies out the last step's 2q losses (replica order) and,
- * if host_g != NULL, its q projected gradients.  Returns the step's deferred status. */
+/* The outputs of Algorithm 1's inner and outer loops: synchronises the stream and copies out the last
+ * step's 2q losses l^(k) of the perturbed parameters theta_l + k eps z_i (replica order n = 2i + {0: +,
+ * 1: -}) and, if host_g != NULL, its q projected gradients g_i = (l^(+1) - l^(-1)) / (2 eps), the
+ * scalars Algorithm 1 stores next to the seeds.  Returns the step's deferred status. */
 ZO_API zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g);
 
 /* Diagnostics: per labelled-row losses of the last step, [2q][rows] with rows in
@@ -296,7 +302,7 @@ ZO_API zo_status zo_profile_read(zo_ctx* ctx, double* host_ms, double* host_flop
                                  int32_t* host_launches);
 
 ZO_API void zo_free(zo_ctx* ctx);
-ZO_API const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo_init failure */
+ZO_API const char* zo_last_error(const zo_ctx* ctx); /* ctx may be NULL: last zo_init failure of the calling thread */
 
 /* The perturbation stream itself (Algorithm 1: z_i from s_i), for bit-level checks:
  * writes the first n raw 32-bit words (dev_u32, may be NULL) and normals (dev_z, may be
@@ -352,6 +358,13 @@ ZO_API zo_status zo_mp_lora_linear_static(void* cuda_stream, int32_t precision, 
                                           int32_t k_out, int32_t r, float scale, uint64_t seed,
                                           uint32_t tensor_id, int32_t q, float eps,
                                           int32_t x_replicated, uint32_t flags);
+/* Deferred device-side status of the calls made so far through zo_mp_lora_linear_static on the
+ * current device: the call itself only enqueues work, and its status word lives inside the fixed
+ * array, out of the caller's reach.  Copies that word to *host_status on `cuda_stream` (use the
+ * stream of the call) and waits for the stream; allocates nothing.  Returns ZO_ERR_TIMEOUT when a
+ * bounded device-side wait ran out (Y is then void), ZO_OK otherwise.  The word is cleared by the
+ * next zo_mp_lora_linear_static call. */
+ZO_API zo_status zo_mp_lora_linear_static_status(void* cuda_stream, uint32_t* host_status);
 
 #ifdef __cplusplus
 }

@@ -11,7 +11,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libzo_b200.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError(
-        f"{_LIB_PATH} is missing: build it with `python -m paper_2409_15520_b200.build` "
+        f"{_LIB_PATH} is missing: build it with `python paper_2409_15520_b200/build.py` "
         "(there is no CPU or PyTorch fallback)")
 LIB = C.CDLL(_LIB_PATH)
 
@@ -105,6 +105,8 @@ zo_mp_lora_linear_static = _sig("zo_mp_lora_linear_static", C.c_int, [
     C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
     C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_uint64, C.c_uint32, C.c_int32,
     C.c_float, C.c_int32, C.c_uint32])
+zo_mp_lora_linear_static_status = _sig("zo_mp_lora_linear_static_status", C.c_int,
+                                       [C.c_void_p, C.POINTER(C.c_uint32)])
 STATIC_SCRATCH_BYTES = 16 << 20
 
 
@@ -360,3 +362,13 @@ def mp_lora_linear_static(X, W, bias, A, B, Y, T, q, scale, seed, tensor_id, eps
     if st:
         raise ZoError(st, "zo_mp_lora_linear_static")
     return Y
+
+
+def mp_lora_linear_static_status():
+    """Waits for the current stream and returns the device status word of the calls made through
+    mp_lora_linear_static on the current device (0 = fine); raises ZoError on a timed-out wait."""
+    word = C.c_uint32()
+    st = zo_mp_lora_linear_static_status(C.c_void_p(torch.cuda.current_stream().cuda_stream), C.byref(word))
+    if st:
+        raise ZoError(st, f"device status word {word.value}")
+    return int(word.value)

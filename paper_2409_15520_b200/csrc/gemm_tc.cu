@@ -33,6 +33,9 @@
 //     word, drains its copies and MMAs, frees its tensor memory and returns.
 #include <cuda.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "common.cuh"
 #include "kernels.h"
 
@@ -913,15 +916,34 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 static EncodeTiledFn g_encode = nullptr;
 
+// Per-device set-up (the opt-in to large dynamic shared memory is a per-device attribute of each
+// kernel, and the number of co-resident CTA pairs is a property of the device): done once per
+// device ordinal, with that device current, under a mutex so that host threads may race into it.
+constexpr int kMaxDevices = 64;
+static std::mutex g_setup_mutex;
+static std::atomic<bool> g_dev_ready[kMaxDevices];
+static int g_max_clusters[kMaxDevices];   // co-resident CTA pairs, 0 = not yet asked
+
+static int current_device(int* dev) {
+  const cudaError_t e = cudaGetDevice(dev);
+  if (e != cudaSuccess) return (int)e;
+  return (*dev < 0 || *dev >= kMaxDevices) ? (int)cudaErrorInvalidDevice : 0;
+}
+
 int gemm_tc_init() {
-  if (g_encode) return 0;
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
-  if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return e ? (int)e : 999;
-  g_encode = (EncodeTiledFn)fn;
-  e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)tc::SMEM_BYTES);
+  int dev = 0;
+  if (const int e = current_device(&dev)) return e;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    const cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return e ? (int)e : 999;
+    g_encode = (EncodeTiledFn)fn;
+  }
+  if (g_dev_ready[dev].load(std::memory_order_relaxed)) return 0;
+  cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)tc::SMEM_BYTES);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
@@ -931,6 +953,7 @@ int gemm_tc_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess) g_dev_ready[dev].store(true, std::memory_order_release);
   return (int)e;
 }
 
@@ -949,9 +972,11 @@ static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, 
 int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_sms) {
   if (G.M <= 0 || G.N <= 0) return 0;
   if (G.K <= 0) return (int)cudaErrorInvalidValue;   // every tile needs at least one base k-block
-  if (!g_encode) {
-    const int e = gemm_tc_init();
-    if (e) return e;
+  int dev = 0;
+  if (const int de = current_device(&dev)) return de;
+  if (!g_dev_ready[dev].load(std::memory_order_acquire)) {
+    const int ie = gemm_tc_init();
+    if (ie) return ie;
   }
   CUtensorMap tmA, tmB;
   int e = make_map(&tmA, G.A, (uint64_t)G.K, (uint64_t)G.M, (uint64_t)G.lda);
@@ -982,7 +1007,11 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.ksplit = 1; P.part = nullptr;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
   const long long tiles2 = (long long)((P.M + 2 * tc::BM - 1) / (2 * tc::BM)) * tiles_n;   // 256-row tiles
-  static int max_clusters = 0;                       // co-resident CTA pairs on this device
+  int max_clusters = 0;                              // co-resident CTA pairs on this device
+  if (G.cta_pair) {
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    max_clusters = g_max_clusters[dev];
+  }
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -997,6 +1026,8 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
       mc = n_sms / 2;
     }
     max_clusters = mc < n_sms / 2 ? mc : n_sms / 2;
+    std::lock_guard<std::mutex> lock(g_setup_mutex);
+    g_max_clusters[dev] = max_clusters;
   }
   // cta_pair 1: pairs wherever the kernel allows; 2: pairs for the launches they were measured faster on:
   // no low-rank term or its one-block tensor-core form (below), at least

@@ -54,3 +54,20 @@ extern "C" zo_status zo_mp_lora_linear_static(void* cuda_stream, int32_t precisi
                            seed, tensor_id, q, eps, x_replicated, scratch,
                            (size_t)ZO_STATIC_SCRATCH_BYTES, flags);
 }
+
+// The status word of the last zo_mp_lora_linear_static call on the current device (it sits at the
+// head of the fixed array, where the caller cannot read it).  One 4-byte copy on the given stream
+// and a wait for that stream; nothing is allocated.
+extern "C" zo_status zo_mp_lora_linear_static_status(void* cuda_stream, uint32_t* host_status) {
+  if (!host_status) return ZO_ERR_INVALID_ARG;
+  void* scratch = nullptr;
+  const zo_status s = static_scratch(&scratch);
+  if (s != ZO_OK) return s;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, scratch, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess)
+    return ZO_ERR_CUDA;
+  *host_status = word;
+  return (word & 1u) ? ZO_ERR_TIMEOUT : ZO_OK;   // bit 0: a bounded device-side wait ran out
+}

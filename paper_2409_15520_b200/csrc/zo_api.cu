@@ -14,7 +14,11 @@ using namespace zo;
 
 namespace {
 
-char g_init_error[256] = "";
+// text of the last zo_init failure of the calling thread (zo_last_error(NULL))
+thread_local char g_init_error[256] = "";
+
+constexpr int ZO_MAX_Q = 32;            // largest q a context accepts; sizes the per-step pass lists
+constexpr int MAX_PASSES = 2 * ZO_MAX_Q;  // the sequential schedule cuts a step into 2q passes
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
@@ -44,7 +48,7 @@ zo_status check_config(const zo_config* c, char* err, size_t errn) {
   if (c->loss_kind < ZO_LOSS_MSE || c->loss_kind > ZO_LOSS_CE_LABEL_WORDS)
     BAD(ZO_ERR_INVALID_ARG, "bad loss_kind");
   if (c->lora_rank < 1 || c->lora_rank > 64) BAD(ZO_ERR_INVALID_ARG, "lora_rank must be 1..64");
-  if (c->max_q < 1 || c->max_q > 32) BAD(ZO_ERR_INVALID_ARG, "max_q must be 1..32");
+  if (c->max_q < 1 || c->max_q > ZO_MAX_Q) BAD(ZO_ERR_INVALID_ARG, "max_q must be 1..32");
   if (c->max_E < 1 || c->max_seq < 1) BAD(ZO_ERR_INVALID_ARG, "max_E and max_seq must be >= 1");
   if (c->d_model < 1) BAD(ZO_ERR_INVALID_ARG, "d_model must be >= 1");
   if (!isfinite(c->lora_scale)) BAD(ZO_ERR_INVALID_ARG, "lora_scale not finite");
@@ -358,7 +362,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   double* rowloss_pass = c->at<double>(c->plan.rowloss_pass);
   float* losses = c->at<float>(c->plan.losses);
   double* losses_d = c->at<double>(c->plan.losses_d);
-  Pass passes[64];
+  Pass passes[MAX_PASSES];
   const int n_pass = step_passes(c, q, passes);
   for (int pi = 0; pi < n_pass; ++pi) {
   const Pass ps = passes[pi];
@@ -430,7 +434,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   }
   PROF(PC_MISC, 0.0, launch_label_scan(st, labels, sl, P, n_classes, lab_idx, lab_val, lab_cnt, status));
 
-  Pass passes[64];
+  Pass passes[MAX_PASSES];
   const int n_pass = step_passes(c, q, passes);
   for (int pi = 0; pi < n_pass; ++pi) {
   const Pass ps = passes[pi];
@@ -653,11 +657,16 @@ zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
       return ZO_ERR_CUDA;
     }
   }
-  zo_ctx* c = new (std::nothrow) zo_ctx;
-  if (!c) { snprintf(g_init_error, sizeof(g_init_error), "out of host memory"); return ZO_ERR_CUDA; }
-  memset(c, 0, sizeof(*c));
-  c->prof = new (std::nothrow) std::vector<ProfRec>();
-  c->evpool = new (std::nothrow) std::vector<cudaEvent_t>();
+  zo_ctx* c = new (std::nothrow) zo_ctx();   // value-initialised: every field zero
+  if (c) {
+    c->prof = new (std::nothrow) std::vector<ProfRec>();
+    c->evpool = new (std::nothrow) std::vector<cudaEvent_t>();
+  }
+  if (!c || !c->prof || !c->evpool) {
+    snprintf(g_init_error, sizeof(g_init_error), "out of host memory");
+    zo_free(c);
+    return ZO_ERR_CUDA;
+  }
   c->cfg = *cfg; c->plan = plan; c->ws = (uint8_t*)workspace; c->st = (cudaStream_t)cuda_stream;
   c->bf = cfg->precision == ZO_BF16; c->n_sms = sms;
   c->nt = cfg->arch == ZO_ARCH_LINEAR ? 1 : n_targets(*cfg);
@@ -671,7 +680,7 @@ zo_status zo_init(const zo_config* cfg, void* workspace, size_t workspace_bytes,
   }
   if (e != cudaSuccess) {
     snprintf(g_init_error, sizeof(g_init_error), "workspace set-up: %s", cudaGetErrorString(e));
-    delete c;
+    zo_free(c);
     return ZO_ERR_CUDA;
   }
   *out = c;
@@ -887,7 +896,7 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
                             void* scratch, size_t scratch_bytes, uint32_t flags) {
   if (!X || !W || !A || !B || !Y || !scratch) return ZO_ERR_INVALID_ARG;
   if (precision != ZO_FP32 && precision != ZO_BF16) return ZO_ERR_INVALID_ARG;
-  if (T < 1 || k_in < 1 || k_out < 1 || r < 1 || r > 64 || q < 1 || q > 32 || !(eps >= 0.f))
+  if (T < 1 || k_in < 1 || k_out < 1 || r < 1 || r > 64 || q < 1 || q > ZO_MAX_Q || !(eps >= 0.f))
     return ZO_ERR_INVALID_ARG;
   const int bf = precision == ZO_BF16;
   if (k_out % 4) return ZO_ERR_UNSUPPORTED;

@@ -70,8 +70,10 @@ def test_bf16_projected_gradients_per_query(arch, targets):
     for kw in (dict(flags=PAIR), dict(flags=LORA_EPI), dict(flags=SIMT), dict(schedule="inner_only"),
                dict(schedule="sequential")):
         got = check_estimate(spec, p, ref, seed, EPS, **kw)
-        if kw.get("flags") == PAIR or "schedule" in kw:
+        if kw.get("flags") == PAIR or kw.get("schedule") == "inner_only":
             # same operands in the same order: the tile shape and the cut into passes change no bit
+            # (the one-replica passes of the sequential schedule are small enough for split K, which
+            # sums in another order)
             assert np.array_equal(got["g"], base["g"]) and np.array_equal(got["losses"], base["losses"])
 
 

@@ -35,7 +35,7 @@ def test_static_scratch_entry_matches_regular_entry_twice(bf16, x_replicated):
         ref = zo.mp_lora_linear(X, W, bias, A, B, T, q, 2.0, seed, 4, eps, x_replicated)
         Y = torch.full((2 * q, T, ko), float("nan"), dtype=dtype, device="cuda")
         zo.mp_lora_linear_static(X, W, bias, A, B, Y, T, q, 2.0, seed, 4, eps, x_replicated)
-        torch.cuda.synchronize()
+        assert zo.binding.mp_lora_linear_static_status() == 0   # also waits for the stream
         got, want = Y.float().cpu().numpy(), ref.float().cpu().numpy()
         assert np.isfinite(got).all()
         # same kernels, same order of operations: the parity tests' bf16 tolerance is 2e-2;
