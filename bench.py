@@ -26,11 +26,11 @@ from workloads.spec import ARCH_LINEAR, ARCH_OPT  # noqa: E402
 
 METRIC, UNIT = "perturbed_fwd_tokens_per_s", "tokens/s"
 
-# DRAM bytes (read + write) of one gate|up GEMM launch of gemm_tc_kernel<false>, from the ncu capture
-# summarised in profiles/kernels_llama7b_q1_2layers.md: 960.4 MB at 8192 token rows.  Traffic
-# grows in proportion to the rows (activations, outputs and one weight-panel read per 2048 rows), so
-# the full launch is scaled by rows.  Set to None whenever that kernel changes after the capture.
-GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 960.4e6 / 8192}
+# DRAM bytes (read + write) per token row of one gate|up launch of the tensor-core GEMM, from an ncu
+# capture (dram__bytes_read.sum + dram__bytes_write.sum) of that launch at 8192 token rows; activations,
+# outputs and one weight-panel read per raster group all grow with the rows, so a full launch is scaled
+# by rows.  None = the kernel changed since the counters were taken.
+GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": None}
 
 
 def _peaks():
@@ -98,6 +98,30 @@ def max_over_ranks(values, device):
     return t.tolist()
 
 
+def rank_command(n, argv):
+    """Command line that starts n ranks of this script on one node (one process per GPU, rendezvous on
+    the loopback address), as the launcher of `--gpus n` does when no launcher started us."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__), *argv]
+
+
+def timed_region(step, steps, barrier, stamp):
+    """Exactly `steps` calls of step(i) between two barriers; the time between the two stamps in ms.
+    `barrier()` lines the ranks up and drains the device; `stamp()` returns an object with
+    elapsed_time(later_stamp) in ms (a CUDA event on the launching stream)."""
+    barrier()
+    t0 = stamp()
+    for i in range(steps):
+        step(i)
+    t1 = stamp()
+    barrier()
+    return t0.elapsed_time(t1)
+
+
 def whole_job_value(world, units_per_step, steps, ms):
     return world * units_per_step * steps / (ms * 1e-3)
 
@@ -129,26 +153,40 @@ def algorithmic_flops_per_step(spec):
 
 
 def oracle_sample(spec, seed=1234):
-    """Bounded CPU sample of the same workload: the oracle's zo_step with q = 1 (one +/- pair) on up to
-    eight sequences of the batch through a 2-block copy of the model.  Returns (seconds, token-forwards done,
-    scale to full depth)."""
+    """Bounded CPU sample of the same workload: the oracle's two perturbed forward passes of one query
+    (q = 1, the +/- pair) on up to eight sequences of the batch through a 2-block copy of the model.
+    The decoder blocks and the loss head (final norm, LM head, cross-entropy on the labelled rows) are
+    timed apart, so only the blocks' time is scaled to the full depth.
+    Returns (seconds of the sample, seconds scaled to the full model, token-forwards done, description)."""
     import oracle
+    from oracle.model import decoder_hidden, row_losses
+    from oracle.zo import draw_z
     if spec.arch == ARCH_LINEAR:
         small = spec.with_(q=1)
         p = make_linear_problem(small, seed=seed, b_std=0.01)
         t0 = time.perf_counter()
         oracle.zo_step(small, p, p["X"], p["target"], 1, 1, spec.eps, spec.lr)
-        return time.perf_counter() - t0, 2 * small.E * small.S, 1.0, "q=1 on the full token block"
+        dt = time.perf_counter() - t0
+        return dt, dt, 2 * small.E * small.S, "q=1 on the full token block"
     L = min(2, spec.n_layers)
     Es = min(8, spec.E)                      # sized for 10-30 s of CPU work at the 7B shape
     small = spec.with_(n_layers=L, E=Es, q=1)
     p = make_decoder_globals(small, seed)
     p["layers"] = [make_decoder_layer(small, seed, l, 0.01) for l in range(L)]
-    t0 = time.perf_counter()
-    oracle.zo_step(small, p, p["tokens"], p["labels"], 1, 1, spec.eps, spec.lr)
-    dt = time.perf_counter() - t0
-    return (dt, 2 * Es * small.S, spec.n_layers / L,
-            f"q=1, {Es} sequences of {small.S} tokens, {L} of {spec.n_layers} blocks (time scaled by depth)")
+    z = draw_z(small, p, 1, 0)
+    t_blocks = t_head = 0.0
+    for k in (+1.0, -1.0):                   # theta + k eps z, one forward pass each (Algorithm 1)
+        Bn = [(np.asarray(Lr["B"], np.float64) + k * spec.eps * z[l])[None] for l, Lr in enumerate(p["layers"])]
+        t0 = time.perf_counter()
+        h = decoder_hidden(small, p, Bn, p["tokens"])
+        t1 = time.perf_counter()
+        row_losses(small, p, h, p["labels"]).mean()
+        t2 = time.perf_counter()
+        t_blocks += t1 - t0
+        t_head += t2 - t1
+    return (t_blocks + t_head, t_blocks * spec.n_layers / L + t_head, 2 * Es * small.S,
+            f"q=1, {Es} sequences of {small.S} tokens, {L} of {spec.n_layers} blocks "
+            f"(blocks' time scaled by depth, loss head timed apart and not scaled)")
 
 
 def run_sweep(args):
@@ -296,8 +334,8 @@ def run_reference(args, spec):
         oracle_sample(spec)
     times = []
     for _ in range(args.steps):
-        dt, toks, scale, what = oracle_sample(spec)
-        times.append(dt * scale)
+        _, full, toks, what = oracle_sample(spec)
+        times.append(full)
     sec = float(np.sum(times))
     value = toks * args.steps / sec
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -358,6 +396,10 @@ def main():
     if args.varlen:
         return run_varlen(args, spec)
 
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # asked for N GPUs without a launcher around us: start the N ranks ourselves
+        raise SystemExit(subprocess.call(rank_command(args.gpus, sys.argv[1:])))
+
     import torch
     import torch.distributed as dist
     import paper_2409_15520_b200 as zo
@@ -370,13 +412,17 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    prob = load_problem(spec, weights=args.weights)
-    est = zo.Estimator(zo.make_config(spec, flags=args.flags, weight_format=args.weights))
-    est.set_schedule(args.schedule)
     E, S, q, eps, lr = spec.E, spec.S, spec.q, spec.eps, spec.lr
     tokens_per_step = 2 * q * E * S
     sharded = args.shard_queries
     jobs = 1 if sharded else world            # independent steps in flight across the ranks
+    if sharded and world > q:
+        raise SystemExit("--shard-queries needs at least one query per rank")
+    # a rank that only ever runs its block of queries needs activations for that block alone
+    max_shard_q = zo.query_shard(q, world, 0)[1] if sharded else 0
+    prob = load_problem(spec, weights=args.weights)
+    est = zo.Estimator(zo.make_config(spec, flags=args.flags, weight_format=args.weights, max_shard_q=max_shard_q))
+    est.set_schedule(args.schedule)
 
     def one_step(seed, host=False):
         if not sharded:
@@ -384,52 +430,50 @@ def main():
         begin, count = zo.query_shard(q, world, rank)
         est.set_query_shard(begin, count)
         (est.step_host if host else est.step)(prob, E, S, seed, q, eps, 0.0)
-        zo.exchange_losses(est.loss_buffer(), q)
+        est.set_query_shard(0, 0)
+        zo.exchange_step(est.loss_buffer())
         est.apply_update(prob, seed, q, eps, lr)
-
-    if sharded and world > q:
-        raise SystemExit("--shard-queries needs at least one query per rank")
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    def stamp():
+        e = torch.cuda.Event(enable_timing=True)
+        e.record()
+        return e
+
     for i in range(max(args.warmup, 3)):
         one_step(100 + i)
     est.losses()
+    # (1) the headline: K steps, no per-launch instrumentation
     sampler = ClockSampler(local)
-    est.profile_enable(True)
-    est.profile_read()
-    barrier()
     sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for i in range(args.steps):
-        one_step(1000 + i)
-    ev1.record()
-    barrier()
+    ms = timed_region(lambda i: one_step(1000 + i), args.steps, barrier, stamp)
     clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1)
-    prof = est.profile_read()
-    est.profile_enable(False)
     losses, g = est.losses()
     launches = est.launch_count() * args.steps
 
-    # end to end: host tokens/labels in, losses out, every step
-    barrier()
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
+    # (2) end to end: host tokens/labels in, losses out, every step
+    def e2e_step(i):
         one_step(2000 + i, host=True)
         est.losses()
-    e1.record()
-    barrier()
-    ms_e2e = max(e0.elapsed_time(e1), 1e3 * (time.perf_counter() - t0))
+    t0 = time.perf_counter()
+    ms_e2e = timed_region(e2e_step, args.steps, barrier, stamp)
+    ms_e2e = max(ms_e2e, 1e3 * (time.perf_counter() - t0))
     h2d = prob.host_tokens.numel() * prob.host_tokens.element_size() + \
         prob.host_labels.numel() * prob.host_labels.element_size()
     d2h = (2 * q + q) * 4 + 4
+
+    # (3) a second, instrumented pass (every launch bracketed by CUDA events on the launching stream) for
+    # the per-kernel figures and the roofline; its events cost time, so it does not feed `value`
+    prof_steps = min(args.steps, 5)
+    est.profile_enable(True)
+    est.profile_read()
+    ms_prof = timed_region(lambda i: one_step(3000 + i), prof_steps, barrier, stamp)
+    prof = est.profile_read()
+    est.profile_enable(False)
 
     ms, ms_e2e = max_over_ranks([ms, ms_e2e], "cuda")
     if rank != 0:
@@ -444,6 +488,7 @@ def main():
     inside_long_step = ms / args.steps > 200.0
     peak = peaks["tflops_sustained"] if inside_long_step else peaks["tflops"]
     total_prof = sum(v[0] for v in prof.values())
+    fc1_bytes_per_row = GEMM_FC1_DRAM_BYTES_PER_ROW.get(args.workload)
     line = {
         "metric": METRIC, "value": whole_job_value(jobs, tokens_per_step, args.steps, ms), "unit": UNIT,
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
@@ -455,7 +500,7 @@ def main():
                    "token_rows_per_step": tokens_per_step, "eps": eps, "lr": lr,
                    "l2": "inputs larger than L2 (weights and activations of several GB stream every step)",
                    "schedule": args.schedule, "weights": args.weights or "bf16",
-                   "parallelism": (f"queries of one step sharded over {world} gpu(s), all-reduce of 2q losses" if sharded
+                   "parallelism": (f"queries of one step sharded over {world} gpu(s), all-reduce of the loss array" if sharded
                                    else "replicas only" if world > 1 else "1 gpu")},
         "zo_steps_per_s": jobs * args.steps / (ms * 1e-3),
         "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,
@@ -466,21 +511,25 @@ def main():
         "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": gemm_tflops, "peak": peak,
                      "unit": "TFLOP/s", "frac": gemm_tflops / peak if peak else None,
                      "peak_source": f"{peaks['source']} ({'sustained' if inside_long_step else 'burst'} bf16)",
+                     "frac_of_burst_peak": gemm_tflops / peaks["tflops"],
+                     "frac_of_sustained_peak": gemm_tflops / peaks["tflops_sustained"],
+                     "frac_of_nominal_2250": gemm_tflops / 2250.0,
+                     "measured_in": f"instrumented pass of {prof_steps} steps, {ms_prof / prof_steps:.3f} ms/step",
                      "launches": gcnt, "avg_launch_ms": gms / gcnt if gcnt else None,
-                     "traffic": (GEMM_FC1_DRAM_BYTES_PER_ROW[args.workload] * tokens_per_step
-                                 if GEMM_FC1_DRAM_BYTES_PER_ROW.get(args.workload)
+                     "traffic": (fc1_bytes_per_row * tokens_per_step
+                                 if fc1_bytes_per_row
                                  and not (args.flags or args.rank or args.targets >= 0 or args.weights) else None),
-                     "traffic_note": "gate|up launch (41 % of the step), ncu capture of the same single-CTA kernel at 8192 rows scaled by rows"},
+                     "traffic_note": "gate|up launch (the largest GEMM class of the step): ncu capture of that launch at 8192 token rows, scaled by rows"},
         "gemm_tflops_by_class": {k: round(prof[k][1] / (prof[k][0] * 1e-3) / 1e12, 1)
                                  for k in gemm_classes if prof[k][0] > 0},
         "kernel_time_share": {k: round(v[0] / total_prof, 4) for k, v in prof.items() if v[2]},
-        "kernel_ms_per_step": {k: round(v[0] / args.steps, 3) for k, v in prof.items() if v[2]},
+        "kernel_ms_per_step": {k: round(v[0] / prof_steps, 3) for k, v in prof.items() if v[2]},
         "loss_mean": float(np.mean(losses)),
     }
     if not args.no_cpu_baseline and world == 1:
         import torch as _t
-        dt, toks, scale, what = oracle_sample(spec)
-        line["cpu_baseline"] = {"value": toks / (dt * scale), "unit": UNIT, "cores": _t.get_num_threads(),
+        dt, full, toks, what = oracle_sample(spec)
+        line["cpu_baseline"] = {"value": toks / full, "unit": UNIT, "cores": _t.get_num_threads(),
                                 "kind": "oracle", "sample": what, "seconds": dt}
     print(json.dumps(line))
     if world > 1:

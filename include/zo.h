@@ -96,7 +96,10 @@ enum { ZO_FLAG_SIMT_GEMM = 1,
        /* ZO_FLAG_LORA_EPILOGUE: the MP-LoRA term is always added on CUDA cores in the GEMM epilogue
         * from fp32 U and fp32 (B + k eps z), never as the extra tensor-core k-block (which rounds
         * U, B and k eps z to bfloat16).  A/B switch. */
-       ZO_FLAG_LORA_EPILOGUE = 4 };
+       ZO_FLAG_LORA_EPILOGUE = 4,
+       /* ZO_FLAG_TEST_EXPIRE_WAIT (zo_mp_lora_linear only; contexts use zo_test_expire_wait): failure-
+        * detection test aid, see zo_test_expire_wait. */
+       ZO_FLAG_TEST_EXPIRE_WAIT = 1 << 24 };
 /* Bits 8..15 of flags, when non-zero, override the tensor-core GEMM's raster group (128-row tiles that
  * sweep the weight panels together; default 16).  Tuning aid; results do not depend on it.
  * Bits 16..20, when non-zero, bound the number of K ranges the tensor-core GEMM cuts a tile into when a
@@ -130,6 +133,10 @@ typedef struct zo_config {
   int32_t tie_lm_head; /* 1: LM head = token embedding                               */
   uint32_t flags;
   int32_t weight_format; /* ZO_W_*; quantised formats need k_in % 64 == 0 (NF4) and decoders   */
+  int32_t max_shard_q;   /* 0, or the largest number of queries this context runs in ONE step when it only
+                          * ever runs query shards (zo_set_query_shard): the activation workspace is then
+                          * sized for 2 * max_shard_q replicas instead of 2 * max_q, so a device's memory
+                          * shrinks with the number of devices.  Steps with more queries are rejected. */
 } zo_config;
 
 /* Frozen tensors of one decoder block (device pointers; element type per precision).
@@ -264,25 +271,41 @@ ZO_API zo_status zo_set_schedule(zo_ctx* ctx, int32_t schedule);
  *       from the step otherwise).  q_count = 0 (with q_begin = 0) switches sharding off.  The
  *       schedule set by zo_set_schedule applies inside the shard.
  *   zo_loss_buffer(ctx, &dev_losses, &capacity)
- *       Device address of the step's float64 loss array (replica order, `capacity` = 2*max_q
- *       entries, inside the caller's workspace).  After a sharded step it holds this shard's
- *       losses and zeros elsewhere, so a sum over devices (an all-reduce of 2q doubles, exact
- *       since every entry has one non-zero contributor) or an all-gather of the shards completes
- *       it.  The exchange itself is the caller's: enqueue it on the context's stream, or order it
- *       with the stream by events.
+ *       Device address of the step's float64 loss array (inside the caller's workspace):
+ *       `capacity` = 2*max_q + 1 entries, the losses in replica order followed by one fault slot.
+ *       After a sharded step it holds this shard's losses, zeros at every other loss, and in the
+ *       fault slot 1.0 if this device's status word is set (bounded wait ran out, bad token or
+ *       label, non-finite loss), else 0.0.  A sum over devices of the WHOLE array (one all-reduce
+ *       of 2*max_q + 1 doubles; exact, since every loss has one non-zero contributor) completes
+ *       the losses and tells every device whether any device faulted.  The exchange itself is the
+ *       caller's: enqueue it on the context's stream, or order it with the stream by events.
  *   zo_apply_update(ctx, lora, seed, q, eps, lr)
  *       g_i = (l_{2i} - l_{2i+1}) / (2 eps) from the loss array as it then stands, and
  *       B <- B - lr (1/q) sum_i g_i z_i on this device's B.  Asynchronous on the context's stream.
- *       A non-finite loss from any device leaves B untouched on every device (all see the same
- *       array); zo_losses afterwards returns all 2q losses and g and the deferred status.
+ *       A non-finite loss from any device, or a non-zero fault slot, leaves B untouched on every
+ *       device (all see the same array), so the copies of B cannot drift apart; zo_losses
+ *       afterwards returns all 2q losses and g and the deferred status: the device's own fault if
+ *       it had one, ZO_ERR_STATE when only another device did.
  *       Also valid after an unsharded step with lr = 0 (apply the step later).
- * A device-side fault on ONE device (ZO_ERR_TIMEOUT, bad token or label) skips that device's update
- * only: check zo_losses on every device before the next step.  zo_row_losses after a sharded step
- * holds this shard's rows only. */
+ * If only the 2q losses are exchanged (fault slot left out), a device-side fault on ONE device skips
+ * that device's update only: check zo_losses on every device before the next step.  zo_row_losses
+ * after a sharded step holds this shard's rows only. */
 ZO_API zo_status zo_set_query_shard(zo_ctx* ctx, int32_t q_begin, int32_t q_count);
 ZO_API zo_status zo_loss_buffer(zo_ctx* ctx, double** dev_losses, int32_t* host_capacity);
 ZO_API zo_status zo_apply_update(zo_ctx* ctx, const zo_lora* lora, uint64_t seed, int32_t q,
                                  float eps, float lr);
+
+/* Failure-detection test aid; off (0) by default and in every measured run.  Every device-side wait of
+ * the tensor-core GEMM (on a shared-memory barrier that a copy or a tensor-core instruction completes) is
+ * bounded: when it runs out, the thread block raises the time-out bit of the status word, lets the copies
+ * and tensor-core instructions it has issued finish, frees its tensor memory and returns, and zo_losses
+ * reports ZO_ERR_TIMEOUT with B untouched.  Nothing in a correct run makes a wait run out, so this call
+ * arranges it without faulting anything: while wait_limit_ns > 0, every tensor-core GEMM launch of the
+ * context runs one thread block per tile, gives up its waits after wait_limit_ns (<= 2e9), and the copy
+ * engine of thread block 0 goes silent after its first k-block (nothing armed, nothing in flight), so
+ * that block's tensor-core warp waits for a stage that never arrives.  wait_limit_ns = 0 restores
+ * normal operation; the context, the stream and the device stay usable throughout. */
+ZO_API zo_status zo_test_expire_wait(zo_ctx* ctx, uint64_t wait_limit_ns);
 
 /* Number of kernels the last zo_step enqueued. */
 ZO_API int32_t zo_launch_count(const zo_ctx* ctx);

@@ -9,4 +9,4 @@ from .binding import (  # noqa: F401
     LIB, ZoConfig, ZoError, Estimator, DeviceProblem, make_config, perturbation,
     mp_lora_linear, mp_lora_linear_static, STATUS_NAMES,
 )
-from .sharding import query_shard, exchange_losses, sharded_step  # noqa: F401
+from .sharding import query_shard, exchange_losses, exchange_step, sharded_step  # noqa: F401

@@ -19,6 +19,7 @@ STATUS_NAMES = ["ZO_OK", "ZO_ERR_INVALID_ARG", "ZO_ERR_UNSUPPORTED", "ZO_ERR_WOR
                 "ZO_ERR_CUDA", "ZO_ERR_TIMEOUT", "ZO_ERR_NONFINITE", "ZO_ERR_STATE"]
 ZO_FP32, ZO_BF16 = 0, 1
 ZO_FLAG_SIMT_GEMM, ZO_FLAG_GEMM_PAIR, ZO_FLAG_LORA_EPILOGUE, ZO_FLAG_GEMM_SINGLE = 1, 2, 4, 8
+ZO_FLAG_TEST_EXPIRE_WAIT = 1 << 24
 
 
 class ZoError(RuntimeError):
@@ -36,7 +37,8 @@ class ZoConfig(C.Structure):
                 ("lora_scale", C.c_float), ("lora_targets", C.c_uint32),
                 ("label_words", C.c_int32 * 2), ("max_q", C.c_int32), ("max_E", C.c_int32),
                 ("max_labelled", C.c_int32), ("norm_eps", C.c_float), ("rope_theta", C.c_float),
-                ("tie_lm_head", C.c_int32), ("flags", C.c_uint32), ("weight_format", C.c_int32)]
+                ("tie_lm_head", C.c_int32), ("flags", C.c_uint32), ("weight_format", C.c_int32),
+                ("max_shard_q", C.c_int32)]
 
 
 _LAYER_FIELDS = ["norm1_g", "norm1_b", "w_qkv", "b_qkv", "w_o", "b_o", "norm2_g", "norm2_b",
@@ -79,6 +81,7 @@ zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTE
 zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
 zo_set_schedule = _sig("zo_set_schedule", C.c_int, [C.c_void_p, C.c_int32])
 zo_set_query_shard = _sig("zo_set_query_shard", C.c_int, [C.c_void_p, C.c_int32, C.c_int32])
+zo_test_expire_wait = _sig("zo_test_expire_wait", C.c_int, [C.c_void_p, C.c_uint64])
 zo_loss_buffer = _sig("zo_loss_buffer", C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32)])
 zo_apply_update = _sig("zo_apply_update", C.c_int, [C.c_void_p, C.POINTER(ZoLora), C.c_uint64, C.c_int32,
                                                     C.c_float, C.c_float])
@@ -114,7 +117,7 @@ WEIGHT_FORMATS = {None: 0, "native": 0, "int8": 1, "nf4": 2}
 
 
 def make_config(spec, *, max_q=None, max_E=None, max_seq=None, max_labelled=None, flags=0,
-                precision=None, weight_format=None) -> ZoConfig:
+                precision=None, weight_format=None, max_shard_q=0) -> ZoConfig:
     """zo_config from a shape record with the attribute names of workloads.ModelSpec."""
     c = ZoConfig()
     c.struct_size = C.sizeof(ZoConfig)
@@ -130,6 +133,7 @@ def make_config(spec, *, max_q=None, max_E=None, max_seq=None, max_labelled=None
     c.norm_eps, c.rope_theta = spec.norm_eps, spec.rope_theta
     c.tie_lm_head, c.flags = int(spec.tie_lm_head), flags
     c.weight_format = WEIGHT_FORMATS[weight_format]
+    c.max_shard_q = max_shard_q
     return c
 
 
@@ -269,8 +273,14 @@ class Estimator:
         (q_count = 0: whole steps again)."""
         self._check(zo_set_query_shard(self._h, q_begin, q_count))
 
+    def test_expire_wait(self, wait_limit_ns):
+        """Failure-detection test aid: bounded waits of the tensor-core GEMM give up after
+        wait_limit_ns and one is made to run out (0 = normal operation)."""
+        self._check(zo_test_expire_wait(self._h, wait_limit_ns))
+
     def loss_buffer(self):
-        """The step's float64 loss array [2 * max_q] as a tensor aliasing the workspace."""
+        """The step's float64 loss array as a tensor aliasing the workspace: [2 * max_q] losses
+        followed by the fault slot of a sharded step."""
         ptr, cap = C.c_void_p(), C.c_int32()
         self._check(zo_loss_buffer(self._h, C.byref(ptr), C.byref(cap)))
         off = ptr.value - self.workspace.data_ptr()

@@ -13,7 +13,8 @@ enum : uint32_t {
   ST_TIMEOUT = 1u,      // a bounded mbarrier wait ran out inside a kernel
   ST_NONFINITE = 2u,    // a replica loss is NaN/Inf
   ST_BAD_LABELS = 4u,   // more labelled positions than max_labelled, or label out of range
-  ST_BAD_TOKEN = 8u     // token id outside [0, vocab)
+  ST_BAD_TOKEN = 8u,    // token id outside [0, vocab)
+  ST_PEER_FAULT = 16u   // sharded step: another device published a fault with its losses
 };
 
 __device__ __forceinline__ float to_f(float x) { return x; }

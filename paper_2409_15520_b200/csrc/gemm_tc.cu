@@ -64,6 +64,7 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct Ctrl {
   unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2], drain, lfull;
+  unsigned long long wait_ns;       // limit of every bounded wait of this CTA
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
@@ -92,6 +93,8 @@ struct Params {
   int n_half;               // 1: at most 128 output columns in all: one weight box per stage, MMAs of N = 128
   int ksplit;               // > 1: the K range of every tile is cut into ksplit units of work
   float4* part;             // ksplit > 1: fp32 partial accumulators, [unit][64 column quads][128 rows]
+  unsigned long long wait_ns;   // limit of the bounded waits (WAIT_LIMIT_NS unless a failure-detection test shortens it)
+  int withhold;             // failure-detection test: CTA 0 never delivers the second k-block of its first tile
 };
 
 // ------------------------------------------------------------------------------ PTX wrappers
@@ -133,7 +136,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctrl* c
     if ((it & 63u) == 0u) {
       if (c->abort) return false;
       if (*reinterpret_cast<volatile uint32_t*>(status) & ST_TIMEOUT) { c->abort = 1u; return false; }
-      if (gtimer() - t0 > WAIT_LIMIT_NS) {
+      if (gtimer() - t0 > c->wait_ns) {
         c->abort = 1u;
         atomicOr(status, ST_TIMEOUT);
         return false;
@@ -358,6 +361,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     mbar_init(smem_u32(&ctrl->lfull), PAIR ? 2 * EP_WARPS : EP_WARPS);
     ctrl->abort = 0u;
     ctrl->ep_go = 0u;
+    ctrl->wait_ns = P.wait_ns;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -386,8 +390,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && SPLIT != 2) {
       uint32_t issued = 0;
-      bool ok = true;
-      for (int tile = t_first; tile < t_end && ok; tile += t_step) {
+      bool ok = true, withheld = false;
+      for (int tile = t_first; tile < t_end && ok && !withheld; tile += t_step) {
         int tm, tn;
         coords(tile, tm, tn);
         const int m0 = tm * TILE_M + (int)rank * BM;
@@ -396,6 +400,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         int ks, kb0, kb1;
         kb_range(tile, ks, kb0, kb1);
         for (int kb = kb0; kb < kb1; ++kb, ++issued) {
+          // failure-detection test: this producer goes silent (nothing armed, nothing in flight), so the
+          // MMA warp's wait for the stage runs out and the CTA takes its abort path
+          if (!PAIR && P.withhold && blockIdx.x == 0 && issued == (kb1 - kb0 > 1 ? 1u : 0u)) { withheld = true; break; }
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
@@ -413,7 +420,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         const int lslot = ks != 0 ? -1 : tile_slot(P, brow0);   // the LoRA block rides with the first K range
-        for (int lkb = 0; ok && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued) {
+        for (int lkb = 0; ok && !withheld && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued) {
           // LoRA k-blocks: only the A operand (packed U) travels through the ring
           const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
@@ -495,7 +502,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       }
       if (!ok) {
-        tc_commit(smem_u32(&ctrl->drain));        // wait for the MMAs already issued
+        // wait for the MMAs already issued (a pair's instructions are tracked by the pair form of the commit)
+        if (PAIR) tc_commit_pair(smem_u32(&ctrl->drain));
+        else tc_commit(smem_u32(&ctrl->drain));
         mbar_wait_drain(smem_u32(&ctrl->drain), 0u);
       }
     }
@@ -1005,6 +1014,8 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   }
   P.status = status;
   P.ksplit = 1; P.part = nullptr;
+  P.wait_ns = G.test_wait_ns ? G.test_wait_ns : tc::WAIT_LIMIT_NS;
+  P.withhold = G.test_wait_ns ? 1 : 0;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
   const long long tiles2 = (long long)((P.M + 2 * tc::BM - 1) / (2 * tc::BM)) * tiles_n;   // 256-row tiles
   int max_clusters = 0;                              // co-resident CTA pairs on this device
@@ -1040,7 +1051,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   // operand serves both 128-row halves of a tile: a replica must then be a whole number of 256-row tiles.
   const bool pair_slab_ok = P.slab && P.kslot == tc::BK && P.L.rows_per_replica % (2 * tc::BM) == 0;
   // (a down-projection that also packs bf16 U always runs single-CTA)
-  const bool pair = P.M > tc::BM && !G.pack_out &&
+  const bool pair = P.M > tc::BM && !G.pack_out && !P.withhold &&
                     (G.cta_pair == 1 || (G.cta_pair == 2 && (!G.lora || pair_slab_ok) && P.N >= tc::BN &&
                                          tiles2 >= 8LL * max_clusters &&
                                          2.0 * (double)G.M * (double)G.N * (double)G.K <= 3.0e12));

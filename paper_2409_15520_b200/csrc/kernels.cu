@@ -987,15 +987,24 @@ __global__ void zo_update_kernel(UpdateDesc D, const double* __restrict__ losses
 // After the losses of other devices' queries have been written into the fp64 array: the fp32 copy
 // that zo_losses reads, and the finiteness check the local reduction did for its own entries.
 __global__ void losses_refresh_kernel(const double* __restrict__ losses_d, float* __restrict__ losses,
-                                      int n, uint32_t* status) {
+                                      int n, const double* __restrict__ fault_slot, uint32_t* status) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  // a fault on any device of a sharded step blocks the update on every device (all see the same slot)
+  if (i == 0 && fault_slot && *fault_slot != 0.0) atomicOr(status, ST_PEER_FAULT);
   if (i >= n) return;
   const float l = (float)losses_d[i];
   losses[i] = l;
   if (!isfinite(l)) atomicOr(status, ST_NONFINITE);
 }
-void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n, uint32_t* status) {
-  losses_refresh_kernel<<<(n + 63) / 64, 64, 0, st>>>(losses_d, losses, n, status);
+void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n,
+                           const double* fault_slot, uint32_t* status) {
+  losses_refresh_kernel<<<(n + 63) / 64, 64, 0, st>>>(losses_d, losses, n, fault_slot, status);
+}
+__global__ void fault_publish_kernel(const uint32_t* __restrict__ status, double* __restrict__ fault_slot) {
+  *fault_slot = *status != 0u ? 1.0 : 0.0;
+}
+void launch_fault_publish(cudaStream_t st, const uint32_t* status, double* fault_slot) {
+  fault_publish_kernel<<<1, 1, 0, st>>>(status, fault_slot);
 }
 
 void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,

@@ -73,6 +73,8 @@ struct GemmDesc {
   int split_units;
   int* extra_launches;          // incremented when the GEMM took a second launch (split K), or null
   int split_cap;                // > 0: upper bound on the number of K ranges per tile (1 = never split)
+  unsigned long long test_wait_ns;  // failure-detection tests only; > 0: the launch runs single-CTA, its bounded waits give
+                                // up after this many ns, and CTA 0 withholds one k-block so that a wait does run out
 };
 
 // --- elementwise / reduction kernels (bf = 1: bfloat16 tensors, 0: float) -------------------
@@ -138,7 +140,12 @@ struct UpdateDesc {
 // or lr == 0).  With write_g, block 0 also stores g[0..q).
 void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g);
-void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n, uint32_t* status);
+// After the exchange of a sharded step: fp32 copy of the completed loss array, finiteness check, and the
+// fault slot (sum over devices of 0/1 flags) folded into the local status word.
+void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n,
+                           const double* fault_slot, uint32_t* status);
+// End of a sharded step: *fault_slot = 1.0 when this device's status word is non-zero, else 0.0.
+void launch_fault_publish(cudaStream_t st, const uint32_t* status, double* fault_slot);
 void launch_perturbation(cudaStream_t st, uint64_t seed, uint32_t tensor, uint32_t query,
                          long long n, uint32_t* u32, float* z);
 

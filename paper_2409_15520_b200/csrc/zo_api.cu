@@ -32,6 +32,8 @@ inline int n_targets(const zo_config& c) {
   return ((c.lora_targets >> 0) & 1) + ((c.lora_targets >> 1) & 1) + ((c.lora_targets >> 2) & 1);
 }
 inline int row_pad(const zo_config& c) { return c.precision == ZO_BF16 ? 128 : 1; }
+// Queries a context runs in one step: all of them, or at most max_shard_q when it only ever runs shards.
+inline int run_q(const zo_config& c) { return c.max_shard_q > 0 ? c.max_shard_q : c.max_q; }
 
 // Returns ZO_OK or the reason the configuration cannot be run.
 zo_status check_config(const zo_config* c, char* err, size_t errn) {
@@ -49,6 +51,7 @@ zo_status check_config(const zo_config* c, char* err, size_t errn) {
     BAD(ZO_ERR_INVALID_ARG, "bad loss_kind");
   if (c->lora_rank < 1 || c->lora_rank > 64) BAD(ZO_ERR_INVALID_ARG, "lora_rank must be 1..64");
   if (c->max_q < 1 || c->max_q > ZO_MAX_Q) BAD(ZO_ERR_INVALID_ARG, "max_q must be 1..32");
+  if (c->max_shard_q < 0 || c->max_shard_q > c->max_q) BAD(ZO_ERR_INVALID_ARG, "max_shard_q must be 0..max_q");
   if (c->max_E < 1 || c->max_seq < 1) BAD(ZO_ERR_INVALID_ARG, "max_E and max_seq must be >= 1");
   if (c->d_model < 1) BAD(ZO_ERR_INVALID_ARG, "d_model must be >= 1");
   if (!isfinite(c->lora_scale)) BAD(ZO_ERR_INVALID_ARG, "lora_scale not finite");
@@ -91,10 +94,11 @@ Plan make_plan(const zo_config& c) {
   Plan p;
   memset(&p, 0, sizeof(p));
   const size_t es = c.precision == ZO_BF16 ? 2 : 4;
-  const size_t n = 2 * (size_t)c.max_q;
+  const size_t n = 2 * (size_t)c.max_q;                 // replicas of a whole step (loss arrays)
+  const size_t na = 2 * (size_t)run_q(c);               // replicas this context ever runs in one step
   const size_t Tm = (size_t)c.max_E * c.max_seq;
   const size_t Tp = up(Tm, row_pad(c));
-  const size_t Mp = n * Tp;
+  const size_t Mp = na * Tp;
   size_t off = 0;
   auto take = [&](size_t bytes) {
     const size_t o = off;
@@ -109,10 +113,10 @@ Plan make_plan(const zo_config& c) {
     p.tok_stage = take(Tm * c.d_model * es);          // host-variant staging of X
     p.lab_stage = take(Tm * c.d_out * 4);             // and of the targets
     p.rowloss = take(n * Tm * 8);
-    p.rowloss_pass = take(n * Tm * 8);
+    p.rowloss_pass = take(na * Tm * 8);
   } else {
     const size_t d = c.d_model, f = c.d_ffn, J = (size_t)n_targets(c) * c.lora_rank;
-    const size_t P = c.max_labelled, Mh = n * c.max_E * P;
+    const size_t P = c.max_labelled, Mh = na * c.max_E * P;
     p.h0 = take(Tp * d * es);
     p.x0 = take(Tp * d * es);
     p.qkv0 = take(Tp * 3 * d * es);
@@ -132,7 +136,7 @@ Plan make_plan(const zo_config& c) {
     p.pos = take(Tp * 4);
     p.xh = take(Mh * d * es);
     if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
-    p.rowloss = take(Mh * 8);
+    p.rowloss = take(n * c.max_E * P * 8);
     p.rowloss_pass = take(Mh * 8);
     if (c.weight_format != ZO_W_NATIVE) {   // one dequantised weight at a time
       size_t big = 3 * d * d;
@@ -142,7 +146,7 @@ Plan make_plan(const zo_config& c) {
     }
   }
   p.losses = take(n * 4);
-  p.losses_d = take(n * 8);
+  p.losses_d = take((n + 1) * 8);   // 2 max_q losses + the fault slot of a sharded step
   p.g = take((size_t)c.max_q * 4);
   p.status = take(256);
   if (c.precision == ZO_BF16) {             // split-K scratch of the tensor-core GEMM (small batches)
@@ -175,6 +179,7 @@ struct zo_ctx {
   int stepped, last_q, last_E, last_S;
   int schedule;
   int shard_begin, shard_count;    // queries this context computes in a step (count 0 = all of them)
+  unsigned long long test_wait_ns; // failure-detection test aid (zo_test_expire_wait), 0 = off
   char err[256];
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -224,6 +229,7 @@ zo_status run_gemm(zo_ctx* c, cudaStream_t st, int bf, uint32_t flags, const Gem
     Gt.cta_pair = (flags & ZO_FLAG_GEMM_PAIR) ? 1 : ((flags & ZO_FLAG_GEMM_SINGLE) ? 0 : 2);
     Gt.group_m = (int)((flags >> 8) & 0xFF);     // diagnostic: raster group override in bits 8..15
     Gt.split_cap = (int)((flags >> 16) & 0x1F);  // diagnostic: bound on the split-K factor in bits 16..20
+    Gt.test_wait_ns = c ? c->test_wait_ns : ((flags & ZO_FLAG_TEST_EXPIRE_WAIT) ? 1000000ull : 0ull);
     if (c && c->plan.split_ws) {
       Gt.split_ws = c->at<float>(c->plan.split_ws); Gt.split_units = SPLIT_UNITS; Gt.extra_launches = launches;
     }
@@ -348,6 +354,17 @@ void enqueue_update(zo_ctx* c, const zo_lora* lora, uint64_t seed, int q, float 
   }
 }
 
+// End of a step: projected gradients and ZO-SGD update of every B tensor; a sharded step stops at its
+// losses and publishes whether this device saw a fault in the slot that is exchanged with them.
+void finish_step(zo_ctx* c, const zo_lora* lora, uint64_t seed, int q, float eps, float lr) {
+  if (c->shard_count == 0) {
+    enqueue_update(c, lora, seed, q, eps, lr);
+    return;
+  }
+  PROF(PC_LOSS, 0.0, launch_fault_publish(c->st, c->at<uint32_t>(c->plan.status),
+                                          c->at<double>(c->plan.losses_d) + 2 * c->cfg.max_q));
+}
+
 zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const void* X,
                       const void* target, int T, uint64_t seed, int q, float eps, float lr) {
   const zo_config& cf = c->cfg;
@@ -388,7 +405,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss_pass));
   PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, nullptr, n, T, ps.base, ps.stride, rowloss, losses, losses_d, status));
   }
-  if (c->shard_count == 0) enqueue_update(c, lora, seed, q, eps, lr);
+  finish_step(c, lora, seed, q, eps, lr);
   return ZO_OK;
 }
 
@@ -549,8 +566,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, lab_val, n, EP, ps.base, ps.stride, rowloss, losses, losses_d, status));
   }  // passes
 
-  // projected gradients and ZO-SGD update of every B tensor (a sharded step stops at its losses)
-  if (c->shard_count == 0) enqueue_update(c, lora, seed, q, eps, lr);
+  finish_step(c, lora, seed, q, eps, lr);
 #undef GEMM
   return ZO_OK;
 }
@@ -593,9 +609,14 @@ zo_status begin_step(zo_ctx* c, int q) {
   c->launches = 0;
   if (c->shard_count && c->shard_begin + c->shard_count > q)
     return fail(c, ZO_ERR_INVALID_ARG, "query shard reaches past q");
+  if ((c->shard_count ? c->shard_count : q) > run_q(c->cfg))
+    return fail(c, ZO_ERR_INVALID_ARG, "more queries in one step than max_shard_q sized the workspace for");
   cudaError_t e = cudaMemsetAsync(c->at<uint32_t>(c->plan.status), 0, 4, c->st);
-  if (e == cudaSuccess && c->shard_count)
-    e = cudaMemsetAsync(c->at<double>(c->plan.losses_d), 0, (size_t)2 * c->cfg.max_q * 8, c->st);
+  if (e == cudaSuccess) {   // a sharded step zeroes the whole loss array; the fault slot is cleared by every step
+    double* ld = c->at<double>(c->plan.losses_d);
+    const size_t n = (size_t)2 * c->cfg.max_q;
+    e = c->shard_count ? cudaMemsetAsync(ld, 0, (n + 1) * 8, c->st) : cudaMemsetAsync(ld + n, 0, 8, c->st);
+  }
   if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "cudaMemsetAsync: %s", cudaGetErrorString(e));
   return ZO_OK;
 }
@@ -754,6 +775,8 @@ zo_status zo_losses(zo_ctx* ctx, float* host_losses, float* host_g) {
   if (st & (ST_BAD_LABELS | ST_BAD_TOKEN))
     return fail(ctx, ZO_ERR_INVALID_ARG, "token id or label out of range, or too many labelled positions");
   if (st & ST_NONFINITE) return fail(ctx, ZO_ERR_NONFINITE, "a replica loss is not finite; B left untouched");
+  if (st & ST_PEER_FAULT)
+    return fail(ctx, ZO_ERR_STATE, "another device of the sharded step reported a fault; no device applied the update");
   return ZO_OK;
 }
 
@@ -787,6 +810,13 @@ zo_status zo_set_schedule(zo_ctx* ctx, int32_t schedule) {
   return ZO_OK;
 }
 
+zo_status zo_test_expire_wait(zo_ctx* ctx, uint64_t wait_limit_ns) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (wait_limit_ns > 2000000000ull) return fail(ctx, ZO_ERR_INVALID_ARG, "wait limit above the regular 2 s");
+  ctx->test_wait_ns = wait_limit_ns;
+  return ZO_OK;
+}
+
 zo_status zo_set_query_shard(zo_ctx* ctx, int32_t q_begin, int32_t q_count) {
   if (!ctx) return ZO_ERR_INVALID_ARG;
   if (q_begin < 0 || q_count < 0 || (q_count == 0 && q_begin != 0) || q_begin + q_count > ctx->cfg.max_q)
@@ -800,7 +830,7 @@ zo_status zo_loss_buffer(zo_ctx* ctx, double** dev_losses, int32_t* host_capacit
   if (!ctx) return ZO_ERR_INVALID_ARG;
   if (!dev_losses) return fail(ctx, ZO_ERR_INVALID_ARG, "dev_losses is NULL");
   *dev_losses = ctx->at<double>(ctx->plan.losses_d);
-  if (host_capacity) *host_capacity = 2 * ctx->cfg.max_q;
+  if (host_capacity) *host_capacity = 2 * ctx->cfg.max_q + 1;
   return ZO_OK;
 }
 
@@ -815,7 +845,8 @@ zo_status zo_apply_update(zo_ctx* ctx, const zo_lora* lora, uint64_t seed, int32
     if (!lora->B[l]) return fail(ctx, ZO_ERR_INVALID_ARG, "null LoRA tensor");
   zo_ctx* c = ctx;
   PROF(PC_LOSS, 0.0, launch_losses_refresh(ctx->st, ctx->at<double>(ctx->plan.losses_d), ctx->at<float>(ctx->plan.losses),
-                                           2 * q, ctx->at<uint32_t>(ctx->plan.status)));
+                                           2 * q, ctx->at<double>(ctx->plan.losses_d) + 2 * ctx->cfg.max_q,
+                                           ctx->at<uint32_t>(ctx->plan.status)));
   enqueue_update(ctx, lora, seed, q, eps, lr);
   const cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return fail(ctx, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));

@@ -30,11 +30,23 @@ def exchange_losses(buf, q: int, group=None):
     return buf
 
 
+def exchange_step(buf, group=None):
+    """The exchange of a sharded step in one collective: the whole loss array of the library, i.e.
+    the 2 * max_q losses (zero outside each rank's block, also beyond 2q) and the fault slot at the
+    end, summed over ranks.  Afterwards every rank holds all losses and knows whether ANY rank saw a
+    device-side fault, so zo_apply_update skips the update everywhere or nowhere."""
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size(group) > 1:
+        dist.all_reduce(buf, op=dist.ReduceOp.SUM, group=group)
+    return buf
+
+
 def sharded_step(est, prob, E, S, seed, q, eps, lr, rank=None, world_size=None, group=None,
                  tokens=None, labels=None):
     """One step of Algorithm 1 with the q queries spread over the ranks of `group`.  Every rank
     passes the same batch, seed, q, eps and lr and holds identical B tensors before and after.
-    The collective runs on the current stream, which must be the estimator's."""
+    The collective runs on the current stream, which must be the estimator's.  The query shard is
+    switched off again before returning, so a later plain `est.step` is a whole step."""
     import torch.distributed as dist
     if world_size is None:
         world_size = dist.get_world_size(group) if dist.is_initialized() else 1
@@ -44,6 +56,9 @@ def sharded_step(est, prob, E, S, seed, q, eps, lr, rank=None, world_size=None, 
         raise ValueError("more ranks than queries: every rank needs at least one query of the step")
     begin, count = query_shard(q, world_size, rank)
     est.set_query_shard(begin, count)
-    est.step(prob, E, S, seed, q, eps, 0.0, tokens=tokens, labels=labels)
-    exchange_losses(est.loss_buffer(), q, group)
+    try:
+        est.step(prob, E, S, seed, q, eps, 0.0, tokens=tokens, labels=labels)
+    finally:
+        est.set_query_shard(0, 0)
+    exchange_step(est.loss_buffer(), group)
     est.apply_update(prob, seed, q, eps, lr)

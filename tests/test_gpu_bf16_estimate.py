@@ -26,12 +26,12 @@ SIMT, PAIR, LORA_EPI = 1, 2, 4
 SHAPE = dict(n_layers=3, d_model=256, n_heads=4, d_ffn=512, vocab=517, max_seq=128, lora_rank=8,
              E=2, S=128, q=3, n_labelled=6, lr=1e-2, bf16=True)
 EPS = 0.25
-# Measured on a B200 (all cases below): max_i |g_gpu_i - g_oracle_i| <= 0.05 max_i |g_oracle_i|;
-# the bound leaves a factor of about 2.  The error is absolute in nature, (loss rounding noise) /
+# Measured on a B200 (all cases below): max_i |g_gpu_i - g_oracle_i| between 0.002 and 0.015 of
+# max_i |g_oracle_i|; the bound leaves a factor of about 3.  The error is absolute in nature, (loss rounding noise) /
 # (2 eps), so it is stated against the largest |g_i| of the step, and every |g_i| used for the sign
 # check is required to stand above it.
-G_TOL = 0.10
-# fp32 arithmetic of the update kernel against the fp64 formula: about 1e-6 of the update
+G_TOL = 0.04
+# fp32 arithmetic of the update kernel against the fp64 formula: measured 0.7e-6 to 1.9e-6 of the update
 UPDATE_TOL = 1e-5
 
 

@@ -45,7 +45,8 @@ def test_opt125m_whole_step_bf16(opt125m):
 def test_opt125m_whole_step_fp32_mode(opt125m):
     """Same bf16-representable weights, fp32 activations and arithmetic, eps = 1e-3: the loss
     difference of a query is about 1e-5 of the loss, so g rests on the last digits of fp32 sums
-    through 12 blocks and a 50272-way softmax.  The measured discrepancy is printed."""
+    through 12 blocks and a 50272-way softmax.  Measured on a B200: losses 4e-8 relative, g 5e-4 of
+    max|g|, update 4e-4 of the update; the stated fp32 tolerances hold at the full configuration."""
     spec, p, seed, ref = opt125m
     got = run_gpu(spec, p, seed, precision=0)
     rel_l = np.max(np.abs(got["losses"] / ref["losses"] - 1))
@@ -55,7 +56,7 @@ def test_opt125m_whole_step_fp32_mode(opt125m):
           f"update err / update {upd:.2e}; g_gpu={got['g']} g_oracle={ref['g']}")
     assert rel_l < 1e-4
     assert rel_g < 1e-2
-    assert upd < 1e-2
+    assert upd < 1e-3
     assert update_from_gpu_g(spec, p, seed, got) < UPDATE_TOL
 
 

@@ -467,7 +467,7 @@ def test_argument_errors_are_reported_not_faulted():
 def test_decoder_fp32_at_the_configured_eps(arch):
     """The named configurations state eps = 1e-3 (the decoder cases above run the paper's MobiZO
     setting, 1e-2).  The loss difference of a query is then ten times smaller against the same fp32
-    rounding of the losses; the measured discrepancy of g is printed."""
+    rounding of the losses; measured on a B200: g within 5e-4 (OPT) and 6e-5 (Llama) of max|g|."""
     spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=False, lora_scale=2.0, **{**TINY, "eps": 1e-3})
     p, tok, lab = make_problem(spec, b_std=0.05)
     ref = run_oracle(spec, p, tok, lab, 11)
@@ -476,4 +476,4 @@ def test_decoder_fp32_at_the_configured_eps(arch):
     print(f"fp32 decoder arch={arch} eps=1e-3: max|dg|/max|g| = {rel_g:.2e}, update err {update_rel_err(spec, p, got['B'], ref['B']):.2e}")
     assert np.allclose(got["losses"], ref["losses"], rtol=1e-4, atol=0)
     assert rel_g < 1e-2
-    assert update_rel_err(spec, p, got["B"], ref["B"]) < 1e-2
+    assert update_rel_err(spec, p, got["B"], ref["B"]) < 1e-3

@@ -127,3 +127,74 @@ def test_nonfinite_loss_from_another_rank_blocks_the_update():
     assert ei.value.status == 6                             # ZO_ERR_NONFINITE
     assert np.array_equal(prob.B_numpy()[0], before)
     est.close()
+
+
+def test_fault_on_one_rank_blocks_the_update_on_every_rank():
+    """Two emulated ranks; rank 1 is given a token id outside the vocabulary.  Its status word travels
+    with the losses (the fault slot at the end of the loss array), so after the sum neither rank updates
+    its B: rank 1 reports its own fault, rank 0 that another device faulted."""
+    import torch
+    import paper_2409_15520_b200 as zo
+    spec = ModelSpec(arch=ARCH_LLAMA, bf16=False, n_layers=1, d_model=64, n_heads=2, d_ffn=96, vocab=101,
+                     max_seq=16, lora_rank=4, E=2, S=16, q=2, n_labelled=3, eps=1e-2, lr=1e-2)
+    p = make_decoder_problem(spec, seed=5, b_std=0.03)
+    ranks = []
+    for rank in range(2):
+        est, prob = zo.Estimator(zo.make_config(spec, max_shard_q=1)), zo.DeviceProblem(p, False)
+        est.set_query_shard(rank, 1)
+        tokens = prob.tokens.clone()
+        if rank == 1:
+            tokens[0, 3] = spec.vocab + 7
+        est.step(prob, spec.E, spec.S, 21, spec.q, spec.eps, 0.0, tokens=tokens)
+        ranks.append((est, prob))
+    torch.cuda.synchronize()
+    bufs = [est.loss_buffer() for est, _ in ranks]
+    assert bufs[0].numel() == 2 * spec.q + 1
+    assert bufs[0][-1].item() == 0.0 and bufs[1][-1].item() == 1.0
+    total = torch.stack(bufs).sum(0)                      # the all-reduce of the whole array
+    before = [prob.B_numpy() for _, prob in ranks]
+    codes = []
+    for (est, prob), buf in zip(ranks, bufs):
+        buf.copy_(total)
+        est.apply_update(prob, 21, spec.q, spec.eps, spec.lr)
+        with pytest.raises(zo.ZoError) as ei:
+            est.losses()
+        codes.append(ei.value.status)
+    assert codes == [7, 1]                                # ZO_ERR_STATE (peer fault), ZO_ERR_INVALID_ARG (own)
+    for (est, prob), b0 in zip(ranks, before):
+        assert all(np.array_equal(a, b) for a, b in zip(prob.B_numpy(), b0))
+        est.close()
+
+
+def test_shard_sized_workspace_and_reset_after_a_sharded_step():
+    """max_shard_q sizes the activation workspace for the shard alone (half the replicas here); the step
+    helper leaves the context unsharded, and a whole step is then refused by a context sized for shards."""
+    import ctypes as C
+    import paper_2409_15520_b200 as zo
+    from paper_2409_15520_b200 import binding as b
+    spec = ModelSpec(arch=ARCH_OPT, tie_lm_head=True, bf16=True, n_layers=2, d_model=256, n_heads=4, d_ffn=512,
+                     vocab=777, max_seq=96, lora_rank=8, E=4, S=96, q=4, n_labelled=6, eps=1e-2, lr=1e-2)
+    full, half = zo.make_config(spec), zo.make_config(spec, max_shard_q=2)
+    nb_full, nb_half = b.zo_workspace_bytes(C.byref(full)), b.zo_workspace_bytes(C.byref(half))
+    assert nb_half < 0.62 * nb_full
+    p = make_decoder_problem(spec, seed=5, b_std=0.03)
+    whole = run_gpu(spec, p, 21)
+    est, prob = zo.Estimator(half), zo.DeviceProblem(p, True)
+    # world size 1 with an explicit block: rank 0 of 2 runs queries 0..1, "receives" the rest from a full run
+    est.set_query_shard(0, 2)
+    est.step(prob, spec.E, spec.S, 21, spec.q, spec.eps, 0.0)
+    est.set_query_shard(0, 0)
+    buf = est.loss_buffer()
+    assert np.array_equal(buf[:4].cpu().numpy().astype(np.float32).astype(np.float64), whole["losses"][:4])
+    assert np.all(buf[4:].cpu().numpy() == 0.0)
+    with pytest.raises(zo.ZoError) as ei:                 # 4 queries in one step do not fit this workspace
+        est.step(prob, spec.E, spec.S, 21, spec.q, spec.eps, 0.0)
+    assert ei.value.status == 1
+    est.close()
+    est2, prob2 = zo.Estimator(full), zo.DeviceProblem(p, True)
+    zo.sharded_step(est2, prob2, spec.E, spec.S, 21, spec.q, spec.eps, spec.lr, rank=0, world_size=1)
+    est2.step(prob2, spec.E, spec.S, 22, spec.q, spec.eps, 0.0)   # a plain step afterwards is a whole step
+    l2, _ = est2.losses()
+    assert np.all(l2 != 0.0)
+    assert all(np.array_equal(a, b_) for a, b_ in zip(prob2.B_numpy(), whole["B"]))
+    est2.close()
