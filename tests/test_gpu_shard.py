@@ -176,7 +176,8 @@ def test_shard_sized_workspace_and_reset_after_a_sharded_step():
                      vocab=777, max_seq=96, lora_rank=8, E=4, S=96, q=4, n_labelled=6, eps=1e-2, lr=1e-2)
     full, half = zo.make_config(spec), zo.make_config(spec, max_shard_q=2)
     nb_full, nb_half = b.zo_workspace_bytes(C.byref(full)), b.zo_workspace_bytes(C.byref(half))
-    assert nb_half < 0.62 * nb_full
+    # the replicated activations (hidden, normed, q|k|v, MLP) of the 4 replicas no longer provided for
+    assert nb_full - nb_half > 4 * 384 * (5 * 256 + 512) * 2
     p = make_decoder_problem(spec, seed=5, b_std=0.03)
     whole = run_gpu(spec, p, 21)
     est, prob = zo.Estimator(half), zo.DeviceProblem(p, True)
