@@ -295,6 +295,57 @@ ZO_API zo_status zo_loss_buffer(zo_ctx* ctx, double** dev_losses, int32_t* host_
 ZO_API zo_status zo_apply_update(zo_ctx* ctx, const zo_lora* lora, uint64_t seed, int32_t q,
                                  float eps, float lr);
 
+/* ---------------------------------------------------------------------------------------------------
+ * The step in the form of the paper's Algorithm 2 ("Mobile MP-LoRA Module", q = 1).
+ *
+ * Algorithm 2 keeps, per trainable tensor, the two perturbed copies B[0] = B + eps z and B[1] = B - eps z
+ * in memory instead of the master copy, takes the projected gradient g of the PREVIOUS step as an input
+ * of the forward pass, and does inside that pass:
+ *     diff = (B[0] - B[1]) / 2;  update = eta g diff / eps;  z = eps randn_like(B[0]);
+ *     B[0] = B[0] - diff - update + z;  B[1] = B[1] + diff - update - z;
+ *     output = x W + bmm(x A, B)
+ * so that nothing but forward passes ever runs: the previous update and the new perturbation ride in
+ * the forward pass, and no host round trip separates two steps.
+ *
+ *   zo_lora_pair.B_pair[l] : float32 [2, n_targets, r, k_out] of layer l, B[0] then B[1]; UPDATED IN
+ *       PLACE by every zo_step_pair.  Before the first step both halves hold the same B (diff = 0).
+ *   zo_step_pair(ctx, weights, pair, tokens, labels, E, S, seed, dev_g_prev, eps, lr)
+ *       One step: applies the lines above to every pair of the model (z = eps * the normals of
+ *       (seed, tensor, query 0), the stream of zo_step), runs the forward pass of the two replicas on
+ *       the stored pair, and leaves the two losses and g = (l0 - l1) / (2 eps) on the device.
+ *       dev_g_prev: DEVICE pointer to the previous step's g (the buffer zo_g_buffer returns, which
+ *       this call overwrites at its end, or any device float), or NULL for g = 0 (first step).
+ *       Asynchronous; steps can be enqueued back to back without reading anything back.  A step that
+ *       faults on the device (status word set) leaves g = 0, so the next step's update is a no-op.
+ *       eps must be > 0.  zo_losses returns the two losses and g as after zo_step with q = 1.
+ *       The mean (B[0] + B[1]) / 2 after the call is the master copy BEFORE this step's own update
+ *       (which the next call applies): it equals the B that zo_step would hold at the same point.
+ *   zo_pair_collapse(ctx, pair, dev_g_prev, eps, lr)
+ *       Applies the pending update without a new perturbation: B[0] = B[1] = the updated master copy
+ *       (to finish a run, or to hand the tensors to zo_step).
+ *   zo_g_buffer(ctx, &dev_g, &capacity)
+ *       Device address of the context's projected gradients (float32 [max_q]; entry 0 after a pair step).
+ *   zo_mp_lora_linear_pair(...)
+ *       The module of Algorithm 2 on its own: the lines above on one stored pair (g_prev by value),
+ *       then Y[n] = X[n or shared] W^T + bias + scale (X A^T) B[n], n = 0, 1.  Arguments as
+ *       zo_mp_lora_linear with q = 1; B_pair is float32 [2, r, k_out], updated in place. */
+typedef struct zo_lora_pair {
+  const void* const* A;      /* HOST array [n_layers] of device pointers, as zo_lora.A */
+  float* const* B_pair;      /* HOST array [n_layers] of device pointers to [2, n_targets, r, k_out] */
+} zo_lora_pair;
+ZO_API zo_status zo_step_pair(zo_ctx* ctx, const zo_weights* weights, const zo_lora_pair* pair,
+                              const void* tokens, const void* labels, int32_t E, int32_t S, uint64_t seed,
+                              const float* dev_g_prev, float eps, float lr);
+ZO_API zo_status zo_pair_collapse(zo_ctx* ctx, const zo_lora_pair* pair, const float* dev_g_prev, float eps,
+                                  float lr);
+ZO_API zo_status zo_g_buffer(zo_ctx* ctx, float** dev_g, int32_t* host_capacity);
+ZO_API zo_status zo_mp_lora_linear_pair(void* cuda_stream, int32_t precision, const void* X, const void* W,
+                                        const void* bias, const void* A, float* B_pair, void* Y, int32_t T,
+                                        int32_t k_in, int32_t k_out, int32_t r, float scale, uint64_t seed,
+                                        uint32_t tensor_id, float g_prev, float eps, float lr,
+                                        int32_t x_replicated, void* scratch, size_t scratch_bytes,
+                                        uint32_t flags);
+
 /* Failure-detection test aid; off (0) by default and in every measured run.  Every device-side wait of
  * the tensor-core GEMM (on a shared-memory barrier that a copy or a tensor-core instruction completes) is
  * bounded: when it runs out, the thread block raises the time-out bit of the status word, lets the copies

@@ -7,6 +7,6 @@ has not been built (``python paper_2409_15520_b200/build.py``).
 """
 from .binding import (  # noqa: F401
     LIB, ZoConfig, ZoError, Estimator, DeviceProblem, make_config, perturbation,
-    mp_lora_linear, mp_lora_linear_static, STATUS_NAMES,
+    mp_lora_linear, mp_lora_linear_static, mp_lora_linear_pair, STATUS_NAMES,
 )
 from .sharding import query_shard, exchange_losses, exchange_step, sharded_step  # noqa: F401

@@ -60,6 +60,10 @@ class ZoLora(C.Structure):
     _fields_ = [("A", C.POINTER(C.c_void_p)), ("B", C.POINTER(C.c_void_p))]
 
 
+class ZoLoraPair(C.Structure):
+    _fields_ = [("A", C.POINTER(C.c_void_p)), ("B_pair", C.POINTER(C.c_void_p))]
+
+
 def _sig(name, res, args):
     f = getattr(LIB, name)
     f.restype, f.argtypes = res, args
@@ -81,6 +85,16 @@ zo_row_losses = _sig("zo_row_losses", C.c_int, [C.c_void_p, C.c_void_p, C.POINTE
 zo_launch_count = _sig("zo_launch_count", C.c_int32, [C.c_void_p])
 zo_set_schedule = _sig("zo_set_schedule", C.c_int, [C.c_void_p, C.c_int32])
 zo_set_query_shard = _sig("zo_set_query_shard", C.c_int, [C.c_void_p, C.c_int32, C.c_int32])
+zo_step_pair = _sig("zo_step_pair", C.c_int, [C.c_void_p, C.POINTER(ZoWeights), C.POINTER(ZoLoraPair), C.c_void_p,
+                                              C.c_void_p, C.c_int32, C.c_int32, C.c_uint64, C.c_void_p, C.c_float,
+                                              C.c_float])
+zo_pair_collapse = _sig("zo_pair_collapse", C.c_int, [C.c_void_p, C.POINTER(ZoLoraPair), C.c_void_p, C.c_float,
+                                                      C.c_float])
+zo_g_buffer = _sig("zo_g_buffer", C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32)])
+zo_mp_lora_linear_pair = _sig("zo_mp_lora_linear_pair", C.c_int, [
+    C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+    C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_uint64, C.c_uint32, C.c_float, C.c_float,
+    C.c_float, C.c_int32, C.c_void_p, C.c_size_t, C.c_uint32])
 zo_test_expire_wait = _sig("zo_test_expire_wait", C.c_int, [C.c_void_p, C.c_uint64])
 zo_loss_buffer = _sig("zo_loss_buffer", C.c_int, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_int32)])
 zo_apply_update = _sig("zo_apply_update", C.c_int, [C.c_void_p, C.POINTER(ZoLora), C.c_uint64, C.c_int32,
@@ -203,6 +217,21 @@ class DeviceProblem:
         self._keep.append(t)
         return t
 
+    def make_pair(self):
+        """The trainable tensors in the stored-pair form of Algorithm 2: per layer a float32 tensor
+        [2, ...] whose two halves both start as the current B.  Returns the zo_lora_pair structure;
+        the tensors are kept in self.B_pair."""
+        self.B_pair = [torch.stack([b, b]).contiguous() if b is not None else None for b in self.B]
+        self._Parr = (C.c_void_p * len(self.B_pair))(*[(t.data_ptr() if t is not None else None)
+                                                       for t in self.B_pair])
+        self.pair = ZoLoraPair()
+        self.pair.A = C.cast(self._Aarr, C.POINTER(C.c_void_p))
+        self.pair.B_pair = C.cast(self._Parr, C.POINTER(C.c_void_p))
+        return self.pair
+
+    def pair_numpy(self):
+        return [t.detach().cpu().numpy().astype(np.float64) if t is not None else None for t in self.B_pair]
+
     def B_numpy(self):
         return [b.detach().cpu().numpy().astype(np.float64) if b is not None else None
                 for b in self.B]
@@ -272,6 +301,26 @@ class Estimator:
         """Later steps run only the queries [q_begin, q_begin + q_count) and stop at their losses
         (q_count = 0: whole steps again)."""
         self._check(zo_set_query_shard(self._h, q_begin, q_count))
+
+    def step_pair(self, prob: DeviceProblem, E, S, seed, g_prev, eps, lr, tokens=None, labels=None):
+        """One step in the stored-pair form (Algorithm 2, q = 1) on prob.pair (see make_pair);
+        g_prev is a device float tensor holding the previous step's g (e.g. g_buffer()) or None."""
+        tok = prob.tokens if tokens is None else tokens
+        lab = prob.labels if labels is None else labels
+        self._check(zo_step_pair(self._h, C.byref(prob.weights), C.byref(prob.pair), _ptr(tok), _ptr(lab),
+                                 E, S, seed, _ptr(g_prev), eps, lr))
+        self.q = 1
+
+    def pair_collapse(self, prob: DeviceProblem, g_prev, eps, lr):
+        self._check(zo_pair_collapse(self._h, C.byref(prob.pair), _ptr(g_prev), eps, lr))
+
+    def g_buffer(self):
+        """The context's projected gradients [max_q] as a float32 tensor aliasing the workspace."""
+        ptr, cap = C.c_void_p(), C.c_int32()
+        self._check(zo_g_buffer(self._h, C.byref(ptr), C.byref(cap)))
+        off = ptr.value - self.workspace.data_ptr()
+        assert off % 4 == 0 and 0 <= off and off + 4 * cap.value <= self.workspace.numel()
+        return self.workspace[off:off + 4 * cap.value].view(torch.float32)
 
     def test_expire_wait(self, wait_limit_ns):
         """Failure-detection test aid: bounded waits of the tensor-core GEMM give up after
@@ -357,6 +406,28 @@ def mp_lora_linear(X, W, bias, A, B, T, q, scale, seed, tensor_id, eps, x_replic
         status = int(scratch.view(torch.int32)[(base - scratch.data_ptr()) // 4].item())
         if status:
             raise ZoError(5, f"device status word {status}")
+    return Y
+
+
+def mp_lora_linear_pair(X, W, bias, A, B_pair, T, scale, seed, tensor_id, g_prev, eps, lr, x_replicated, flags=0):
+    """The module of Algorithm 2 on its own: updates the stored pair B_pair [2, r, k_out] in place
+    (previous update from g_prev, new perturbation from the seed) and returns Y [2, T, k_out]."""
+    bf = X.dtype == torch.bfloat16
+    k_out, k_in = W.shape
+    r = A.shape[0]
+    Y = torch.empty((2, T, k_out), dtype=X.dtype, device=X.device)
+    nb = zo_mp_lora_scratch_bytes(int(bf), T, k_in, k_out, r, 1, int(x_replicated))
+    scratch = torch.empty(nb + 256, dtype=torch.uint8, device=X.device)
+    base = (scratch.data_ptr() + 255) // 256 * 256
+    st = zo_mp_lora_linear_pair(C.c_void_p(torch.cuda.current_stream().cuda_stream), int(bf), _ptr(X), _ptr(W),
+                                _ptr(bias), _ptr(A), _ptr(B_pair), _ptr(Y), T, k_in, k_out, r, scale, seed,
+                                tensor_id, g_prev, eps, lr, int(x_replicated), C.c_void_p(base), nb, flags)
+    if st:
+        raise ZoError(st, "zo_mp_lora_linear_pair")
+    torch.cuda.synchronize()
+    status = int(scratch.view(torch.int32)[(base - scratch.data_ptr()) // 4].item())
+    if status:
+        raise ZoError(5, f"device status word {status}")
     return Y
 
 

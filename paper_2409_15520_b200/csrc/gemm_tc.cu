@@ -38,6 +38,7 @@
 
 #include "common.cuh"
 #include "kernels.h"
+#include "lora_operand.cuh"
 
 namespace zo {
 
@@ -527,8 +528,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (slot < 0 || g_tile % ksplit != 0) return;  // uniform over the CTA (same decision as the MMA warp's)
       const int sec = n0g / P.L.width, cs = n0g - sec * P.L.width;
       const int repg = P.L.rep_base + P.L.rep_stride * ((tm * TILE_M) / P.L.rows_per_replica);
-      const float sz = ((repg & 1) ? -P.L.eps : P.L.eps) * P.L.scale;
-      const float* Bm = P.L.B + (size_t)slot * P.L.r * P.L.width;
       const int kgroups = (P.L.r + 7) / 8;
       constexpr int CQ = PAIR ? 32 : 64;               // column quads of the operand rows this CTA holds
       for (int unit_i = et; unit_i < CQ * kgroups; unit_i += EP_THREADS) {
@@ -539,13 +538,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int kk = 0; kk < 8; ++kk) {
           const int k = k0 + kk;
           float4 b = make_float4(0.f, 0.f, 0.f, 0.f), z = b;
-          if (k < P.L.r) {
-            const size_t e = (size_t)k * P.L.width + cs + c4;
-            b = *reinterpret_cast<const float4*>(Bm + e);
-            if (P.L.eps != 0.f) z = z_block(P.L.seed, P.L.tensor_base + slot, (uint32_t)(repg >> 1), (uint32_t)(e >> 2));
-          }
+          if (k < P.L.r) lora_operand(P.L, slot, (size_t)k * P.L.width + cs + c4, repg, b, z);
           bb[kk][0] = b.x * P.L.scale; bb[kk][1] = b.y * P.L.scale; bb[kk][2] = b.z * P.L.scale; bb[kk][3] = b.w * P.L.scale;
-          zz[kk][0] = z.x * sz; zz[kk][1] = z.y * sz; zz[kk][2] = z.z * sz; zz[kk][3] = z.w * sz;
+          zz[kk][0] = z.x * P.L.scale; zz[kk][1] = z.y * P.L.scale; zz[kk][2] = z.z * P.L.scale; zz[kk][3] = z.w * P.L.scale;
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -657,7 +652,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int rrow = P.res ? (P.res_mod > 0 ? row % P.res_mod : row) : 0;
       // per-tile LoRA constants: all rows of the tile belong to one replica
       const int rep = P.has_lora ? P.L.rep_base + P.L.rep_stride * (m0 / P.L.rows_per_replica) : 0;
-      const float sgn = (rep & 1) ? -P.L.eps : P.L.eps;
       const float* urow = P.has_lora ? P.L.U + (size_t)min(row, P.M - 1) * P.L.ldu : nullptr;
       const bool u_vec = P.has_lora && (P.L.ldu % 4 == 0) && (P.L.r % 4 == 0) && (((uintptr_t)P.L.U & 15) == 0);
       const int nchunk = ncol_tile / 32;
@@ -741,14 +735,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                   const int sec = col / P.L.width;
                   const int slot = P.L.slot_of_sec[sec];
                   if (slot >= 0) {
-                    const size_t e = (size_t)k * P.L.width + (col - sec * P.L.width);
-                    b = *reinterpret_cast<const float4*>(P.L.B + (size_t)slot * P.L.r * P.L.width + e);
-                    if (P.L.eps != 0.f) {
-                      const float4 z = z_block(P.L.seed, P.L.tensor_base + slot, (uint32_t)(rep >> 1),
-                                               (uint32_t)(e >> 2));
-                      b.x = fmaf(sgn, z.x, b.x); b.y = fmaf(sgn, z.y, b.y);
-                      b.z = fmaf(sgn, z.z, b.z); b.w = fmaf(sgn, z.w, b.w);
-                    }
+                    b = lora_replica_b(P.L, slot, (size_t)k * P.L.width + (col - sec * P.L.width), rep);
                     b.x *= P.L.scale; b.y *= P.L.scale; b.z *= P.L.scale; b.w *= P.L.scale;
                   }
                 }

@@ -1,6 +1,7 @@
 // Bandwidth-bound and small kernels of the perturbed forward, the losses and the update.
 #include "common.cuh"
 #include "kernels.h"
+#include "lora_operand.cuh"
 
 namespace zo {
 
@@ -393,20 +394,11 @@ lora_apply_kernel(const T* base, int ldb, int base_shared, T* out, int ldo, int 
   const int ncols = min(LA_COLS, L.width - cc_t);
   if (slot >= 0) {
     const int rid = L.rep_base + L.rep_stride * n;    // replica id within the step
-    const float sgn = (rid & 1) ? -L.eps : L.eps;
-    const uint32_t query = (uint32_t)(rid >> 1);
-    const float* Bs = L.B + (size_t)slot * L.r * L.width;
     for (int i = threadIdx.x; i < L.r * (LA_COLS / 4); i += blockDim.x) {
       const int k = i / (LA_COLS / 4), c4 = (i % (LA_COLS / 4)) * 4;
       float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
       if (c4 < ncols) {
-        const size_t e = (size_t)k * L.width + cc_t + c4;
-        v = *reinterpret_cast<const float4*>(Bs + e);
-        if (L.eps != 0.f) {
-          const float4 z = z_block(L.seed, L.tensor_base + slot, query, (uint32_t)(e >> 2));
-          v.x = fmaf(sgn, z.x, v.x); v.y = fmaf(sgn, z.y, v.y);
-          v.z = fmaf(sgn, z.z, v.z); v.w = fmaf(sgn, z.w, v.w);
-        }
+        v = lora_replica_b(L, slot, (size_t)k * L.width + cc_t + c4, rid);
         v.x *= L.scale; v.y *= L.scale; v.z *= L.scale; v.w *= L.scale;
       }
       *reinterpret_cast<float4*>(sB + k * LA_COLS + c4) = v;
@@ -1005,6 +997,57 @@ __global__ void fault_publish_kernel(const uint32_t* __restrict__ status, double
 }
 void launch_fault_publish(cudaStream_t st, const uint32_t* status, double* fault_slot) {
   fault_publish_kernel<<<1, 1, 0, st>>>(status, fault_slot);
+}
+
+// =========================================================================================
+// Stored-pair form of the trainable tensors (Algorithm 2, "Mobile MP-LoRA", q = 1): B[0] = B + eps z
+// and B[1] = B - eps z live in memory.  At the start of a forward pass the previous step's update and
+// the new perturbation are applied to both, in the algorithm's order of operations:
+//   diff = (B[0] - B[1]) / 2;  update = eta g diff / eps;  z = eps randn;
+//   B[0] = B[0] - diff - update + z;  B[1] = B[1] + diff - update - z.
+// g is the previous step's projected gradient (device pointer, or a value).  draw = 0 leaves z = 0:
+// both tensors end at the updated master copy.
+// =========================================================================================
+__global__ void pair_update_kernel(UpdateDesc D, long long pair_stride, const float* __restrict__ g_dev,
+                                   float g_val, float eps, float lr, uint64_t seed, int draw) {
+  const long long blk = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long e = blk * 4;
+  if (e >= D.elems_per_slot) return;
+  const int slot = blockIdx.y, li = blockIdx.z;
+  const float g = g_dev ? *g_dev : g_val;
+  float* p0 = D.B[li] + (size_t)slot * D.elems_per_slot + e;
+  float* p1 = p0 + pair_stride;
+  float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (draw) {
+    const float4 n4 = z_block(seed, D.tensor_base[li] + slot, 0u, (uint32_t)blk);
+    z = make_float4(eps * n4.x, eps * n4.y, eps * n4.z, eps * n4.w);
+  }
+  const float zz[4] = {z.x, z.y, z.z, z.w};
+  const long long left = D.elems_per_slot - e;
+  for (int j = 0; j < 4 && j < left; ++j) {
+    const float b0 = p0[j], b1 = p1[j];
+    const float diff = (b0 - b1) / 2.f;
+    const float update = lr * g * diff / eps;
+    p0[j] = b0 - diff - update + zz[j];
+    p1[j] = b1 + diff - update - zz[j];
+  }
+}
+void launch_pair_update(cudaStream_t st, const UpdateDesc& D, long long pair_stride, const float* g_dev,
+                        float g_val, float eps, float lr, uint64_t seed, int draw) {
+  const long long blks = (D.elems_per_slot + 3) / 4;
+  if (blks <= 0 || D.count <= 0 || D.n_slots <= 0) return;
+  dim3 grid((unsigned)((blks + 127) / 128), D.n_slots, D.count);
+  pair_update_kernel<<<grid, 128, 0, st>>>(D, pair_stride, g_dev, g_val, eps, lr, seed, draw);
+}
+// Projected gradient of a stored-pair step, kept on the device for the next step's forward:
+// g = (l0 - l1) / (2 eps), or 0 when the step faulted (its update is then a no-op).
+__global__ void pair_g_kernel(const double* __restrict__ losses, float* __restrict__ g, float eps,
+                              const uint32_t* __restrict__ status) {
+  const float v = (float)((losses[0] - losses[1]) / (2.0 * (double)eps));
+  g[0] = (*status == 0u && isfinite(v)) ? v : 0.f;
+}
+void launch_pair_g(cudaStream_t st, const double* losses, float* g, float eps, const uint32_t* status) {
+  pair_g_kernel<<<1, 1, 0, st>>>(losses, g, eps, status);
 }
 
 void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses, float* g, int q,

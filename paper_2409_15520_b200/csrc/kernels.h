@@ -9,7 +9,9 @@ namespace zo {
 struct LoraDesc {
   const float* U;        // [rows, ldu] fp32 down-projections X A^T, row-indexed like the X operand
   int ldu;
-  const float* B;        // [n_slots, r, width] fp32 master copy of this layer
+  const float* B;        // [n_slots, r, width] fp32 master copy of this layer (stored pair: B[0] = B + eps z)
+  const float* B1;       // null, or the second tensor of a stored pair (B[1] = B - eps z): replica n then uses
+                         // the stored B[n & 1] and nothing is regenerated (Algorithm 2, q = 1)
   int r;
   int width;             // k_out of one section
   int slot_of_sec[3];    // output columns [j*width, (j+1)*width) -> slot, or -1 (not adapted)
@@ -142,6 +144,13 @@ void launch_zo_update(cudaStream_t st, const UpdateDesc& D, const double* losses
                       float eps, float lr, uint64_t seed, const uint32_t* status, int write_g);
 // After the exchange of a sharded step: fp32 copy of the completed loss array, finiteness check, and the
 // fault slot (sum over devices of 0/1 flags) folded into the local status word.
+// Stored-pair form (Algorithm 2): D.B[i] points at B[0] of tensor group i, B[1] lies pair_stride floats
+// further.  Applies the previous step's update (g from g_dev if non-null, else g_val) and, with draw != 0,
+// the new perturbation eps z of query 0 to both tensors.
+void launch_pair_update(cudaStream_t st, const UpdateDesc& D, long long pair_stride, const float* g_dev,
+                        float g_val, float eps, float lr, uint64_t seed, int draw);
+// g[0] = (losses[0] - losses[1]) / (2 eps), or 0 when the status word is set.
+void launch_pair_g(cudaStream_t st, const double* losses, float* g, float eps, const uint32_t* status);
 void launch_losses_refresh(cudaStream_t st, const double* losses_d, float* losses, int n,
                            const double* fault_slot, uint32_t* status);
 // End of a sharded step: *fault_slot = 1.0 when this device's status word is non-zero, else 0.0.

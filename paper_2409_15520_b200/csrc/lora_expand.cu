@@ -10,6 +10,7 @@
 // shared memory as 16 bytes per lane on contiguous row segments.  Sections that carry
 // no adapter are copied through the same pipeline.
 #include "kernels.h"
+#include "lora_operand.cuh"
 #include "mma.cuh"
 
 namespace zo {
@@ -61,20 +62,15 @@ lora_expand_kernel(const bf16* __restrict__ base, int ldb, bf16* __restrict__ ou
     for (int i = threadIdx.x; i < XT * LDB / 8; i += 256) reinterpret_cast<uint4*>(Bs)[i] = make_uint4(0, 0, 0, 0);
     __syncthreads();
     const int rid = L.rep_base + L.rep_stride * n;     // replica id within the step
-    const float sz = ((rid & 1) ? -L.eps : L.eps) * L.scale;
-    const uint32_t query = (uint32_t)(rid >> 1);
-    const float* Bm = L.B + (size_t)slot * r * L.width;
     for (int i = threadIdx.x; i < r * (XT / 4); i += 256) {
       const int k = i / (XT / 4), c4 = (i % (XT / 4)) * 4;
-      const size_t e = (size_t)k * L.width + cs + c4;
-      const float4 b = *reinterpret_cast<const float4*>(Bm + e);
-      float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (L.eps != 0.f) z = z_block(L.seed, L.tensor_base + slot, query, (uint32_t)(e >> 2));
+      float4 b, z;
+      lora_operand(L, slot, (size_t)k * L.width + cs + c4, rid, b, z);
       const float bb[4] = {b.x, b.y, b.z, b.w}, zz[4] = {z.x, z.y, z.z, z.w};
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         Bs[(c4 + j) * LDB + k] = __float2bfloat16_rn(bb[j] * L.scale);
-        Bs[(c4 + j) * LDB + r + k] = __float2bfloat16_rn(zz[j] * sz);
+        Bs[(c4 + j) * LDB + r + k] = __float2bfloat16_rn(zz[j] * L.scale);
       }
     }
     __syncthreads();                                   // operand complete: the only CTA-wide hand-over

@@ -180,6 +180,7 @@ struct zo_ctx {
   int schedule;
   int shard_begin, shard_count;    // queries this context computes in a step (count 0 = all of them)
   unsigned long long test_wait_ns; // failure-detection test aid (zo_test_expire_wait), 0 = off
+  int pair_mode;                   // the running step uses the stored +/- pair of Algorithm 2 (lora->B[l] = the pair)
   char err[256];
   template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -357,6 +358,11 @@ void enqueue_update(zo_ctx* c, const zo_lora* lora, uint64_t seed, int q, float 
 // End of a step: projected gradients and ZO-SGD update of every B tensor; a sharded step stops at its
 // losses and publishes whether this device saw a fault in the slot that is exchanged with them.
 void finish_step(zo_ctx* c, const zo_lora* lora, uint64_t seed, int q, float eps, float lr) {
+  if (c->pair_mode) {   // Algorithm 2: g stays on the device as the next forward pass's input; no update here
+    PROF(PC_UPDATE, 0.0, launch_pair_g(c->st, c->at<double>(c->plan.losses_d), c->at<float>(c->plan.g), eps,
+                                       c->at<uint32_t>(c->plan.status)));
+    return;
+  }
   if (c->shard_count == 0) {
     enqueue_update(c, lora, seed, q, eps, lr);
     return;
@@ -394,6 +400,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   if (s) return s;
   LoraDesc L{};
   L.U = U; L.ldu = r; L.B = lora->B[0]; L.r = r; L.width = ko;
+  L.B1 = c->pair_mode ? L.B + (size_t)r * ko : nullptr;
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
   L.rep_base = ps.base; L.rep_stride = ps.stride;
@@ -468,6 +475,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, hin, xn, W.norm1_g, W.norm1_b, rows, d, cf.norm_eps, nullptr, 0, 0));
     LoraDesc L{};
     L.U = U; L.ldu = J; L.B = J ? lora->B[l] : nullptr; L.r = r; L.width = d;
+    L.B1 = (J && c->pair_mode) ? L.B + (size_t)nt * r * d : nullptr;
     for (int j = 0; j < 3; ++j) L.slot_of_sec[j] = c->slot_of_sec[j];
     L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = (uint32_t)(l * nt);
     L.rows_per_replica = Tp;
@@ -920,8 +928,12 @@ size_t zo_mp_lora_scratch_bytes(int32_t precision, int32_t T, int32_t k_in, int3
   return b;
 }
 
-zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X, const void* W,
-                            const void* bias, const void* A, const float* B, void* Y, int32_t T,
+}  // extern "C"
+
+// The layer with either storage form of B: B1 == null is the master-copy form (z regenerated), otherwise
+// (B, B1) is a stored pair and q must be 1.
+static zo_status mp_lora_linear_impl(void* cuda_stream, int32_t precision, const void* X, const void* W,
+                            const void* bias, const void* A, const float* B, const float* B1, void* Y, int32_t T,
                             int32_t k_in, int32_t k_out, int32_t r, float scale, uint64_t seed,
                             uint32_t tensor_id, int32_t q, float eps, int32_t x_replicated,
                             void* scratch, size_t scratch_bytes, uint32_t flags) {
@@ -949,7 +961,7 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
   void* pack = (uint8_t*)base + (x_replicated ? 0 : up((size_t)T * k_out * (bf ? 2 : 4), 256));
   if (cudaMemsetAsync(status, 0, 4, st) != cudaSuccess) return ZO_ERR_CUDA;
   LoraDesc L{};
-  L.U = U; L.ldu = r; L.B = B; L.r = r; L.width = k_out;
+  L.U = U; L.ldu = r; L.B = B; L.B1 = B1; L.r = r; L.width = k_out;
   L.slot_of_sec[0] = 0; L.slot_of_sec[1] = L.slot_of_sec[2] = -1;
   L.scale = scale; L.eps = eps; L.seed = seed; L.tensor_base = tensor_id; L.rows_per_replica = T;
   L.rep_base = 0; L.rep_stride = 1;
@@ -985,6 +997,124 @@ zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X,
     launch_lora_apply(st, bf, Y, k_out, 0, Y, k_out, n, T, L, 1);
   }
   return cudaGetLastError() == cudaSuccess ? ZO_OK : ZO_ERR_CUDA;
+}
+
+extern "C" {
+
+zo_status zo_mp_lora_linear(void* cuda_stream, int32_t precision, const void* X, const void* W,
+                            const void* bias, const void* A, const float* B, void* Y, int32_t T,
+                            int32_t k_in, int32_t k_out, int32_t r, float scale, uint64_t seed,
+                            uint32_t tensor_id, int32_t q, float eps, int32_t x_replicated,
+                            void* scratch, size_t scratch_bytes, uint32_t flags) {
+  return mp_lora_linear_impl(cuda_stream, precision, X, W, bias, A, B, nullptr, Y, T, k_in, k_out, r, scale, seed,
+                             tensor_id, q, eps, x_replicated, scratch, scratch_bytes, flags);
+}
+
+zo_status zo_mp_lora_linear_pair(void* cuda_stream, int32_t precision, const void* X, const void* W,
+                                 const void* bias, const void* A, float* B_pair, void* Y, int32_t T,
+                                 int32_t k_in, int32_t k_out, int32_t r, float scale, uint64_t seed,
+                                 uint32_t tensor_id, float g_prev, float eps, float lr, int32_t x_replicated,
+                                 void* scratch, size_t scratch_bytes, uint32_t flags) {
+  if (!B_pair || r < 1 || k_out < 1 || !(eps > 0.f) || !isfinite(eps) || !isfinite(lr) || !isfinite(g_prev))
+    return ZO_ERR_INVALID_ARG;
+  if (k_out % 4) return ZO_ERR_UNSUPPORTED;
+  // lines 2-6 of Algorithm 2 on the stored pair, then the layer on the pair as it then stands
+  UpdateDesc D{};
+  D.B[0] = B_pair; D.tensor_base[0] = tensor_id; D.count = 1; D.n_slots = 1;
+  D.elems_per_slot = (long long)r * k_out;
+  launch_pair_update((cudaStream_t)cuda_stream, D, D.elems_per_slot, nullptr, g_prev, eps, lr, seed, 1);
+  return mp_lora_linear_impl(cuda_stream, precision, X, W, bias, A, B_pair, B_pair + (size_t)r * k_out, Y, T, k_in,
+                             k_out, r, scale, seed, tensor_id, 1, eps, x_replicated, scratch, scratch_bytes, flags);
+}
+
+}  // extern "C"
+
+namespace {
+
+// Previous update and (draw != 0) new perturbation applied to every stored pair of the model.
+void enqueue_pair_update(zo_ctx* c, const zo_lora_pair* pair, uint64_t seed, const float* dev_g_prev, float eps,
+                         float lr, int draw) {
+  const zo_config& cf = c->cfg;
+  const int r = cf.lora_rank;
+  if (cf.arch == ZO_ARCH_LINEAR) {
+    UpdateDesc D{};
+    D.B[0] = pair->B_pair[0]; D.tensor_base[0] = 0; D.count = 1; D.n_slots = 1;
+    D.elems_per_slot = (long long)r * cf.d_out;
+    PROF(PC_UPDATE, 0.0, launch_pair_update(c->st, D, D.elems_per_slot, dev_g_prev, 0.f, eps, lr, seed, draw));
+    return;
+  }
+  const int nt = c->nt;
+  for (int l0 = 0; l0 < cf.n_layers && nt; l0 += UpdateDesc::MAX_T) {
+    UpdateDesc D{};
+    D.count = cf.n_layers - l0 < UpdateDesc::MAX_T ? cf.n_layers - l0 : UpdateDesc::MAX_T;
+    D.n_slots = nt;
+    D.elems_per_slot = (long long)r * cf.d_model;
+    for (int i = 0; i < D.count; ++i) {
+      D.B[i] = pair->B_pair[l0 + i];
+      D.tensor_base[i] = (uint32_t)((l0 + i) * nt);
+    }
+    PROF(PC_UPDATE, 0.0, launch_pair_update(c->st, D, (long long)nt * D.elems_per_slot, dev_g_prev, 0.f, eps, lr,
+                                            seed, draw));
+  }
+}
+
+zo_status check_pair_args(zo_ctx* c, const zo_lora_pair* pair, float eps, float lr) {
+  if (!c) return ZO_ERR_INVALID_ARG;
+  if (!pair || !pair->A || !pair->B_pair) return fail(c, ZO_ERR_INVALID_ARG, "lora pair is NULL");
+  if (!(eps > 0.f) || !isfinite(eps)) return fail(c, ZO_ERR_INVALID_ARG, "the stored-pair step needs eps > 0");
+  if (!isfinite(lr)) return fail(c, ZO_ERR_INVALID_ARG, "lr must be finite");
+  if (c->shard_count) return fail(c, ZO_ERR_STATE, "the stored-pair step has one query: switch query sharding off");
+  const int n_b = c->cfg.arch == ZO_ARCH_LINEAR ? 1 : (c->nt ? c->cfg.n_layers : 0);
+  for (int l = 0; l < n_b; ++l)
+    if (!pair->B_pair[l]) return fail(c, ZO_ERR_INVALID_ARG, "null LoRA pair tensor");
+  return ZO_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+zo_status zo_step_pair(zo_ctx* ctx, const zo_weights* weights, const zo_lora_pair* pair, const void* tokens,
+                       const void* labels, int32_t E, int32_t S, uint64_t seed, const float* dev_g_prev,
+                       float eps, float lr) {
+  zo_status s = check_pair_args(ctx, pair, eps, lr);
+  if (s) return s;
+  const zo_lora view{pair->A, pair->B_pair};          // B[l] of the view = B[0] of the pair; B[1] follows it
+  s = check_step_args(ctx, weights, &view, tokens, labels, E, S, 1, eps, lr);
+  if (s) return s;
+  s = begin_step(ctx, 1);
+  if (s) return s;
+  zo_ctx* c = ctx;
+  enqueue_pair_update(c, pair, seed, dev_g_prev, eps, lr, 1);
+  c->pair_mode = 1;
+  if (c->cfg.arch == ZO_ARCH_LINEAR)
+    s = step_linear(c, weights, &view, tokens, labels, E * S, seed, 1, eps, 0.f);
+  else
+    s = step_decoder(c, weights, &view, (const int32_t*)tokens, (const int32_t*)labels, E, S, seed, 1, eps, 0.f);
+  c->pair_mode = 0;
+  if (s) return s;
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  c->stepped = 1; c->last_q = 1; c->last_E = E; c->last_S = S;
+  return ZO_OK;
+}
+
+zo_status zo_pair_collapse(zo_ctx* ctx, const zo_lora_pair* pair, const float* dev_g_prev, float eps, float lr) {
+  const zo_status s = check_pair_args(ctx, pair, eps, lr);
+  if (s) return s;
+  zo_ctx* c = ctx;
+  enqueue_pair_update(c, pair, 0, dev_g_prev, eps, lr, 0);
+  const cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return fail(c, ZO_ERR_CUDA, "kernel launch: %s", cudaGetErrorString(e));
+  return ZO_OK;
+}
+
+zo_status zo_g_buffer(zo_ctx* ctx, float** dev_g, int32_t* host_capacity) {
+  if (!ctx) return ZO_ERR_INVALID_ARG;
+  if (!dev_g) return fail(ctx, ZO_ERR_INVALID_ARG, "dev_g is NULL");
+  *dev_g = ctx->at<float>(ctx->plan.g);
+  if (host_capacity) *host_capacity = ctx->cfg.max_q;
+  return ZO_OK;
 }
 
 }  // extern "C"
