@@ -69,6 +69,8 @@ struct Ctrl {
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
+  volatile uint32_t dq_go[2];       // decode warps: did the wait for a free stage succeed (alternating slots)
+  float nf4[16];                    // the NormalFloat-4 levels
 };
 constexpr uint32_t SLAB_BYTES = BN * BK * 2;     // generated B operand of the LoRA k-block (aliases the fp32 staging)
 constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + SLAB_BYTES + sizeof(Ctrl);  // both variants: 192 KiB of stages
@@ -94,9 +96,22 @@ struct Params {
   int n_half;               // 1: at most 128 output columns in all: one weight box per stage, MMAs of N = 128
   int ksplit;               // > 1: the K range of every tile is cut into ksplit units of work
   float4* part;             // ksplit > 1: fp32 partial accumulators, [unit][64 column quads][128 rows]
+  // Weight-only quantised B operand decoded inside the kernel (small batches: the GEMM is a stream of
+  // weights, and a weight is then read once, as codes): 0 = bf16 weights through TMA, 1 = int8 codes with one
+  // scale per row, 2 = NF4 codes (two per byte, blocks of 64 along K) with one absmax per row and k-block.
+  int wfmt;
+  const uint8_t* wq;
+  const float* wscale;
   unsigned long long wait_ns;   // limit of the bounded waits (WAIT_LIMIT_NS unless a failure-detection test shortens it)
   int withhold;             // failure-detection test: CTA 0 never delivers the second k-block of its first tile
 };
+
+// The 16 levels of the 4-bit NormalFloat format (Dettmers et al., "QLoRA"): normal quantiles scaled to [-1, 1].
+__constant__ float c_nf4_levels[16] = {-1.0f, -0.6961928009986877f, -0.5250730514526367f, -0.39491748809814453f,
+                                       -0.28444138169288635f, -0.18477343022823334f, -0.09105003625154495f, 0.0f,
+                                       0.07958029955625534f, 0.16093020141124725f, 0.24611230194568634f,
+                                       0.33791524171829224f, 0.44070982933044434f, 0.5626170039176941f,
+                                       0.7229568362236023f, 1.0f};
 
 // ------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -310,7 +325,9 @@ __device__ __forceinline__ int tile_slot(const Params& P, int n0) {
 // runs no MMA at all: its CTAs take a quarter of a tile's column chunks each, sum the parts in K order
 // (so the result does not depend on timing) and run the same fused epilogue as SPLIT 0.
 constexpr int FIN_GROUPS = 4;
-template <bool PAIR, int SPLIT>
+// WQ: the B operand is decoded inside the kernel from weight-only quantised codes (instantiated apart so
+// that the decode path costs the bf16 kernels no registers).
+template <bool PAIR, int SPLIT, bool WQ = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmU, const Params P) {
@@ -351,9 +368,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < MAX_STAGES; ++s) {
-      mbar_init(smem_u32(&ctrl->full[s]), 1);
+      // a quantised B operand is written into the stage by the eight decode warps, who arrive too
+      mbar_init(smem_u32(&ctrl->full[s]), WQ ? 1 + EP_WARPS : 1);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
+    if (WQ) for (int i = 0; i < 16; ++i) ctrl->nf4[i] = c_nf4_levels[i];
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctrl->tfull[a]), 1);
       mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 2 * EP_WARPS : EP_WARPS);
@@ -413,6 +432,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (rank == 0) mbar_expect_tx(bar, Cfg<PAIR>::TX_BYTES);
             tma_load_2d_pair(sa, &tmA, kb * BK, m0, bar);
             tma_load_2d_pair(sa + A_BYTES, &tmB, kb * BK, rank == 0 ? brow0 : brow1, bar);
+          } else if (WQ) {
+            mbar_expect_tx(bar, A_BYTES);            // the B operand of the stage comes from the decode warps
+            tma_load_2d(sa, &tmA, kb * BK, m0, bar);
           } else {
             mbar_expect_tx(bar, P.n_half ? A_BYTES + BOX_BYTES : Cfg<PAIR>::TX_BYTES);
             tma_load_2d(sa, &tmA, kb * BK, m0, bar);
@@ -568,6 +590,102 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ep_bar();
     }
     if (P.slab && SPLIT != 2 && t_first < t_end) gen_slab(t_first);
+    // Quantised weights: these warps are the producer of the B operand.  Thread `et` owns row `et` of
+    // the 256-row operand tile (= one output column): it reads the row's codes of DQ_G k-blocks at a
+    // time (128 contiguous bytes), one group ahead of the one it decodes, and writes each k-block as
+    // eight 16-byte chunks of bf16 into the stage, in the swizzled K-major layout of the TMA path.
+    // One fp32 product and one rounding per weight, as the stand-alone decoder does.
+    uint32_t dissued = 0;                            // stages used so far (mirrors the TMA producer's count)
+    auto decode_unit = [&](int d_tile) -> bool {
+      if constexpr (!WQ) return true;
+      int tm, tn, ks, kb0, kb1;
+      coords(d_tile, tm, tn);
+      kb_range(d_tile, ks, kb0, kb1);
+      const int brow0 = tn * ncol_tile;
+      const int wrow = P.swiglu ? (et < 128 ? brow0 + et : P.N + brow0 + (et - 128)) : brow0 + et;
+      const bool live = (P.swiglu ? (brow0 + (et & 127)) < P.N : wrow < P.N) && !(P.n_half && et >= 128);
+      const int nkb_all = P.K / BK;
+      const bool nf4 = P.wfmt == 2;
+      const int DQ_G = nf4 ? 4 : 2;                  // k-blocks per 128-byte group of a row's codes
+      const uint8_t* crow = P.wq + (size_t)wrow * (nf4 ? P.K / 2 : P.K);
+      const float* srow = P.wscale + (nf4 ? (size_t)wrow * nkb_all : (size_t)wrow);
+      const float rscale = (!nf4 && live) ? srow[0] : 0.f;
+      uint4 cur[8], nxt[8];
+      float csc[4], nsc[4];
+      auto load_group = [&](int g0, uint4 (&buf)[8], float (&sc)[4]) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          // NF4: k-block g0 + j/2, half j%2 (32 bytes per k-block); int8: k-block g0 + j/4, quarter j%4
+          const int kb = g0 + (nf4 ? (j >> 1) : (j >> 2));
+          buf[j] = (live && kb < kb1) ? __ldg(reinterpret_cast<const uint4*>(crow + (size_t)g0 * (nf4 ? 32 : 64)) + j)
+                                      : make_uint4(0, 0, 0, 0);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) sc[j] = (nf4 && live && g0 + j < kb1) ? __ldg(srow + g0 + j) : 0.f;
+      };
+      load_group(kb0, cur, csc);
+      for (int g0 = kb0; g0 < kb1; g0 += DQ_G) {
+        if (g0 + DQ_G < kb1) load_group(g0 + DQ_G, nxt, nsc);
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi) {
+          const int kb = g0 + gi;
+          if (gi < DQ_G && kb < kb1) {                // uniform over the CTA
+            const uint32_t s = dissued % STAGES, ph = (dissued / STAGES) & 1u;
+            if (et == 0) ctrl->dq_go[dissued & 1u] = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status) ? 1u : 0u;
+            ep_bar();
+            if (ctrl->dq_go[dissued & 1u] == 0u) return false;
+            uint8_t* brow = smem + s * STAGE_BYTES + A_BYTES + et * 128;
+            if (!(P.n_half && et >= 128)) {
+#pragma unroll
+              for (int c = 0; c < 8; ++c) {           // 16-byte chunk c: K elements 8c .. 8c+7 of the k-block
+                float w[8];
+                if (nf4) {
+                  // 4 code bytes of chunk c: the even element sits in the high nibble
+                  const uint4 q4 = cur[2 * gi + (c >> 2)];
+                  const uint32_t word = (c & 3) == 0 ? q4.x : (c & 3) == 1 ? q4.y : (c & 3) == 2 ? q4.z : q4.w;
+#pragma unroll
+                  for (int b = 0; b < 4; ++b) {
+                    const uint32_t byte = (word >> (8 * b)) & 0xFFu;
+                    w[2 * b] = ctrl->nf4[byte >> 4] * csc[gi];
+                    w[2 * b + 1] = ctrl->nf4[byte & 15u] * csc[gi];
+                  }
+                } else {
+                  const uint4 q4 = cur[4 * gi + (c >> 1)];
+                  const uint32_t w0 = (c & 1) ? q4.z : q4.x, w1 = (c & 1) ? q4.w : q4.y;
+#pragma unroll
+                  for (int b = 0; b < 4; ++b) {
+                    w[b] = (float)(int)(int8_t)((w0 >> (8 * b)) & 0xFFu) * rscale;
+                    w[4 + b] = (float)(int)(int8_t)((w1 >> (8 * b)) & 0xFFu) * rscale;
+                  }
+                }
+                *reinterpret_cast<uint4*>(brow + ((c ^ (et & 7)) << 4)) =
+                    make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]), pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7]));
+              }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
+            ++dissued;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) csc[j] = nsc[j];
+      }
+      // the LoRA k-blocks of the unit bring only their A operand through the ring: arrive for the stage
+      if (ks == 0 && tile_slot(P, brow0) >= 0) {
+        for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++dissued) {
+          const uint32_t s = dissued % STAGES, ph = (dissued / STAGES) & 1u;
+          if (et == 0) ctrl->dq_go[dissued & 1u] = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status) ? 1u : 0u;
+          ep_bar();
+          if (ctrl->dq_go[dissued & 1u] == 0u) return false;
+          if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
+        }
+      }
+      return true;
+    };
+    constexpr bool wq_mode = WQ;
     uint32_t titer = 0;
     // iteration space: the units of this CTA; in the summing launch (tile, chunk group) pairs
     const int e_first = SPLIT == 2 ? (int)blockIdx.x : t_first;
@@ -577,6 +695,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int tile = SPLIT == 2 ? (it / FIN_GROUPS) * ksplit : it;   // (summing launch: first unit of the tile)
       const int grp = SPLIT == 2 ? it % FIN_GROUPS : -1;
       const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
+      if constexpr (WQ) {
+        // this unit's operands first: its LoRA operand (the first unit's was built above; the slab is free
+        // again because the previous unit's accumulator has been waited for), then its decoded weights
+        if (P.slab && titer > 0) gen_slab(tile);
+        if (!decode_unit(tile)) break;
+      }
       if (SPLIT != 2) {
         if (et == 0) ctrl->ep_go = mbar_wait(smem_u32(&ctrl->tfull[a]), aph, ctrl, P.status) ? 1u : 0u;
         ep_bar();
@@ -585,7 +709,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!go) break;
         tc_fence_after();
         // this tile's MMAs have retired, so the slab is free: build the next tile's operand first
-        if (P.slab && tile + t_step < t_end) gen_slab(tile + t_step);
+        if (P.slab && !wq_mode && tile + t_step < t_end) gen_slab(tile + t_step);
       }
       int tm, tn;
       coords(tile, tm, tn);
@@ -949,6 +1073,12 @@ int gemm_tc_init() {
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
   if (e == cudaSuccess) g_dev_ready[dev].store(true, std::memory_order_release);
   return (int)e;
 }
@@ -977,8 +1107,14 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   CUtensorMap tmA, tmB;
   int e = make_map(&tmA, G.A, (uint64_t)G.K, (uint64_t)G.M, (uint64_t)G.lda);
   if (e) return 10000 + e;
-  e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
-  if (e) return 10000 + e;
+  if (G.wfmt) {
+    // codes are decoded inside the kernel; only whole k-blocks, one thread block per tile
+    if (!G.wq || !G.wscale || G.K % tc::BK != 0) return (int)cudaErrorInvalidValue;
+    tmB = tmA;
+  } else {
+    e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
+    if (e) return 10000 + e;
+  }
   tc::Params P;
   P.M = G.M;
   P.N = G.swiglu ? G.N / 2 : G.N;
@@ -1001,6 +1137,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   }
   P.status = status;
   P.ksplit = 1; P.part = nullptr;
+  P.wfmt = G.wfmt; P.wq = (const uint8_t*)G.wq; P.wscale = G.wscale;
   P.wait_ns = G.test_wait_ns ? G.test_wait_ns : tc::WAIT_LIMIT_NS;
   P.withhold = G.test_wait_ns ? 1 : 0;
   const int tiles_n = (P.N + (G.swiglu ? 128 : tc::BN) - 1) / (G.swiglu ? 128 : tc::BN);
@@ -1038,7 +1175,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   // operand serves both 128-row halves of a tile: a replica must then be a whole number of 256-row tiles.
   const bool pair_slab_ok = P.slab && P.kslot == tc::BK && P.L.rows_per_replica % (2 * tc::BM) == 0;
   // (a down-projection that also packs bf16 U always runs single-CTA)
-  const bool pair = P.M > tc::BM && !G.pack_out && !P.withhold &&
+  const bool pair = P.M > tc::BM && !G.pack_out && !P.withhold && !G.wfmt &&
                     (G.cta_pair == 1 || (G.cta_pair == 2 && (!G.lora || pair_slab_ok) && P.N >= tc::BN &&
                                          tiles2 >= 8LL * max_clusters &&
                                          2.0 * (double)G.M * (double)G.N * (double)G.K <= 3.0e12));
@@ -1066,11 +1203,14 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   const long long units = tiles * P.ksplit;
   const int grid = (int)(units < n_sms ? units : n_sms);
   if (P.ksplit > 1) {
-    tc::gemm_tc_kernel<false, 1><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+    if (G.wfmt) tc::gemm_tc_kernel<false, 1, true><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+    else tc::gemm_tc_kernel<false, 1><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
     const long long fin = tiles * tc::FIN_GROUPS;
     tc::gemm_tc_kernel<false, 2><<<(int)(fin < n_sms ? fin : n_sms), tc::THREADS, tc::SMEM_BYTES_SUM, st>>>(tmA, tmB, tmU, P);
     if (G.extra_launches) ++*G.extra_launches;
-  } else
+  } else if (G.wfmt)
+    tc::gemm_tc_kernel<false, 0, true><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+  else
     tc::gemm_tc_kernel<false, 0><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
   return (int)cudaGetLastError();
 }

@@ -75,6 +75,9 @@ struct GemmDesc {
   int split_units;
   int* extra_launches;          // incremented when the GEMM took a second launch (split K), or null
   int split_cap;                // > 0: upper bound on the number of K ranges per tile (1 = never split)
+  int wfmt;                     // tensor-core kernel: 0 = W holds bf16 weights; 1 / 2 = W is unused and the B operand is decoded
+  const void* wq;               // inside the kernel from int8 / NF4 codes [N, K] / [N, K/2] ...
+  const float* wscale;          // ... and their float32 scales [N] / [N, K/64] (K % 64 == 0; at most 256 rows M)
   unsigned long long test_wait_ns;  // failure-detection tests only; > 0: the launch runs single-CTA, its bounded waits give
                                 // up after this many ns, and CTA 0 withholds one k-block so that a wait does run out
 };

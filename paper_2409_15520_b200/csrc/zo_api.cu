@@ -488,12 +488,20 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
                         &c->launches, c->err, sizeof(c->err), (slab && !first) ? ub : nullptr, nt * kslot, r, kslot);
       if (s) return s;
     }
-    // quantised storage: decode each weight right before its GEMM, once for all replicas of the pass
+    // Quantised storage.  Launches of at most 256 rows (small batches: the GEMM is a stream of weights) decode
+    // the codes inside the tensor-core kernel's operand producer, so a weight is read once, as codes, and never
+    // written back.  Larger launches reuse every weight tile hundreds of times: there the weight is decoded
+    // once per forward pass into scratch, right before its GEMM, for all replicas of the pass.
+    const bool tcore = bf && !(cf.flags & ZO_FLAG_SIMT_GEMM);
     void* wdq = c->at<uint8_t>(c->plan.wdq);
-    auto weight = [&](const void* wq, const float* sc, int n_rows, int k_in) -> const void* {
-      if (cf.weight_format == ZO_W_NATIVE) return wq;
+    auto set_weight = [&](GemmDesc& D, const void* wq, const float* sc, int n_rows, int k_in) {
+      if (cf.weight_format == ZO_W_NATIVE) { D.W = wq; return; }
+      if (tcore && D.M <= 256 && !(cf.flags & ZO_FLAG_DEQUANT_SCRATCH)) {
+        D.W = nullptr; D.wfmt = cf.weight_format; D.wq = wq; D.wscale = sc;
+        return;
+      }
       PROF(PC_DEQUANT, 0.0, launch_dequant(st, bf, cf.weight_format, wq, sc, wdq, n_rows, k_in));
-      return wdq;
+      D.W = wdq;
     };
     // The rotary embedding rides in the epilogue of whichever tensor-core GEMM writes q|k|v last.
     bool rope_done = opt;
@@ -501,9 +509,9 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       D.rope_tab = rope; D.rope_cols = 2 * d; D.rope_dh = d / H; D.rope_s = S; D.rope_tp = Tp; D.rope_pos = sl.pos;
       rope_done = true;
     };
-    const bool tcore = bf && !(cf.flags & ZO_FLAG_SIMT_GEMM);
     GemmDesc G{};
-    G.A = xn; G.lda = d; G.W = weight(W.w_qkv, W.s_qkv, 3 * d, d); G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
+    G.A = xn; G.lda = d; G.M = rows; G.N = 3 * d; G.K = d; G.bias = W.b_qkv;
+    set_weight(G, W.w_qkv, W.s_qkv, 3 * d, d);
     G.prof_class = PC_GEMM_QKV;
     if (first) {
       // first perturbed layer: one base product on the shared block, expanded to 2q outputs
@@ -533,12 +541,14 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, sl, Tp, d, H));
     }
     GemmDesc O{};
-    O.A = x; O.lda = d; O.W = weight(W.w_o, W.s_o, d, d); O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
+    O.A = x; O.lda = d; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
+    set_weight(O, W.w_o, W.s_o, d, d);
     O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0; O.prof_class = PC_GEMM_O;
     GEMM(O);
     PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0));
     GemmDesc F1{};
-    F1.A = x; F1.lda = d; F1.W = weight(W.w_fc1, W.s_fc1, opt ? f : 2 * f, d); F1.M = M; F1.K = d; F1.bias = W.b_fc1; F1.prof_class = PC_GEMM_FC1;
+    F1.A = x; F1.lda = d; F1.M = M; F1.K = d; F1.bias = W.b_fc1; F1.prof_class = PC_GEMM_FC1;
+    set_weight(F1, W.w_fc1, W.s_fc1, opt ? f : 2 * f, d);
     if (opt) {
       F1.N = f; F1.out = a; F1.ldo = f; F1.act = ACT_RELU;
       GEMM(F1);
@@ -551,7 +561,8 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(F1);
     }
     GemmDesc F2{};
-    F2.A = a; F2.lda = f; F2.W = weight(W.w_fc2, W.s_fc2, d, f); F2.M = M; F2.N = d; F2.K = f; F2.out = h; F2.ldo = d;
+    F2.A = a; F2.lda = f; F2.M = M; F2.N = d; F2.K = f; F2.out = h; F2.ldo = d;
+    set_weight(F2, W.w_fc2, W.s_fc2, d, f);
     F2.bias = W.b_fc2; F2.res = h; F2.ldr = d; F2.prof_class = PC_GEMM_FC2;
     GEMM(F2);
   }
