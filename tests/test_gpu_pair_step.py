@@ -122,8 +122,9 @@ def test_pair_steps_follow_the_master_copy_recurrence(kind):
             assert err < 5e-3, t
     est.pair_collapse(prob, gbuf, spec.eps, spec.lr)
     final = prob.pair_numpy()
-    for x in final:      # both halves at the updated master copy (B[0] - diff and B[1] + diff round apart by an ulp)
-        assert np.allclose(x[0], x[1], rtol=0, atol=4 * 2.0 ** -24 * np.max(np.abs(x)))
+    for x in final:      # both halves at the updated master copy: B[0] - diff and B[1] + diff round apart by an
+        # ulp of the perturbed values they are formed from
+        assert np.allclose(x[0], x[1], rtol=0, atol=2.0 ** -22 * (np.max(np.abs(x)) + 6 * spec.eps))
     if not spec.bf16:
         assert _rel([x[0] for x in final], masters[-1], masters[0]) < 1e-2
     # the same chain with nothing read back between the steps: g travels on the device only
