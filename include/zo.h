@@ -102,6 +102,11 @@ enum { ZO_FLAG_SIMT_GEMM = 1,
         * inside the tensor-core kernel (which small launches, at most 256 rows, do by default).  A/B switch;
         * both forms compute the same bits. */
        ZO_FLAG_DEQUANT_SCRATCH = 16,
+       /* ZO_FLAG_CE_LOGITS: the full-vocabulary loss stores float32 logits [2q*E*max_labelled, vocab] in the
+        * workspace and reduces them in a second kernel.  Default in bfloat16 mode: the LM-head GEMM's epilogue
+        * folds its tile of logits into (max, sum of exp) pairs and the logits never reach memory.  Checker /
+        * A/B switch; the two forms differ in summation order only. */
+       ZO_FLAG_CE_LOGITS = 32,
        /* ZO_FLAG_TEST_EXPIRE_WAIT (zo_mp_lora_linear only; contexts use zo_test_expire_wait): failure-
         * detection test aid, see zo_test_expire_wait. */
        ZO_FLAG_TEST_EXPIRE_WAIT = 1 << 24 };

@@ -821,6 +821,49 @@ void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const 
   ce_rows_kernel<<<rows, 256, 0, st>>>(logits, ldl, V, lab_val, EP, row_loss);
 }
 
+// Second half of the fused cross-entropy head: one warp per labelled row merges the (max, sum) pairs of
+// the row's column tiles.  Lane l folds pairs l, l + 32, ... in index order, then the lanes are folded by
+// a fixed butterfly: the order, and with it every bit of the result, is the same from run to run.
+__global__ void __launch_bounds__(256)
+ce_merge_kernel(const float2* __restrict__ part, int ppr, const float* __restrict__ logit,
+                const int32_t* __restrict__ lab_val, int EP, int rows, double* __restrict__ row_loss) {
+  const int row = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  if (lab_val[row % EP] < 0) {
+    if (lane == 0) row_loss[row] = 0.0;
+    return;
+  }
+  const float2* p = part + (size_t)row * ppr;
+  double m = -INFINITY, s = 0.0;
+  auto fold = [&](double m2, double s2) {
+    if (m2 == -INFINITY) return;                 // an empty share
+    if (m2 > m) { s = s * exp(m - m2) + s2; m = m2; }   // (first pair: m = -inf, s = 0)
+    else s += s2 * exp(m2 - m);
+  };
+  for (int i = lane; i < ppr; i += 32) {
+    const float2 v = p[i];
+    fold((double)v.x, (double)v.y);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const double m2 = __shfl_xor_sync(0xffffffffu, m, o), s2 = __shfl_xor_sync(0xffffffffu, s, o);
+    // both partners must end with the same bits: fold the pair in lane order, whichever side this is
+    double ma = (lane & o) ? m2 : m, sa = (lane & o) ? s2 : s;
+    const double mb = (lane & o) ? m : m2, sb = (lane & o) ? s : s2;
+    if (mb != -INFINITY) {
+      if (mb > ma) { sa = sa * exp(ma - mb) + sb; ma = mb; }
+      else sa += sb * exp(mb - ma);
+    }
+    m = ma; s = sa;
+  }
+  if (lane == 0) row_loss[row] = (m - (double)logit[row]) + log(s);
+}
+void launch_ce_merge(cudaStream_t st, const void* ce_part, int parts_per_row, const float* ce_logit,
+                     const int32_t* lab_val, int EP, int rows, double* row_loss) {
+  if (rows <= 0) return;
+  ce_merge_kernel<<<(rows + 7) / 8, 256, 0, st>>>((const float2*)ce_part, parts_per_row, ce_logit, lab_val, EP, rows, row_loss);
+}
+
 // Two-way softmax over the two label-word logits at the labelled (final) position.
 template <typename T>
 __global__ void label_word_rows_kernel(const T* __restrict__ xh, const T* __restrict__ head,

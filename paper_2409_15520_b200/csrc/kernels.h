@@ -75,6 +75,11 @@ struct GemmDesc {
   int split_units;
   int* extra_launches;          // incremented when the GEMM took a second launch (split K), or null
   int split_cap;                // > 0: upper bound on the number of K ranges per tile (1 = never split)
+  void* ce_part;                // tensor-core kernel, cross-entropy head: non-null = store no output; per (row, 256-column tile,
+                                // sibling warp) one float2 (max, sum of exp(logit - max)) into ce_part [M][ceil(N/256)][2] ...
+  float* ce_logit;              // ... and the label's logit of every row whose label is >= 0 into ce_logit [M]
+  const int32_t* ce_label;      // label of row m = ce_label[m % ce_ep]
+  int ce_ep;
   int wfmt;                     // tensor-core kernel: 0 = W holds bf16 weights; 1 / 2 = W is unused and the B operand is decoded
   const void* wq;               // inside the kernel from int8 / NF4 codes [N, K] / [N, K/2] ...
   const float* wscale;          // ... and their float32 scales [N] / [N, K/64] (K % 64 == 0; at most 256 rows M)
@@ -120,6 +125,10 @@ void launch_label_scan(cudaStream_t st, const int32_t* labels, SeqLayout sl, int
                        int32_t* lab_idx, int32_t* lab_val, int32_t* lab_cnt, uint32_t* status);
 void launch_ce_rows(cudaStream_t st, const float* logits, int ldl, int V, const int32_t* lab_val,
                     int EP, int rows, double* row_loss);
+// Row losses from the partial (max, sum) pairs the cross-entropy head GEMM left: pairs merged in a fixed
+// order in fp64, loss = max + log(sum) - label logit (0 for rows whose label is < 0).
+void launch_ce_merge(cudaStream_t st, const void* ce_part, int parts_per_row, const float* ce_logit,
+                     const int32_t* lab_val, int EP, int rows, double* row_loss);
 void launch_label_word_rows(cudaStream_t st, int bf, const void* xh, const void* head, int d,
                             int w0, int w1, const int32_t* lab_val, int EP, int rows,
                             double* row_loss);

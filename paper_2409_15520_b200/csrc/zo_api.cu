@@ -22,7 +22,7 @@ constexpr int MAX_PASSES = 2 * ZO_MAX_Q;  // the sequential schedule cuts a step
 
 struct Plan {  // byte offsets into the workspace
   size_t h0, x0, qkv0, h, x, qkv, a, gu, U, rope, lab_idx, lab_val, lab_cnt, tok_stage, lab_stage,
-      xh, logits, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, pos, split_ws, total;
+      xh, logits, ce_part, ce_logit, rowloss, rowloss_pass, losses, losses_d, g, status, ub, wdq, pos, split_ws, total;
 };
 
 inline size_t up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -31,6 +31,13 @@ constexpr int SPLIT_UNITS = 160;   // units of split-K work the scratch can hold
 inline int n_targets(const zo_config& c) {
   return ((c.lora_targets >> 0) & 1) + ((c.lora_targets >> 1) & 1) + ((c.lora_targets >> 2) & 1);
 }
+// Full-vocabulary loss without the logits round trip: the head GEMM's epilogue reduces its tile to
+// (max, sum of exp) pairs.  Tensor-core path only; ZO_FLAG_CE_LOGITS keeps the stored-logits form.
+inline bool fused_ce(const zo_config& c) {
+  return c.loss_kind == ZO_LOSS_CE_FULL_VOCAB && c.precision == ZO_BF16 &&
+         !(c.flags & (ZO_FLAG_SIMT_GEMM | ZO_FLAG_CE_LOGITS));
+}
+inline size_t ce_parts_per_row(const zo_config& c) { return 2 * (((size_t)c.vocab + 255) / 256); }
 inline int row_pad(const zo_config& c) { return c.precision == ZO_BF16 ? 128 : 1; }
 // Queries a context runs in one step: all of them, or at most max_shard_q when it only ever runs shards.
 inline int run_q(const zo_config& c) { return c.max_shard_q > 0 ? c.max_shard_q : c.max_q; }
@@ -135,7 +142,12 @@ Plan make_plan(const zo_config& c) {
     p.lab_stage = take(Tm * 4);
     p.pos = take(Tp * 4);
     p.xh = take(Mh * d * es);
-    if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) p.logits = take(Mh * (size_t)c.vocab * 4);
+    if (fused_ce(c)) {
+      p.ce_part = take(Mh * ce_parts_per_row(c) * 8);
+      p.ce_logit = take(Mh * 4);
+    } else if (c.loss_kind == ZO_LOSS_CE_FULL_VOCAB) {
+      p.logits = take(Mh * (size_t)c.vocab * 4);
+    }
     p.rowloss = take(n * c.max_E * P * 8);
     p.rowloss_pass = take(Mh * 8);
     if (c.weight_format != ZO_W_NATIVE) {   // one dequantised weight at a time
@@ -572,7 +584,15 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   void* xh = c->at<uint8_t>(c->plan.xh);
   PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, xh, w->final_norm_g, w->final_norm_b, Mh, d, cf.norm_eps, lab_idx, EP, Tp));
   const void* head = cf.tie_lm_head ? w->tok_emb : w->lm_head;
-  if (cf.loss_kind == ZO_LOSS_CE_FULL_VOCAB) {
+  if (fused_ce(cf)) {
+    // LM head and log-softmax in one pass: the logits stay in tensor memory and registers
+    GemmDesc Hd{};
+    Hd.A = xh; Hd.lda = d; Hd.W = head; Hd.M = Mh; Hd.N = cf.vocab; Hd.K = d; Hd.prof_class = PC_GEMM_HEAD;
+    Hd.ce_part = c->at<uint8_t>(c->plan.ce_part); Hd.ce_logit = c->at<float>(c->plan.ce_logit);
+    Hd.ce_label = lab_val; Hd.ce_ep = EP;
+    GEMM(Hd);
+    PROF(PC_LOSS, 0.0, launch_ce_merge(st, Hd.ce_part, (int)ce_parts_per_row(cf), Hd.ce_logit, lab_val, EP, Mh, rowloss_pass));
+  } else if (cf.loss_kind == ZO_LOSS_CE_FULL_VOCAB) {
     float* logits = c->at<float>(c->plan.logits);
     GemmDesc Hd{};
     Hd.A = xh; Hd.lda = d; Hd.W = head; Hd.M = Mh; Hd.N = cf.vocab; Hd.K = d;

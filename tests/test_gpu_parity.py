@@ -477,3 +477,27 @@ def test_decoder_fp32_at_the_configured_eps(arch):
     assert np.allclose(got["losses"], ref["losses"], rtol=1e-4, atol=0)
     assert rel_g < 1e-2
     assert update_rel_err(spec, p, got["B"], ref["B"]) < 1e-3
+
+
+@pytest.mark.parametrize("arch,vocab,flags", [(ARCH_LLAMA, 1003, 0), (ARCH_OPT, 517, 0), (ARCH_OPT, 1003, PAIR),
+                                              (ARCH_LLAMA, 256, 0), (ARCH_LLAMA, 70, 0)])
+def test_fused_head_loss_matches_stored_logits(arch, vocab, flags):
+    """bf16 mode folds the LM-head tile into (max, sum of exp) pairs inside the GEMM epilogue; with
+    ZO_FLAG_CE_LOGITS the logits are stored and reduced by the stand-alone kernel.  Same accumulators,
+    another summation order: per-row losses agree to fp32 rounding, both stay within the bf16 tolerance
+    of the oracle.  Vocabularies with a ragged last column tile, exactly one tile, and less than one
+    32-column chunk; single-CTA and CTA-pair kernels."""
+    CE_LOGITS = 32
+    spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
+                     **{**TINY, "d_model": 256, "n_heads": 4, "d_ffn": 512, "vocab": vocab, "S": 80, "E": 4,
+                        "max_seq": 80, "q": 2, "n_labelled": 7, "lora_rank": 8})
+    p, tok, lab = make_problem(spec, b_std=0.05)
+    ref = run_oracle(spec, p, tok, lab, 37)
+    fused = run_gpu(spec, p, 37, flags=flags)
+    stored = run_gpu(spec, p, 37, flags=flags | CE_LOGITS)
+    assert np.allclose(fused["losses"], ref["losses"], rtol=2e-2, atol=0), (fused["losses"], ref["losses"])
+    assert np.allclose(fused["rows"], stored["rows"], rtol=2e-6, atol=0)
+    assert np.allclose(fused["losses"], stored["losses"], rtol=1e-6, atol=0)
+    assert fused["launches"] == stored["launches"]
+    again = run_gpu(spec, p, 37, flags=flags)
+    assert np.array_equal(fused["rows"], again["rows"])     # fixed merge order: same bits from run to run
