@@ -69,8 +69,8 @@ enum { ZO_LOSS_MSE = 0, ZO_LOSS_CE_FULL_VOCAB = 1, ZO_LOSS_CE_LABEL_WORDS = 2 };
 enum { ZO_TARGET_Q = 1, ZO_TARGET_K = 2, ZO_TARGET_V = 4 };
 /* Storage of the four frozen linear weights of a decoder block (w_qkv, w_o, w_fc1, w_fc2), after the
  * paper's appendix "MobiZO with weight-only quantization" (Q-LoRA style): stored low-bit, dequantised
- * to the compute type once per forward pass, i.e. once per step for all 2q replicas.  bfloat16 launches
- * of at most 256 rows decode inside the GEMM's operand producer instead (codes in, nothing written back).
+ * to the compute type once per forward pass, i.e. once per step for all 2q replicas (ZO_FLAG_DEQUANT_FUSED:
+ * small bfloat16 launches decode inside the GEMM's operand producer instead).
  *   ZO_W_NATIVE  element type of `precision`
  *   ZO_W_INT8    int8 codes [k_out, k_in] + float32 scale [k_out]:      w = code * scale[row]
  *   ZO_W_NF4     4-bit NormalFloat codes, two per byte (even element in the high nibble), uint8
@@ -98,10 +98,13 @@ enum { ZO_FLAG_SIMT_GEMM = 1,
         * from fp32 U and fp32 (B + k eps z), never as the extra tensor-core k-block (which rounds
         * U, B and k eps z to bfloat16).  A/B switch. */
        ZO_FLAG_LORA_EPILOGUE = 4,
-       /* ZO_FLAG_DEQUANT_SCRATCH: quantised weights are always decoded into scratch before their GEMM, never
-        * inside the tensor-core kernel (which small launches, at most 256 rows, do by default).  A/B switch;
-        * both forms compute the same bits. */
-       ZO_FLAG_DEQUANT_SCRATCH = 16,
+       /* ZO_FLAG_DEQUANT_FUSED: bfloat16 GEMM launches of at most 256 rows decode quantised weights inside
+        * the tensor-core kernel's operand producer (codes brought to shared memory by bulk tensor copies,
+        * decoded by the epilogue warps straight into the MMA's operand stage; a weight is read once, as
+        * codes, and nothing is written back) instead of decoding every weight into scratch before its GEMM.
+        * Same bf16 operands, same accumulation order: both forms compute the same bits.  Off by default:
+        * with eight decode warps per SM the in-kernel form is slower on B200 than decode-then-GEMM. */
+       ZO_FLAG_DEQUANT_FUSED = 16,
        /* ZO_FLAG_CE_LOGITS: the full-vocabulary loss stores float32 logits [2q*E*max_labelled, vocab] in the
         * workspace and reduces them in a second kernel.  Default in bfloat16 mode: the LM-head GEMM's epilogue
         * folds its tile of logits into (max, sum of exp) pairs and the logits never reach memory.  Checker /

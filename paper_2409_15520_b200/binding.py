@@ -19,7 +19,7 @@ STATUS_NAMES = ["ZO_OK", "ZO_ERR_INVALID_ARG", "ZO_ERR_UNSUPPORTED", "ZO_ERR_WOR
                 "ZO_ERR_CUDA", "ZO_ERR_TIMEOUT", "ZO_ERR_NONFINITE", "ZO_ERR_STATE"]
 ZO_FP32, ZO_BF16 = 0, 1
 ZO_FLAG_SIMT_GEMM, ZO_FLAG_GEMM_PAIR, ZO_FLAG_LORA_EPILOGUE, ZO_FLAG_GEMM_SINGLE = 1, 2, 4, 8
-ZO_FLAG_DEQUANT_SCRATCH = 16
+ZO_FLAG_DEQUANT_FUSED = 16
 ZO_FLAG_CE_LOGITS = 32
 ZO_FLAG_TEST_EXPIRE_WAIT = 1 << 24
 

@@ -65,12 +65,11 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct Ctrl {
   unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2], drain, lfull;
+  unsigned long long rawfull[2], rawempty[2];   // ring of quantised-code groups (kernels that decode weights)
   unsigned long long wait_ns;       // limit of every bounded wait of this CTA
   uint32_t tmem_base;
   volatile uint32_t abort;
   volatile uint32_t ep_go;
-  volatile uint32_t dq_go[2];       // decode warps: did the wait for a free stage succeed (alternating slots)
-  float nf4[16];                    // the NormalFloat-4 levels
 };
 constexpr uint32_t SLAB_BYTES = BN * BK * 2;     // generated B operand of the LoRA k-block (aliases the fp32 staging)
 constexpr size_t SMEM_BYTES = 1024 + 4 * 49152 + SLAB_BYTES + sizeof(Ctrl);  // both variants: 192 KiB of stages
@@ -187,9 +186,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // ring depth: one stage is given up when the LoRA term needs two generated k-blocks (rank > 32);
   // narrow-output launches stage one weight box, so the same 192 KiB hold six stages of 32 KiB
   const bool narrow = !PAIR && P.n_half;
+  // (the kernels that decode quantised weights keep two stages: the other two hold the ring of raw codes)
   const int STAGES = PAIR ? Cfg<PAIR>::STAGES
-                          : (narrow ? 6 : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0));
-  const uint32_t STAGE_BYTES = narrow ? A_BYTES + BOX_BYTES : Cfg<PAIR>::STAGE_BYTES;
+                          : (narrow && !WQ ? 6 : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0) - (WQ ? 2 : 0));
+  const uint32_t STAGE_BYTES = narrow && !WQ ? A_BYTES + BOX_BYTES : Cfg<PAIR>::STAGE_BYTES;
   constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
   const int GROUP_M = PAIR ? (P.group_m + 1) / 2 : P.group_m;   // row tiles of a raster group
   extern __shared__ uint8_t smem_raw[];
@@ -197,6 +197,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // the summing launch of split K stages nothing: its shared memory starts at the LoRA staging area
   float* lbuf = (float*)(smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES));
   Ctrl* ctrl = (Ctrl*)(smem + (SPLIT == 2 ? 0 : Cfg<PAIR>::STAGES * Cfg<PAIR>::STAGE_BYTES) + SLAB_BYTES);
+  // quantised weights: two slots of raw codes (a group of k-blocks: 256 rows x 128 bytes each) behind the slab area
+  constexpr uint32_t RAW_BYTES = 2 * BOX_BYTES;
+  uint8_t* raw_ring = smem + STAGES * STAGE_BYTES + (P.kslot > 64 ? 2 : 1) * SLAB_BYTES;
+  // NF4: code byte -> (level of its high nibble, level of its low nibble): one 8-byte look-up per two weights
+  float2* nf4_pairs = reinterpret_cast<float2*>(raw_ring + 2 * RAW_BYTES);
   const uint32_t tiles_base = smem_u32(smem);
   const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -225,10 +230,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&ctrl->full[s]), WQ ? 1 + EP_WARPS : 1);
       mbar_init(smem_u32(&ctrl->empty[s]), 1);
     }
-    if (WQ) for (int i = 0; i < 16; ++i) ctrl->nf4[i] = c_nf4_levels[i];
+
     for (int a = 0; a < 2; ++a) {
       mbar_init(smem_u32(&ctrl->tfull[a]), 1);
       mbar_init(smem_u32(&ctrl->tempty[a]), PAIR ? 2 * EP_WARPS : EP_WARPS);
+    }
+    if (WQ) {
+      for (int r = 0; r < 2; ++r) {
+        mbar_init(smem_u32(&ctrl->rawfull[r]), 1);
+        mbar_init(smem_u32(&ctrl->rawempty[r]), EP_WARPS);
+      }
     }
     mbar_init(smem_u32(&ctrl->drain), 1);
     mbar_init(smem_u32(&ctrl->lfull), PAIR ? 2 * EP_WARPS : EP_WARPS);
@@ -238,6 +249,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (WQ)
+    for (int i = threadIdx.x; i < 256; i += THREADS) nf4_pairs[i] = make_float2(c_nf4_levels[i >> 4], c_nf4_levels[i & 15]);
   if (warp == 1 && SPLIT != 2) {
     if (PAIR) {
       asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -443,100 +456,142 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       ep_bar();
     }
     if (P.slab && SPLIT != 2 && t_first < t_end) gen_slab(t_first);
-    // Quantised weights: these warps are the producer of the B operand.  Thread `et` owns row `et` of
-    // the 256-row operand tile (= one output column): it reads the row's codes of DQ_G k-blocks at a
-    // time (128 contiguous bytes), one group ahead of the one it decodes, and writes each k-block as
-    // eight 16-byte chunks of bf16 into the stage, in the swizzled K-major layout of the TMA path.
-    // One fp32 product and one rounding per weight, as the stand-alone decoder does.
+    // Quantised weights: these warps are the producer of the B operand.  The codes of a GROUP of k-blocks
+    // (128 bytes of every one of the tile's 256 weight rows: 4 k-blocks of NF4, 2 of int8) are brought
+    // into a two-slot ring in shared memory by bulk tensor copies (issued by the first decode warp, one
+    // group ahead), so the weight stream moves in full lines with many bytes in flight.  Thread `et`
+    // owns row `et` of the operand tile (= one output column): it reads the row's codes from the slot and
+    // writes each k-block as eight 16-byte chunks of bf16 into the stage, in the swizzled K-major layout
+    // of the TMA path.  One fp32 product and one rounding per weight, as the stand-alone decoder does.
+    // The warps run independently (each polls the barriers itself, one lane per warp).
     uint32_t dissued = 0;                            // stages used so far (mirrors the TMA producer's count)
-    auto decode_unit = [&](int d_tile) -> bool {
-      if constexpr (!WQ) return true;
+    uint32_t rgroups = 0;                            // code groups consumed so far (slot and phase of the ring)
+    bool dq_ok = true;                               // this warp's waits so far succeeded
+    auto warp_wait = [&](uint32_t bar, uint32_t parity) -> bool {   // one lane waits, all lanes learn the outcome
+      uint32_t ok = 1u;
+      if (lane == 0) ok = mbar_wait(bar, parity, ctrl, P.status) ? 1u : 0u;
+      return __shfl_sync(0xffffffffu, ok, 0) != 0u;
+    };
+    auto decode_unit = [&](int d_tile) {
+      if constexpr (!WQ) return;
       int tm, tn, ks, kb0, kb1;
       coords(d_tile, tm, tn);
       kb_range(d_tile, ks, kb0, kb1);
       const int brow0 = tn * ncol_tile;
-      const int wrow = P.swiglu ? (et < 128 ? brow0 + et : P.N + brow0 + (et - 128)) : brow0 + et;
+      const int brow1 = P.swiglu ? P.N + brow0 : brow0 + 128;
+      const int wrow = et < 128 ? brow0 + et : brow1 + (et - 128);
       const bool live = (P.swiglu ? (brow0 + (et & 127)) < P.N : wrow < P.N) && !(P.n_half && et >= 128);
       const int nkb_all = P.K / BK;
       const bool nf4 = P.wfmt == 2;
       const int DQ_G = nf4 ? 4 : 2;                  // k-blocks per 128-byte group of a row's codes
-      const uint8_t* crow = P.wq + (size_t)wrow * (nf4 ? P.K / 2 : P.K);
       const float* srow = P.wscale + (nf4 ? (size_t)wrow * nkb_all : (size_t)wrow);
       const float rscale = (!nf4 && live) ? srow[0] : 0.f;
-      uint4 cur[8], nxt[8];
-      float csc[4], nsc[4];
-      auto load_group = [&](int g0, uint4 (&buf)[8], float (&sc)[4]) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          // NF4: k-block g0 + j/2, half j%2 (32 bytes per k-block); int8: k-block g0 + j/4, quarter j%4
-          const int kb = g0 + (nf4 ? (j >> 1) : (j >> 2));
-          buf[j] = (live && kb < kb1) ? __ldg(reinterpret_cast<const uint4*>(crow + (size_t)g0 * (nf4 ? 32 : 64)) + j)
-                                      : make_uint4(0, 0, 0, 0);
+      // group `gr` of this CTA's sequence -> ring slot gr & 1; its codes start at k-block g0
+      auto issue_group = [&](uint32_t gr, int g0) -> bool {       // first decode warp only
+        const uint32_t slot = gr & 1u, ph = (gr >> 1) & 1u;
+        if (!warp_wait(smem_u32(&ctrl->rawempty[slot]), ph ^ 1u)) return false;
+        if (lane == 0) {
+          const uint32_t bar = smem_u32(&ctrl->rawfull[slot]);
+          const uint32_t dst = smem_u32(raw_ring + slot * RAW_BYTES);
+          const int xb = g0 * (nf4 ? 32 : 64);                    // byte offset inside a weight row
+          mbar_expect_tx(bar, P.n_half ? BOX_BYTES : RAW_BYTES);
+          tma_load_2d(dst, &tmB, xb, brow0, bar);
+          if (!P.n_half) tma_load_2d(dst + BOX_BYTES, &tmB, xb, brow1, bar);
         }
+        return true;
+      };
+      float csc[4] = {0.f, 0.f, 0.f, 0.f}, nsc[4] = {0.f, 0.f, 0.f, 0.f};
+      auto load_scales = [&](int g0, float (&sc)[4]) {
 #pragma unroll
         for (int j = 0; j < 4; ++j) sc[j] = (nf4 && live && g0 + j < kb1) ? __ldg(srow + g0 + j) : 0.f;
       };
-      load_group(kb0, cur, csc);
-      for (int g0 = kb0; g0 < kb1; g0 += DQ_G) {
-        if (g0 + DQ_G < kb1) load_group(g0 + DQ_G, nxt, nsc);
+      if (warp == 2) dq_ok = issue_group(rgroups, kb0);
+      load_scales(kb0, csc);
+      for (int g0 = kb0; g0 < kb1 && dq_ok; g0 += DQ_G, ++rgroups) {
+        if (g0 + DQ_G < kb1) {
+          if (warp == 2) dq_ok = issue_group(rgroups + 1, g0 + DQ_G);
+          load_scales(g0 + DQ_G, nsc);
+          if (!dq_ok) break;
+        }
+        const uint32_t slot = rgroups & 1u;
+        if (!warp_wait(smem_u32(&ctrl->rawfull[slot]), (rgroups >> 1) & 1u)) { dq_ok = false; break; }
+        // this thread's 128 code bytes of the group, chunk c16 at its swizzled place
+        const uint8_t* rrow = raw_ring + slot * RAW_BYTES + (et >> 7) * BOX_BYTES + (et & 127) * 128;
 #pragma unroll
         for (int gi = 0; gi < 4; ++gi) {
           const int kb = g0 + gi;
-          if (gi < DQ_G && kb < kb1) {                // uniform over the CTA
+          if (gi < DQ_G && kb < kb1 && dq_ok) {       // uniform over the warp
             const uint32_t s = dissued % STAGES, ph = (dissued / STAGES) & 1u;
-            if (et == 0) ctrl->dq_go[dissued & 1u] = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status) ? 1u : 0u;
-            ep_bar();
-            if (ctrl->dq_go[dissued & 1u] == 0u) return false;
-            uint8_t* brow = smem + s * STAGE_BYTES + A_BYTES + et * 128;
-            if (!(P.n_half && et >= 128)) {
-#pragma unroll
-              for (int c = 0; c < 8; ++c) {           // 16-byte chunk c: K elements 8c .. 8c+7 of the k-block
-                float w[8];
+            dq_ok = warp_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u);
+            if (dq_ok) {
+              uint8_t* brow = smem + s * STAGE_BYTES + A_BYTES + et * 128;
+              if (!(P.n_half && et >= 128)) {
                 if (nf4) {
-                  // 4 code bytes of chunk c: the even element sits in the high nibble
-                  const uint4 q4 = cur[2 * gi + (c >> 2)];
-                  const uint32_t word = (c & 3) == 0 ? q4.x : (c & 3) == 1 ? q4.y : (c & 3) == 2 ? q4.z : q4.w;
+                  const float sc = csc[gi];
 #pragma unroll
-                  for (int b = 0; b < 4; ++b) {
-                    const uint32_t byte = (word >> (8 * b)) & 0xFFu;
-                    w[2 * b] = ctrl->nf4[byte >> 4] * csc[gi];
-                    w[2 * b + 1] = ctrl->nf4[byte & 15u] * csc[gi];
+                  for (int h = 0; h < 2; ++h) {       // 16 code bytes = 32 weights = 4 output chunks
+                    const uint4 q4 = *reinterpret_cast<const uint4*>(rrow + (((2 * gi + h) ^ (et & 7)) << 4));
+                    const uint32_t cw[4] = {q4.x, q4.y, q4.z, q4.w};
+                    float w[32];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {    // byte i: element 2i in the high nibble, 2i + 1 in the low one
+                      const float2 pr = nf4_pairs[(cw[i >> 2] >> (8 * (i & 3))) & 0xFFu];
+                      w[2 * i] = pr.x;
+                      w[2 * i + 1] = pr.y;
+                    }
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) w[i] *= sc;
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                      *reinterpret_cast<uint4*>(brow + (((4 * h + c) ^ (et & 7)) << 4)) =
+                          make_uint4(pack_bf16(w[8 * c], w[8 * c + 1]), pack_bf16(w[8 * c + 2], w[8 * c + 3]),
+                                     pack_bf16(w[8 * c + 4], w[8 * c + 5]), pack_bf16(w[8 * c + 6], w[8 * c + 7]));
                   }
                 } else {
-                  const uint4 q4 = cur[4 * gi + (c >> 1)];
-                  const uint32_t w0 = (c & 1) ? q4.z : q4.x, w1 = (c & 1) ? q4.w : q4.y;
 #pragma unroll
-                  for (int b = 0; b < 4; ++b) {
-                    w[b] = (float)(int)(int8_t)((w0 >> (8 * b)) & 0xFFu) * rscale;
-                    w[4 + b] = (float)(int)(int8_t)((w1 >> (8 * b)) & 0xFFu) * rscale;
+                  for (int h = 0; h < 4; ++h) {       // 16 code bytes = 16 weights = 2 output chunks
+                    const uint4 q4 = *reinterpret_cast<const uint4*>(rrow + (((4 * gi + h) ^ (et & 7)) << 4));
+                    const uint32_t cw[4] = {q4.x, q4.y, q4.z, q4.w};
+                    float w[16];
+                    // int8 -> float without a conversion instruction: byte b ^ 0x80 placed in the low mantissa
+                    // byte of 2^23 is the float 8388608 + (b + 128), so subtracting 8388736 leaves b exactly
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                      const uint32_t bits = __byte_perm(cw[i >> 2] ^ 0x80808080u, 0x4B000000u, 0x7650 + (i & 3));
+                      w[i] = (__uint_as_float(bits) - 8388736.f) * rscale;
+                    }
+#pragma unroll
+                    for (int c = 0; c < 2; ++c)
+                      *reinterpret_cast<uint4*>(brow + (((2 * h + c) ^ (et & 7)) << 4)) =
+                          make_uint4(pack_bf16(w[8 * c], w[8 * c + 1]), pack_bf16(w[8 * c + 2], w[8 * c + 3]),
+                                     pack_bf16(w[8 * c + 4], w[8 * c + 5]), pack_bf16(w[8 * c + 6], w[8 * c + 7]));
                   }
                 }
-                *reinterpret_cast<uint4*>(brow + ((c ^ (et & 7)) << 4)) =
-                    make_uint4(pack_bf16(w[0], w[1]), pack_bf16(w[2], w[3]), pack_bf16(w[4], w[5]), pack_bf16(w[6], w[7]));
               }
+              asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+              __syncwarp();
+              if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
+              ++dissued;
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
-            ++dissued;
           }
         }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) cur[j] = nxt[j];
+        // done with the slot (on the abort path nobody refills it)
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->rawempty[slot]));
 #pragma unroll
         for (int j = 0; j < 4; ++j) csc[j] = nsc[j];
       }
       // the LoRA k-blocks of the unit bring only their A operand through the ring: arrive for the stage
       if (ks == 0 && tile_slot(P, brow0) >= 0) {
-        for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++dissued) {
+        for (int lkb = 0; lkb < P.kslot / BK && dq_ok; ++lkb) {
           const uint32_t s = dissued % STAGES, ph = (dissued / STAGES) & 1u;
-          if (et == 0) ctrl->dq_go[dissued & 1u] = mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status) ? 1u : 0u;
-          ep_bar();
-          if (ctrl->dq_go[dissued & 1u] == 0u) return false;
-          if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
+          dq_ok = warp_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u);
+          if (dq_ok) {
+            if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
+            ++dissued;
+          }
         }
       }
-      return true;
     };
     constexpr bool wq_mode = WQ;
     uint32_t titer = 0;
@@ -551,8 +606,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if constexpr (WQ) {
         // this unit's operands first: its LoRA operand (the first unit's was built above; the slab is free
         // again because the previous unit's accumulator has been waited for), then its decoded weights
+        // (a warp whose wait ran out stops decoding; the CTA-wide decision to leave is taken at the wait
+        // for the accumulator below, where one thread sees the abort flag for all)
         if (P.slab && titer > 0) gen_slab(tile);
-        if (!decode_unit(tile)) break;
+        decode_unit(tile);
       }
       if (SPLIT != 2) {
         if (et == 0) ctrl->ep_go = mbar_wait(smem_u32(&ctrl->tfull[a]), aph, ctrl, P.status) ? 1u : 0u;
@@ -974,6 +1031,17 @@ static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, 
                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+// 2-D byte tensor map over quantised codes: rows x row_bytes, box 128 rows x 128 bytes, 128-byte swizzle.
+static int make_code_map(CUtensorMap* m, const void* ptr, uint64_t row_bytes, uint64_t rows) {
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {128u, 128u};
+  const cuuint32_t es[2] = {1u, 1u};
+  return (int)g_encode(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_sms) {
   if (G.M <= 0 || G.N <= 0) return 0;
   if (G.K <= 0) return (int)cudaErrorInvalidValue;   // every tile needs at least one base k-block
@@ -989,7 +1057,8 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   if (G.wfmt) {
     // codes are decoded inside the kernel; only whole k-blocks, one thread block per tile
     if (!G.wq || !G.wscale || G.K % tc::BK != 0) return (int)cudaErrorInvalidValue;
-    tmB = tmA;
+    e = make_code_map(&tmB, G.wq, (uint64_t)(G.wfmt == 2 ? G.K / 2 : G.K), (uint64_t)G.N);
+    if (e) return 10000 + e;
   } else {
     e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K);
     if (e) return 10000 + e;

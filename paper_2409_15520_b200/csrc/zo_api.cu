@@ -500,15 +500,16 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
                         &c->launches, c->err, sizeof(c->err), (slab && !first) ? ub : nullptr, nt * kslot, r, kslot);
       if (s) return s;
     }
-    // Quantised storage.  Launches of at most 256 rows (small batches: the GEMM is a stream of weights) decode
-    // the codes inside the tensor-core kernel's operand producer, so a weight is read once, as codes, and never
-    // written back.  Larger launches reuse every weight tile hundreds of times: there the weight is decoded
-    // once per forward pass into scratch, right before its GEMM, for all replicas of the pass.
+    // Quantised storage.  Default: each weight is decoded once per forward pass into scratch, right before
+    // its GEMM, for all replicas of the pass (large launches reuse every weight tile hundreds of times).
+    // ZO_FLAG_DEQUANT_FUSED: launches of at most 256 rows (small batches: the GEMM is a stream of weights)
+    // decode the codes inside the tensor-core kernel's operand producer instead, so a weight is read once, as
+    // codes, and never written back.
     const bool tcore = bf && !(cf.flags & ZO_FLAG_SIMT_GEMM);
     void* wdq = c->at<uint8_t>(c->plan.wdq);
     auto set_weight = [&](GemmDesc& D, const void* wq, const float* sc, int n_rows, int k_in) {
       if (cf.weight_format == ZO_W_NATIVE) { D.W = wq; return; }
-      if (tcore && D.M <= 256 && !(cf.flags & ZO_FLAG_DEQUANT_SCRATCH)) {
+      if (tcore && D.M <= 256 && (cf.flags & ZO_FLAG_DEQUANT_FUSED)) {
         D.W = nullptr; D.wfmt = cf.weight_format; D.wq = wq; D.wscale = sc;
         return;
       }

@@ -59,9 +59,9 @@ def test_step_on_quantised_checkpoint(arch, bf16, fmt):
 @pytest.mark.parametrize("arch,E,S,sched", [(ARCH_LLAMA, 1, 100, None), (ARCH_OPT, 2, 128, "sequential"),
                                             (ARCH_LLAMA, 1, 128, "sequential")])
 def test_decode_inside_the_gemm_matches_decode_to_scratch(arch, E, S, sched, fmt):
-    """Small batches (at most 256 rows per GEMM launch) decode the codes inside the tensor-core kernel's
-    operand producer; ZO_FLAG_DEQUANT_SCRATCH forces the decode-then-GEMM form.  Same bf16 operands, same
-    accumulation order: the two steps agree bit for bit, whole tiles (E*S*2 = 200 -> 256 rows, two row
+    """With ZO_FLAG_DEQUANT_FUSED, GEMM launches of at most 256 rows decode the codes inside the tensor-core
+    kernel's operand producer; the default decodes every weight into scratch first.  Same bf16 operands,
+    same accumulation order: the two steps agree bit for bit, whole tiles (E*S*2 = 200 -> 256 rows, two row
     tiles), K ranges of split launches (d = 512, ffn = 1024) and the SwiGLU gate|up layout included.
     The oracle's step on the same stored bytes bounds both."""
     spec = ModelSpec(arch=arch, tie_lm_head=(arch == ARCH_OPT), bf16=True,
@@ -70,8 +70,8 @@ def test_decode_inside_the_gemm_matches_decode_to_scratch(arch, E, S, sched, fmt
     p = make_decoder_problem(spec, seed=8, b_std=0.05)
     p["layers"] = [quantize_layer(L, fmt) for L in p["layers"]]
     ref = run_oracle(spec, p, p["tokens"], p["labels"], 29)
-    fused = run_gpu(spec, p, 29, weight_format=fmt, schedule=sched)
-    scratch = run_gpu(spec, p, 29, weight_format=fmt, schedule=sched, flags=16)
+    fused = run_gpu(spec, p, 29, weight_format=fmt, schedule=sched, flags=16)
+    scratch = run_gpu(spec, p, 29, weight_format=fmt, schedule=sched)
     assert np.allclose(fused["losses"], ref["losses"], rtol=2e-2, atol=0), (fused["losses"], ref["losses"])
     assert np.array_equal(fused["losses"], scratch["losses"]) and np.array_equal(fused["rows"], scratch["rows"])
     assert np.array_equal(fused["g"], scratch["g"])
