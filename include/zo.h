@@ -105,6 +105,11 @@ enum { ZO_FLAG_SIMT_GEMM = 1,
         * Same bf16 operands, same accumulation order: both forms compute the same bits.  Off by default:
         * with eight decode warps per SM the in-kernel form is slower on B200 than decode-then-GEMM. */
        ZO_FLAG_DEQUANT_FUSED = 16,
+       /* ZO_FLAG_ATTN_WARP_MMA: bfloat16 attention always runs the warp-level (mma.sync) kernel.  Default for
+        * head_dim 64 / 128 and sequences of at most 256 tokens: the tcgen05 kernel (scores and P V on the
+        * fifth-generation tensor cores with tensor-memory accumulators, q / k / v brought in by bulk tensor
+        * copies).  A/B switch. */
+       ZO_FLAG_ATTN_WARP_MMA = 64,
        /* ZO_FLAG_CE_LOGITS: the full-vocabulary loss stores float32 logits [2q*E*max_labelled, vocab] in the
         * workspace and reduces them in a second kernel.  Default in bfloat16 mode: the LM-head GEMM's epilogue
         * folds its tile of logits into (max, sum of exp) pairs and the logits never reach memory.  Checker /

@@ -21,6 +21,7 @@ ZO_FP32, ZO_BF16 = 0, 1
 ZO_FLAG_SIMT_GEMM, ZO_FLAG_GEMM_PAIR, ZO_FLAG_LORA_EPILOGUE, ZO_FLAG_GEMM_SINGLE = 1, 2, 4, 8
 ZO_FLAG_DEQUANT_FUSED = 16
 ZO_FLAG_CE_LOGITS = 32
+ZO_FLAG_ATTN_WARP_MMA = 64
 ZO_FLAG_TEST_EXPIRE_WAIT = 1 << 24
 
 

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libzo_b200.so")
-SOURCES = ["kernels.cu", "gemm_simt.cu", "gemm_tc.cu", "attention_mma.cu", "lora_expand.cu", "zo_api.cu", "no_alloc.cu"]
+SOURCES = ["kernels.cu", "gemm_simt.cu", "gemm_tc.cu", "attention_mma.cu", "attention_tc.cu", "lora_expand.cu", "zo_api.cu", "no_alloc.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

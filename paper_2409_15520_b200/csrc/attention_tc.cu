@@ -1,0 +1,382 @@
+// Causal attention on the Blackwell tensor cores for sequences of up to 256 tokens (bf16, head_dim 64
+// or 128): softmax(Q K^T / sqrt(dh) + causal) V over the n*E sequences of the replicated batch (q and
+// k already carry their rotary embedding).  Attention is ~1 % of the step's flops; the kernel's job is
+// to read q, k, v once, write the context once, and keep those streams in flight.
+//
+//   * persistent CTAs, one per SM; a job is one (sequence, head).  Warp 0 is the copy engine's
+//     producer (cp.async.bulk.tensor boxes of 128 rows x 64 columns, 128-byte swizzle, no multicast),
+//     warp 1 issues tcgen05.mma, warps 2-5 own one query row per thread (softmax and output).
+//   * a sequence of <= 256 tokens is at most two query tiles and two key tiles, so the scores of a
+//     whole query tile fit in tensor memory (128 + 256 columns for the two tiles): the row maximum is
+//     exact, nothing is ever rescaled.  S = Q K^T (both operands K-major), the row threads read S twice
+//     with tcgen05.ld (maximum, then exponentials), write P in bf16 into a two-slot ring of 64-key
+//     chunks in the K-major swizzled layout, and O += P V runs with V as an MN-major operand (V sits in
+//     shared memory as the copy engine delivers it: key rows, head_dim contiguous).
+//   * the loads of job j+1 overlap the arithmetic of job j: Q and K are free as soon as both score
+//     products have retired (early in the job), V when the last P V product has.
+//   * every wait is bounded; on expiry the CTA raises ST_TIMEOUT, drains its copies and MMAs, frees its
+//     tensor memory and returns.
+#include <math.h>
+
+#include <atomic>
+
+#include "kernels.h"
+#include "tcgen05.cuh"
+
+namespace zo {
+namespace atc {
+
+using namespace tc;
+
+constexpr int THREADS = 192;
+constexpr uint32_t BOX = 128 * 128;                 // one 128-row x 64-column bf16 box, 16 KiB
+constexpr uint32_t TMEM_COLS = 512;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
+
+struct Ctrl {
+  unsigned long long qk_full, qk_empty, v_full, v_empty, s_full[2], s_empty[2], p_full[2], p_empty[2], o_full, o_empty,
+      drain;
+  uint32_t tmem_base;
+  volatile uint32_t abort;
+};
+
+template <int DH> struct Lay {
+  static constexpr int KB = DH / 64;                // 64-column boxes per head
+  static constexpr uint32_t Q_OFF = 0;              // [query tile][box][128 rows x 128 B]
+  static constexpr uint32_t K_OFF = 2 * KB * BOX;   // [box][256 key rows x 128 B]
+  static constexpr uint32_t V_OFF = K_OFF + 2 * KB * BOX;
+  static constexpr uint32_t P_OFF = V_OFF + 2 * KB * BOX;   // two chunks of [128 rows x 64 keys]
+  static constexpr uint32_t DATA = P_OFF + 2 * BOX;
+  static constexpr size_t SMEM = 1024 + DATA + sizeof(Ctrl);
+};
+
+struct Params {
+  bf16* ctx;
+  SeqLayout sl;
+  int n, Tp, d, H;
+  float scale_log2e;                                // log2(e) / sqrt(dh)
+  uint32_t* status;
+};
+
+// bf16 x bf16 -> fp32, M = 128; B K-major or MN-major
+__host__ __device__ constexpr uint32_t idesc(int n, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | ((uint32_t)(n >> 3) << 17) |
+         ((uint32_t)(128 >> 4) << 24);
+}
+// MN-major operand, 128-byte swizzle: 64 elements contiguous along MN, rows (K) 128 B apart, groups of
+// eight rows 1024 B apart (stride offset), the next 64 elements along MN `lbo_bytes` further (leading offset)
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, uint32_t lbo_bytes) {
+  uint64_t dsc = 0;
+  dsc |= (uint64_t)((addr & 0x3FFFFu) >> 4);
+  dsc |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  dsc |= (uint64_t)(1024u >> 4) << 32;
+  dsc |= (uint64_t)1 << 46;
+  dsc |= (uint64_t)2 << 61;
+  return dsc;
+}
+__device__ __forceinline__ float ex2f(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+template <int DH>
+__global__ void __launch_bounds__(THREADS, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
+  using L = Lay<DH>;
+  constexpr int KB = L::KB;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  Ctrl* ctrl = (Ctrl*)(smem + L::DATA);
+  const uint32_t base = smem_u32(smem);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_jobs = P.n * P.sl.E * P.H;
+
+  if (threadIdx.x == 0) {
+    mbar_init(smem_u32(&ctrl->qk_full), 1);
+    mbar_init(smem_u32(&ctrl->qk_empty), 1);
+    mbar_init(smem_u32(&ctrl->v_full), 1);
+    mbar_init(smem_u32(&ctrl->v_empty), 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_u32(&ctrl->s_full[i]), 1);
+      mbar_init(smem_u32(&ctrl->s_empty[i]), 4);
+      mbar_init(smem_u32(&ctrl->p_full[i]), 4);
+      mbar_init(smem_u32(&ctrl->p_empty[i]), 1);
+    }
+    mbar_init(smem_u32(&ctrl->o_full), 1);
+    mbar_init(smem_u32(&ctrl->o_empty), 4);
+    mbar_init(smem_u32(&ctrl->drain), 1);
+    ctrl->abort = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctrl->tmem_base)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = ctrl->tmem_base;
+  auto wait = [&](unsigned long long* bar, uint32_t parity) {
+    return mbar_wait_bounded(smem_u32(bar), parity, &ctrl->abort, WAIT_LIMIT_NS, P.status);
+  };
+  // job -> (first row of the sequence in the replicated buffer, its length, head)
+  auto job_of = [&](int job, size_t& row_base, int& S_len, int& h) {
+    const int sq = job / P.H;
+    h = job - sq * P.H;
+    const int rep = sq / P.sl.E, b = sq - rep * P.sl.E;
+    row_base = (size_t)rep * P.Tp + (size_t)P.sl.start(b);
+    S_len = min(P.sl.len(b), 256);
+  };
+
+  if (warp == 0) {
+    // ---------------------------------------------------------------- copy producer
+    if (lane == 0) {
+      uint32_t it = 0, qk_issued = 0, v_issued = 0;
+      bool ok = true;
+      for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+        size_t row_base; int S_len, h;
+        job_of(job, row_base, S_len, h);
+        if (S_len <= 0) continue;
+        const int nqt = (S_len + 127) >> 7;
+        const int y0 = (int)row_base;
+        if (!wait(&ctrl->qk_empty, (it & 1u) ^ 1u)) { ok = false; break; }
+        {
+          const uint32_t bar = smem_u32(&ctrl->qk_full);
+          mbar_expect_tx(bar, (uint32_t)(2 * nqt * KB) * BOX);
+          for (int t = 0; t < nqt; ++t)
+            for (int kb = 0; kb < KB; ++kb) {
+              tma_load_2d(base + L::Q_OFF + (t * KB + kb) * BOX, &tm, h * DH + kb * 64, y0 + t * 128, bar);
+              tma_load_2d(base + L::K_OFF + kb * 2 * BOX + t * BOX, &tm, P.d + h * DH + kb * 64, y0 + t * 128, bar);
+            }
+          ++qk_issued;
+        }
+        if (!wait(&ctrl->v_empty, (it & 1u) ^ 1u)) { ok = false; break; }
+        {
+          const uint32_t bar = smem_u32(&ctrl->v_full);
+          mbar_expect_tx(bar, (uint32_t)(nqt * KB) * BOX);
+          for (int t = 0; t < nqt; ++t)
+            for (int kb = 0; kb < KB; ++kb)
+              tma_load_2d(base + L::V_OFF + kb * 2 * BOX + t * BOX, &tm, 2 * P.d + h * DH + kb * 64, y0 + t * 128, bar);
+          ++v_issued;
+        }
+        ++it;
+      }
+      if (!ok) {
+        // abort: let the copies already issued land before the CTA goes away (a phase that completed
+        // long ago answers at once)
+        if (qk_issued) mbar_wait_drain(smem_u32(&ctrl->qk_full), (qk_issued - 1u) & 1u);
+        if (v_issued) mbar_wait_drain(smem_u32(&ctrl->v_full), (v_issued - 1u) & 1u);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      uint32_t it = 0, us[2] = {0u, 0u}, pc = 0, oc = 0;
+      bool ok = true;
+      for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+        size_t row_base; int S_len, h;
+        job_of(job, row_base, S_len, h);
+        if (S_len <= 0) continue;
+        const int nqt = (S_len + 127) >> 7;
+        if (!wait(&ctrl->qk_full, it & 1u)) { ok = false; break; }
+        for (int t = 0; t < nqt && ok; ++t) {
+          // S_t = Q_t K^T over the keys 0 .. 128 (t + 1) - 1 (causal: later keys are never needed)
+          if (!wait(&ctrl->s_empty[t], (us[t] & 1u) ^ 1u)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t dcol = tmem + (t == 0 ? 0u : 128u);
+          for (int kb = 0; kb < KB; ++kb) {
+            const uint64_t ad = smem_desc(base + L::Q_OFF + (t * KB + kb) * BOX);
+            const uint64_t bd = smem_desc(base + L::K_OFF + kb * 2 * BOX);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              tc_mma(dcol, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), t == 0 ? idesc(128, false) : idesc(256, false),
+                     (uint32_t)((kb | k) != 0));
+          }
+          tc_commit(smem_u32(&ctrl->s_full[t]));
+          ++us[t];
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&ctrl->qk_empty));        // Q and K may be overwritten once both products retire
+        if (!wait(&ctrl->v_full, it & 1u)) { ok = false; break; }
+        for (int t = 0; t < nqt && ok; ++t) {
+          const int kend = min(S_len, (t + 1) * 128), nch = (kend + 63) >> 6;
+          if (!wait(&ctrl->o_empty, (oc & 1u) ^ 1u)) { ok = false; break; }
+          tc_fence_after();
+          for (int c = 0; c < nch; ++c, ++pc) {
+            const uint32_t slot = pc & 1u;
+            if (!wait(&ctrl->p_full[slot], (pc >> 1) & 1u)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t ad = smem_desc(base + L::P_OFF + slot * BOX);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              // V rows (keys) 64 c + 16 k ..: MN-major operand, the second 64 columns of a 128-wide head 32 KiB on
+              const uint64_t bd = smem_desc_mn(base + L::V_OFF + (uint32_t)(c * 64 + k * 16) * 128u, 2 * BOX);
+              tc_mma(tmem + 384u, ad + (uint64_t)(2 * k), bd, idesc(DH, true), (uint32_t)((c | k) != 0));
+            }
+            tc_commit(smem_u32(&ctrl->p_empty[slot]));
+          }
+          if (!ok) break;
+          tc_commit(smem_u32(&ctrl->o_full));
+          ++oc;
+        }
+        if (!ok) break;
+        tc_commit(smem_u32(&ctrl->v_empty));
+        ++it;
+      }
+      if (!ok) {
+        tc_commit(smem_u32(&ctrl->drain));           // wait for the MMAs already issued
+        mbar_wait_drain(smem_u32(&ctrl->drain), 0u);
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- one query row per thread
+    const int wq = warp & 3;                         // tensor-memory lane quarter of this warp
+    const int r = wq * 32 + lane;                    // row of the query tile
+    const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
+    uint32_t us[2] = {0u, 0u}, pc = 0, oc = 0;
+    bool ok = true;
+    // one lane waits, the warp learns the outcome
+    auto warp_wait = [&](unsigned long long* bar, uint32_t parity) -> bool {
+      uint32_t good = 1u;
+      if (lane == 0) good = wait(bar, parity) ? 1u : 0u;
+      return __shfl_sync(0xffffffffu, good, 0) != 0u;
+    };
+    for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
+      size_t row_base; int S_len, h;
+      job_of(job, row_base, S_len, h);
+      if (S_len <= 0) continue;
+      const int nqt = (S_len + 127) >> 7;
+      for (int t = 0; t < nqt && ok; ++t) {
+        const int qpos = t * 128 + r;
+        const int kend = min(S_len, (t + 1) * 128), nch = (kend + 63) >> 6;
+        const uint32_t scol = lane_base + (t == 0 ? 0u : 128u);
+        if (!warp_wait(&ctrl->s_full[t], us[t] & 1u)) { ok = false; break; }
+        ++us[t];
+        tc_fence_after();
+        // key k counts for this row when k <= qpos (causal) and k < S_len (rows past the end of the
+        // sequence in the loaded tiles belong to other sequences)
+        const int klim = min(qpos, S_len - 1);
+        float m = -INFINITY;
+        for (int j = 0; j < 2 * nch; ++j) {
+          uint32_t v[32];
+          tc_ld32(scol + j * 32, v);
+          tc_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 32; ++i)
+            if (j * 32 + i <= klim) m = fmaxf(m, __uint_as_float(v[i]));
+        }
+        const float ms = m * P.scale_log2e;
+        float l = 0.f;
+        for (int c = 0; c < nch && ok; ++c, ++pc) {
+          const uint32_t slot = pc & 1u;
+          if (!warp_wait(&ctrl->p_empty[slot], ((pc >> 1) & 1u) ^ 1u)) { ok = false; break; }
+          uint8_t* prow = smem + L::P_OFF + slot * BOX + r * 128;
+#pragma unroll
+          for (int hh = 0; hh < 2; ++hh) {
+            const int j = 2 * c + hh;
+            uint32_t v[32];
+            tc_ld32(scol + j * 32, v);
+            tc_ld_wait();
+            float p[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              p[i] = (j * 32 + i <= klim) ? ex2f(fmaf(__uint_as_float(v[i]), P.scale_log2e, -ms)) : 0.f;
+              l += p[i];
+            }
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4)           // 16-byte chunk hh*4 + q4 of the row's 128 bytes: keys 8 per chunk
+              *reinterpret_cast<uint4*>(prow + (((hh * 4 + q4) ^ (r & 7)) << 4)) =
+                  make_uint4(pack_bf16(p[8 * q4], p[8 * q4 + 1]), pack_bf16(p[8 * q4 + 2], p[8 * q4 + 3]),
+                             pack_bf16(p[8 * q4 + 4], p[8 * q4 + 5]), pack_bf16(p[8 * q4 + 6], p[8 * q4 + 7]));
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&ctrl->p_full[slot]));
+        }
+        if (!ok) break;
+        // scores consumed: the next job's product for this tile may overwrite them
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->s_empty[t]));
+        // normalised output of the tile
+        if (!warp_wait(&ctrl->o_full, oc & 1u)) { ok = false; break; }
+        ++oc;
+        tc_fence_after();
+        const float inv = 1.f / l;
+        bf16* orow = P.ctx + (row_base + (size_t)qpos) * P.d + h * DH;
+#pragma unroll
+        for (int j = 0; j < DH / 32; ++j) {
+          uint32_t v[32];
+          tc_ld32(lane_base + 384u + j * 32, v);
+          tc_ld_wait();
+          if (qpos < S_len) {
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4)
+              *reinterpret_cast<uint4*>(orow + j * 32 + q4 * 8) = make_uint4(
+                  pack_bf16(__uint_as_float(v[8 * q4]) * inv, __uint_as_float(v[8 * q4 + 1]) * inv),
+                  pack_bf16(__uint_as_float(v[8 * q4 + 2]) * inv, __uint_as_float(v[8 * q4 + 3]) * inv),
+                  pack_bf16(__uint_as_float(v[8 * q4 + 4]) * inv, __uint_as_float(v[8 * q4 + 5]) * inv),
+                  pack_bf16(__uint_as_float(v[8 * q4 + 6]) * inv, __uint_as_float(v[8 * q4 + 7]) * inv));
+          }
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&ctrl->o_empty));
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(TMEM_COLS) : "memory");
+  }
+}
+
+}  // namespace atc
+
+// ---------------------------------------------------------------------------------- host side
+bool attention_tc_supported(int dh, int max_len) { return (dh == 64 || dh == 128) && max_len <= 256; }
+
+template <int DH>
+static int launch_t(cudaStream_t st, const CUtensorMap& tm, const atc::Params& P, int n_sms, int n_jobs) {
+  static std::atomic<unsigned long long> ready{0};   // bit per device ordinal: shared-memory opt-in done
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return (int)e;
+  if (dev < 0 || dev >= 64) return (int)cudaErrorInvalidDevice;
+  if (!(ready.load(std::memory_order_acquire) >> dev & 1ull)) {
+    e = cudaFuncSetAttribute(atc::attention_tc_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)atc::Lay<DH>::SMEM);
+    if (e != cudaSuccess) return (int)e;
+    ready.fetch_or(1ull << dev, std::memory_order_release);
+  }
+  const int grid = n_jobs < n_sms ? n_jobs : n_sms;
+  atc::attention_tc_kernel<DH><<<grid, atc::THREADS, atc::Lay<DH>::SMEM, st>>>(tm, P);
+  return (int)cudaGetLastError();
+}
+
+int launch_attention_tc(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl, int Tp, int d, int H,
+                        uint32_t* status, int n_sms) {
+  const int dh = d / H;
+  const int n_jobs = n * sl.E * H;
+  if (n_jobs <= 0) return 0;
+  CUtensorMap tm;
+  // rows of the replicated q|k|v buffer x 3d columns; boxes of 128 rows x 64 columns, 128-byte swizzle
+  const int me = tc_make_map_bf16(&tm, qkv, (uint64_t)3 * d, (uint64_t)n * Tp, (uint64_t)3 * d);
+  if (me) return 10000 + me;
+  atc::Params P;
+  P.ctx = (bf16*)ctx; P.sl = sl; P.n = n; P.Tp = Tp; P.d = d; P.H = H;
+  P.scale_log2e = 1.4426950408889634f / sqrtf((float)dh);
+  P.status = status;
+  return dh == 64 ? launch_t<64>(st, tm, P, n_sms, n_jobs) : launch_t<128>(st, tm, P, n_sms, n_jobs);
+}
+
+}  // namespace zo

@@ -1031,6 +1031,14 @@ static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, 
                        CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
 }
 
+int tc_make_map_bf16(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, uint64_t pitch_elems) {
+  if (!g_encode) {
+    const int e = gemm_tc_init();
+    if (e) return e;
+  }
+  return make_map(m, ptr, K, rows, pitch_elems);
+}
+
 // 2-D byte tensor map over quantised codes: rows x row_bytes, box 128 rows x 128 bytes, 128-byte swizzle.
 static int make_code_map(CUtensorMap* m, const void* ptr, uint64_t row_bytes, uint64_t rows) {
   const cuuint64_t dims[2] = {row_bytes, rows};

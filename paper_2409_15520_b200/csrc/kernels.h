@@ -116,6 +116,11 @@ void launch_attention_simt(cudaStream_t st, int bf, const void* qkv, void* ctx, 
 bool attention_mma_supported(int dh);
 void launch_attention_mma(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl, int Tp,
                           int d, int H);
+// Causal attention on tcgen05 tensor cores (bf16, head_dim 64 or 128, sequences of at most 256 tokens).
+// Returns a CUDA error code (0 = ok).
+bool attention_tc_supported(int dh, int max_len);
+int launch_attention_tc(cudaStream_t st, const void* qkv, void* ctx, int n, SeqLayout sl, int Tp, int d, int H,
+                        uint32_t* status, int n_sms);
 void launch_swiglu(cudaStream_t st, int bf, const void* gu, void* out, int rows, int ffn);
 // Positions of packed rows: pos[t] = t - cu[b] for the sequence b that holds row t (0 for pad rows);
 // flags sequences longer than max_len or a non-monotone cu.

@@ -7,6 +7,11 @@
 #include "common.cuh"
 
 namespace zo {
+
+// 2-D bf16 tensor map (host): rows x K elements with K contiguous and a row pitch of pitch_elems; boxes of
+// 128 rows x 64 columns, 128-byte swizzle, out-of-range elements read as zero.  0 = ok.
+int tc_make_map_bf16(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, uint64_t pitch_elems);
+
 namespace tc {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {

@@ -548,7 +548,14 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
     if (!rope_done) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, sl, d, H, rope)); }
-    if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
+    if (tcore && !(cf.flags & ZO_FLAG_ATTN_WARP_MMA) && attention_tc_supported(d / H, S)) {
+      int ae = 0;
+      PROF(PC_ATTN, 0.0, ae = launch_attention_tc(st, qkv, x, n, sl, Tp, d, H, status, c->n_sms));
+      if (ae) {
+        snprintf(c->err, sizeof(c->err), "tensor-core attention launch failed (code %d)", ae);
+        return ZO_ERR_CUDA;
+      }
+    } else if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
       PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, sl, Tp, d, H));
     } else {
       PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, sl, Tp, d, H));
