@@ -5,7 +5,9 @@
 //
 //   * persistent CTAs, one per SM; a job is one (sequence, head).  Warp 0 is the copy engine's
 //     producer (cp.async.bulk.tensor boxes of 128 rows x 64 columns, 128-byte swizzle, no multicast),
-//     warp 1 issues tcgen05.mma, warps 2-5 own one query row per thread (softmax and output).
+//     warp 1 issues tcgen05.mma, warps 2-9 are two threads per query row (softmax and output), each taking
+//     one half of every 64-key chunk of the row; pieces that the causal mask blanks for a whole warp are skipped,
+//     and the next piece is requested from tensor memory while the current one is worked on.
 //   * a sequence of <= 256 tokens is at most two query tiles and two key tiles, so the scores of a
 //     whole query tile fit in tensor memory (128 + 256 columns for the two tiles): the row maximum is
 //     exact, nothing is ever rescaled.  S = Q K^T (both operands K-major), the row threads read S twice
@@ -28,7 +30,8 @@ namespace atc {
 
 using namespace tc;
 
-constexpr int THREADS = 192;
+constexpr int SM_WARPS = 8;                        // softmax / output warps: two per tensor-memory lane quarter
+constexpr int THREADS = 64 + 32 * SM_WARPS;
 constexpr uint32_t BOX = 128 * 128;                 // one 128-row x 64-column bf16 box, 16 KiB
 constexpr uint32_t TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
@@ -38,7 +41,11 @@ struct Ctrl {
       drain;
   uint32_t tmem_base;
   volatile uint32_t abort;
+  unsigned long long pair[4];                       // meeting point of the two warps of a lane quarter
+  float xmax[2][128];                               // row maxima of the two threads of a row, exchanged both ways
+  float xsum[128];                                  // row sum of the odd-chunk thread, handed to the even-chunk one
 };
+static_assert(sizeof(Ctrl) <= 2048 - 128, "control block must fit beside 224 KiB of tiles");
 
 template <int DH> struct Lay {
   static constexpr int KB = DH / 64;                // 64-column boxes per head
@@ -99,13 +106,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
     mbar_init(smem_u32(&ctrl->v_empty), 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_u32(&ctrl->s_full[i]), 1);
-      mbar_init(smem_u32(&ctrl->s_empty[i]), 4);
-      mbar_init(smem_u32(&ctrl->p_full[i]), 4);
+      mbar_init(smem_u32(&ctrl->s_empty[i]), SM_WARPS);
+      mbar_init(smem_u32(&ctrl->p_full[i]), SM_WARPS);
       mbar_init(smem_u32(&ctrl->p_empty[i]), 1);
     }
     mbar_init(smem_u32(&ctrl->o_full), 1);
-    mbar_init(smem_u32(&ctrl->o_empty), 4);
+    mbar_init(smem_u32(&ctrl->o_empty), SM_WARPS / 2);
     mbar_init(smem_u32(&ctrl->drain), 1);
+    for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&ctrl->pair[i]), 2);
     ctrl->abort = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -177,31 +185,49 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
     if (lane == 0) {
       uint32_t it = 0, us[2] = {0u, 0u}, pc = 0, oc = 0;
       bool ok = true;
+      bool s0_ahead = false;                         // S_0 of the job about to start was already issued (hoisted)
+      // S_t = Q_t K^T of the job whose tiles are in shared memory, keys 0 .. 128 (t + 1) - 1 (causal: later
+      // keys are never needed); the caller has seen qk_full and s_empty[t]
+      auto issue_scores = [&](int t) {
+        tc_fence_after();
+        const uint32_t dcol = tmem + (t == 0 ? 0u : 128u);
+        for (int kb = 0; kb < KB; ++kb) {
+          const uint64_t ad = smem_desc(base + L::Q_OFF + (t * KB + kb) * BOX);
+          const uint64_t bd = smem_desc(base + L::K_OFF + kb * 2 * BOX);
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            tc_mma(dcol, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), t == 0 ? idesc(128, false) : idesc(256, false),
+                   (uint32_t)((kb | k) != 0));
+        }
+        tc_commit(smem_u32(&ctrl->s_full[t]));
+        ++us[t];
+      };
+      // next job of this CTA with a non-empty sequence (n_jobs if none)
+      auto next_job = [&](int job) {
+        for (job += gridDim.x; job < n_jobs; job += gridDim.x) {
+          size_t rb; int sl_, h_;
+          job_of(job, rb, sl_, h_);
+          if (sl_ > 0) return job;
+        }
+        return n_jobs;
+      };
       for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
         size_t row_base; int S_len, h;
         job_of(job, row_base, S_len, h);
         if (S_len <= 0) continue;
         const int nqt = (S_len + 127) >> 7;
-        if (!wait(&ctrl->qk_full, it & 1u)) { ok = false; break; }
-        for (int t = 0; t < nqt && ok; ++t) {
-          // S_t = Q_t K^T over the keys 0 .. 128 (t + 1) - 1 (causal: later keys are never needed)
-          if (!wait(&ctrl->s_empty[t], (us[t] & 1u) ^ 1u)) { ok = false; break; }
-          tc_fence_after();
-          const uint32_t dcol = tmem + (t == 0 ? 0u : 128u);
-          for (int kb = 0; kb < KB; ++kb) {
-            const uint64_t ad = smem_desc(base + L::Q_OFF + (t * KB + kb) * BOX);
-            const uint64_t bd = smem_desc(base + L::K_OFF + kb * 2 * BOX);
-#pragma unroll
-            for (int k = 0; k < 4; ++k)
-              tc_mma(dcol, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), t == 0 ? idesc(128, false) : idesc(256, false),
-                     (uint32_t)((kb | k) != 0));
-          }
-          tc_commit(smem_u32(&ctrl->s_full[t]));
-          ++us[t];
+        if (!s0_ahead) {
+          if (!wait(&ctrl->qk_full, it & 1u) || !wait(&ctrl->s_empty[0], (us[0] & 1u) ^ 1u)) { ok = false; break; }
+          issue_scores(0);
         }
-        if (!ok) break;
+        s0_ahead = false;
+        if (nqt > 1) {
+          if (!wait(&ctrl->s_empty[1], (us[1] & 1u) ^ 1u)) { ok = false; break; }
+          issue_scores(1);
+        }
         tc_commit(smem_u32(&ctrl->qk_empty));        // Q and K may be overwritten once both products retire
         if (!wait(&ctrl->v_full, it & 1u)) { ok = false; break; }
+        const int nj = next_job(job);
         for (int t = 0; t < nqt && ok; ++t) {
           const int kend = min(S_len, (t + 1) * 128), nch = (kend + 63) >> 6;
           if (!wait(&ctrl->o_empty, (oc & 1u) ^ 1u)) { ok = false; break; }
@@ -222,6 +248,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
           if (!ok) break;
           tc_commit(smem_u32(&ctrl->o_full));
           ++oc;
+          // the next job's first score product, as soon as its tiles have landed and this job's S_0 has been
+          // read (never waited for here: the remaining P V work of this job must not queue behind a load)
+          if (t == 0 && !s0_ahead && nj < n_jobs && mbar_test(smem_u32(&ctrl->qk_full), (it + 1u) & 1u) &&
+              mbar_test(smem_u32(&ctrl->s_empty[0]), (us[0] & 1u) ^ 1u)) {
+            issue_scores(0);
+            s0_ahead = true;
+          }
         }
         if (!ok) break;
         tc_commit(smem_u32(&ctrl->v_empty));
@@ -233,8 +266,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
       }
     }
   } else {
-    // ---------------------------------------------------------------- one query row per thread
+    // ---------------------------------------------------------------- two threads per query row
     const int wq = warp & 3;                         // tensor-memory lane quarter of this warp
+    const int half = (warp - 2) >> 2;                // which of the row's two threads: even or odd 32-column chunks
     const int r = wq * 32 + lane;                    // row of the query tile
     const uint32_t lane_base = tmem + ((uint32_t)(wq * 32) << 16);
     uint32_t us[2] = {0u, 0u}, pc = 0, oc = 0;
@@ -244,6 +278,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
       uint32_t good = 1u;
       if (lane == 0) good = wait(bar, parity) ? 1u : 0u;
       return __shfl_sync(0xffffffffu, good, 0) != 0u;
+    };
+    // the two warps of a lane quarter meet (bounded like every other wait: false once the CTA is aborting)
+    uint32_t n_meet = 0;
+    auto pair_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&ctrl->pair[wq]));
+      return warp_wait(&ctrl->pair[wq], n_meet++ & 1u);
     };
     for (int job = blockIdx.x; job < n_jobs && ok; job += gridDim.x) {
       size_t row_base; int S_len, h;
@@ -260,39 +301,62 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
         // key k counts for this row when k <= qpos (causal) and k < S_len (rows past the end of the
         // sequence in the loaded tiles belong to other sequences)
         const int klim = min(qpos, S_len - 1);
-        float m = -INFINITY;
-        for (int j = 0; j < 2 * nch; ++j) {
-          uint32_t v[32];
+        const int klim_lo = min(t * 128 + wq * 32, S_len - 1);        // smallest and largest limit in this warp
+        const int klim_hi = min(t * 128 + wq * 32 + 31, S_len - 1);
+        // this thread owns the 32-column pieces j of the row with j % 2 == half: one half of every 64-key
+        // chunk.  A piece is needed unless the causal mask blanks it for the whole warp (then so are all
+        // later ones).  The loops are kept rolled: ten warps in four roles share one instruction cache.
+        // (four independent running maxima / sums: a single chain of 32 dependent operations would leave the
+        // two warps of a scheduler waiting on arithmetic latency)
+        float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        for (int j = half; j < 2 * nch; j += 4) {    // two pieces per round trip to tensor memory
+          if (j * 32 > klim_hi) break;
+          const bool two = j + 2 < 2 * nch && (j + 2) * 32 <= klim_hi;
+          uint32_t v[32], w[32];
           tc_ld32(scol + j * 32, v);
+          if (two) tc_ld32(scol + (j + 2) * 32, w);
           tc_ld_wait();
+          const int lim = klim - j * 32;             // elements 0 .. lim of the piece count (>= 31: all of them)
 #pragma unroll
-          for (int i = 0; i < 32; ++i)
-            if (j * 32 + i <= klim) m = fmaxf(m, __uint_as_float(v[i]));
+          for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], i <= lim ? __uint_as_float(v[i]) : -INFINITY);
+          if (two) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              m4[i & 3] = fmaxf(m4[i & 3], i + 64 <= lim ? __uint_as_float(w[i]) : -INFINITY);
+          }
         }
+        float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
+        ctrl->xmax[half][r] = m;
+        if (!pair_sync()) { ok = false; break; }
+        m = fmaxf(m, ctrl->xmax[half ^ 1][r]);       // (key 0 counts for every row: the maximum is finite)
         const float ms = m * P.scale_log2e;
-        float l = 0.f;
+        float l4[4] = {0.f, 0.f, 0.f, 0.f};
         for (int c = 0; c < nch && ok; ++c, ++pc) {
           const uint32_t slot = pc & 1u;
           if (!warp_wait(&ctrl->p_empty[slot], ((pc >> 1) & 1u) ^ 1u)) { ok = false; break; }
           uint8_t* prow = smem + L::P_OFF + slot * BOX + r * 128;
+          const int j = 2 * c + half;                // this thread's half of the 64-key chunk
+          uint32_t pk[16];                           // P of the piece, bf16 pairs
+          if (j * 32 > klim_hi) {
 #pragma unroll
-          for (int hh = 0; hh < 2; ++hh) {
-            const int j = 2 * c + hh;
+            for (int i = 0; i < 16; ++i) pk[i] = 0u;
+          } else {
             uint32_t v[32];
             tc_ld32(scol + j * 32, v);
             tc_ld_wait();
-            float p[32];
+            const int lim = klim - j * 32;
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              p[i] = (j * 32 + i <= klim) ? ex2f(fmaf(__uint_as_float(v[i]), P.scale_log2e, -ms)) : 0.f;
-              l += p[i];
+            for (int i = 0; i < 32; i += 2) {
+              const float p0 = i <= lim ? ex2f(fmaf(__uint_as_float(v[i]), P.scale_log2e, -ms)) : 0.f;
+              const float p1 = i + 1 <= lim ? ex2f(fmaf(__uint_as_float(v[i + 1]), P.scale_log2e, -ms)) : 0.f;
+              l4[(i >> 1) & 3] += p0 + p1;
+              pk[i >> 1] = pack_bf16(p0, p1);
             }
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4)           // 16-byte chunk hh*4 + q4 of the row's 128 bytes: keys 8 per chunk
-              *reinterpret_cast<uint4*>(prow + (((hh * 4 + q4) ^ (r & 7)) << 4)) =
-                  make_uint4(pack_bf16(p[8 * q4], p[8 * q4 + 1]), pack_bf16(p[8 * q4 + 2], p[8 * q4 + 3]),
-                             pack_bf16(p[8 * q4 + 4], p[8 * q4 + 5]), pack_bf16(p[8 * q4 + 6], p[8 * q4 + 7]));
           }
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4)             // 16-byte chunk half*4 + q4 of the row's 128 bytes: 8 keys per chunk
+            *reinterpret_cast<uint4*>(prow + (((half * 4 + q4) ^ (r & 7)) << 4)) =
+                make_uint4(pk[4 * q4], pk[4 * q4 + 1], pk[4 * q4 + 2], pk[4 * q4 + 3]);
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&ctrl->p_full[slot]));
@@ -302,25 +366,34 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&ctrl->s_empty[t]));
-        // normalised output of the tile
+        // the even-chunk thread of a row writes the row's output; its partner hands over its share of the sum
+        // (this meeting also orders the tile's reads of xmax before the next tile's writes)
+        float l = (l4[0] + l4[1]) + (l4[2] + l4[3]);
+        if (half) ctrl->xsum[r] = l;
+        if (!pair_sync()) { ok = false; break; }
+        if (half) continue;
+        l += ctrl->xsum[r];
         if (!warp_wait(&ctrl->o_full, oc & 1u)) { ok = false; break; }
         ++oc;
         tc_fence_after();
         const float inv = 1.f / l;
         bf16* orow = P.ctx + (row_base + (size_t)qpos) * P.d + h * DH;
 #pragma unroll
-        for (int j = 0; j < DH / 32; ++j) {
-          uint32_t v[32];
-          tc_ld32(lane_base + 384u + j * 32, v);
+        for (int j = 0; j < DH / 64; ++j) {
+          uint32_t v0[32], v1[32];
+          tc_ld32(lane_base + 384u + j * 64, v0);
+          tc_ld32(lane_base + 384u + j * 64 + 32, v1);
           tc_ld_wait();
           if (qpos < S_len) {
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4)
-              *reinterpret_cast<uint4*>(orow + j * 32 + q4 * 8) = make_uint4(
-                  pack_bf16(__uint_as_float(v[8 * q4]) * inv, __uint_as_float(v[8 * q4 + 1]) * inv),
-                  pack_bf16(__uint_as_float(v[8 * q4 + 2]) * inv, __uint_as_float(v[8 * q4 + 3]) * inv),
-                  pack_bf16(__uint_as_float(v[8 * q4 + 4]) * inv, __uint_as_float(v[8 * q4 + 5]) * inv),
-                  pack_bf16(__uint_as_float(v[8 * q4 + 6]) * inv, __uint_as_float(v[8 * q4 + 7]) * inv));
+            for (int q4 = 0; q4 < 8; ++q4) {
+              const uint32_t* v = q4 < 4 ? v0 + 8 * q4 : v1 + 8 * (q4 - 4);
+              *reinterpret_cast<uint4*>(orow + j * 64 + q4 * 8) = make_uint4(
+                  pack_bf16(__uint_as_float(v[0]) * inv, __uint_as_float(v[1]) * inv),
+                  pack_bf16(__uint_as_float(v[2]) * inv, __uint_as_float(v[3]) * inv),
+                  pack_bf16(__uint_as_float(v[4]) * inv, __uint_as_float(v[5]) * inv),
+                  pack_bf16(__uint_as_float(v[6]) * inv, __uint_as_float(v[7]) * inv));
+            }
           }
         }
         tc_fence_before();
