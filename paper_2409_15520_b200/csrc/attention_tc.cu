@@ -39,6 +39,7 @@ constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 struct Ctrl {
   unsigned long long qk_full, qk_empty, v_full, v_empty, s_full[2], s_empty[2], p_full[2], p_empty[2], o_full, o_empty,
       drain;
+  unsigned long long wait_ns;                       // limit of every bounded wait
   uint32_t tmem_base;
   volatile uint32_t abort;
   unsigned long long pair[4];                       // meeting point of the two warps of a lane quarter
@@ -115,6 +116,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
     mbar_init(smem_u32(&ctrl->drain), 1);
     for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&ctrl->pair[i]), 2);
     ctrl->abort = 0u;
+    ctrl->wait_ns = WAIT_LIMIT_NS;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -129,7 +131,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
   tc_fence_after();
   const uint32_t tmem = ctrl->tmem_base;
   auto wait = [&](unsigned long long* bar, uint32_t parity) {
-    return mbar_wait_bounded(smem_u32(bar), parity, &ctrl->abort, WAIT_LIMIT_NS, P.status);
+    return mbar_wait_bounded(smem_u32(bar), parity, &ctrl->abort, &ctrl->wait_ns, P.status);
   };
   // job -> (first row of the sequence in the replicated buffer, its length, head)
   auto job_of = [&](int job, size_t& row_base, int& S_len, int& h) {

@@ -121,7 +121,7 @@ __constant__ float c_nf4_levels[16] = {-1.0f, -0.6961928009986877f, -0.525073051
 
 // Bounded wait of this kernel's roles (limit and abort flag live in the CTA's control block).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, Ctrl* c, uint32_t* status) {
-  return mbar_wait_bounded(bar, parity, &c->abort, c->wait_ns, status);
+  return mbar_wait_bounded(bar, parity, &c->abort, &c->wait_ns, status);
 }
 __device__ __forceinline__ void ep_bar() { asm volatile("bar.sync 1, %0;" ::"n"(EP_THREADS) : "memory"); }
 // Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128, N = 256.
@@ -179,7 +179,8 @@ __device__ __forceinline__ int tile_slot(const Params& P, int n0) {
 constexpr int FIN_GROUPS = 4;
 // WQ: the B operand is decoded inside the kernel from weight-only quantised codes (instantiated apart so
 // that the decode path costs the bf16 kernels no registers).
-template <bool PAIR, int SPLIT, bool WQ = false>
+// CE: the cross-entropy head (epilogue folds the logits instead of storing them); also its own instantiation.
+template <bool PAIR, int SPLIT, bool WQ = false, bool CE = false>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const __grid_constant__ CUtensorMap tmU, const Params P) {
@@ -747,7 +748,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
       };
       float ce_m = -INFINITY, ce_s = 0.f;          // cross-entropy head: this thread's share of the tile
-      const int ce_lab = (P.ce_part && row_ok) ? P.ce_label[row % P.ce_ep] : -1;
+      int ce_lab = -1;
+      if constexpr (CE) ce_lab = row_ok ? P.ce_label[row % P.ce_ep] : -1;
       for (int c = 0; c < nchunk; ++c) {
         const int col0 = n0 + c * 32;
         if (col0 >= P.N) break;
@@ -856,7 +858,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         if (!row_ok) continue;
-        if (P.ce_part) {
+        if constexpr (CE) {
           float cm = -INFINITY;
 #pragma unroll
           for (int j = 0; j < 32; ++j)
@@ -934,7 +936,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         emit(col0, f);
         if (have2) emit(col0 + po * 32, f2);
       }
-      if (P.ce_part && row_ok) P.ce_part[((size_t)row * tiles_n + tn) * 2 + half] = make_float2(ce_m, ce_s);
+      if constexpr (CE)
+        if (row_ok) P.ce_part[((size_t)row * tiles_n + tn) * 2 + half] = make_float2(ce_m, ce_s);
       // accumulator buffer drained: hand it back to the MMA warp (split K did so when it delivered)
       tc_fence_before();
       __syncwarp();
@@ -1014,6 +1017,12 @@ int gemm_tc_init() {
                              (int)tc::SMEM_BYTES);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<false, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)tc::SMEM_BYTES);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(tc::gemm_tc_kernel<true, 0, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)tc::SMEM_BYTES);
   if (e == cudaSuccess) g_dev_ready[dev].store(true, std::memory_order_release);
   return (int)e;
@@ -1095,7 +1104,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.ksplit = 1; P.part = nullptr;
   P.wfmt = G.wfmt; P.wq = (const uint8_t*)G.wq; P.wscale = G.wscale;
   P.ce_part = (float2*)G.ce_part; P.ce_logit = G.ce_logit; P.ce_label = G.ce_label; P.ce_ep = G.ce_ep;
-  if (G.ce_part && (G.swiglu || G.lora || G.rope_tab || !G.ce_logit || !G.ce_label || G.ce_ep < 1))
+  if (G.ce_part && (G.wfmt || G.swiglu || G.lora || G.rope_tab || !G.ce_logit || !G.ce_label || G.ce_ep < 1))
     return (int)cudaErrorInvalidValue;
   P.wait_ns = G.test_wait_ns ? G.test_wait_ns : tc::WAIT_LIMIT_NS;
   P.withhold = G.test_wait_ns ? 1 : 0;
@@ -1144,6 +1153,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     const int pairs = (int)(tiles2 < max_clusters ? tiles2 : max_clusters);
     cfg.gridDim = dim3(2 * pairs);
     if (!pair_slab_ok) P.slab = 0;
+    if (G.ce_part) return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true, 0, false, true>, tmA, tmB, tmU, P);
     return (int)cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel<true, 0>, tmA, tmB, tmU, P);
   }
   const int tiles_m = (P.M + tc::BM - 1) / tc::BM;
@@ -1169,6 +1179,8 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
     if (G.extra_launches) ++*G.extra_launches;
   } else if (G.wfmt)
     tc::gemm_tc_kernel<false, 0, true><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
+  else if (G.ce_part)
+    tc::gemm_tc_kernel<false, 0, false, true><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
   else
     tc::gemm_tc_kernel<false, 0><<<grid, tc::THREADS, tc::SMEM_BYTES, st>>>(tmA, tmB, tmU, P);
   return (int)cudaGetLastError();

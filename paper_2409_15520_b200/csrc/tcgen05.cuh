@@ -169,9 +169,11 @@ __device__ __forceinline__ void unpack8(const uint4 v, float* f) {
 
 // Bounded wait on an mbarrier phase.  Returns false when the CTA is aborting: this wait ran out of time
 // (it then raises ST_TIMEOUT in the device status word and the CTA's abort flag), or another role of
-// the CTA, or another CTA of the launch, already did.
+// the CTA, or another CTA of the launch, already did.  The limit is read through `limit_ns` only on the
+// slow path: a wait that succeeds at once costs one try_wait and nothing else (the MMA issuer waits once
+// per k-block).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                                  unsigned long long limit_ns, uint32_t* status) {
+                                                  const unsigned long long* limit_ns, uint32_t* status) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = gtimer();
   for (uint32_t it = 1;; ++it) {
@@ -179,7 +181,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
       if (*reinterpret_cast<volatile uint32_t*>(status) & ST_TIMEOUT) { *abort_flag = 1u; return false; }
-      if (gtimer() - t0 > limit_ns) {
+      if (gtimer() - t0 > *reinterpret_cast<const volatile unsigned long long*>(limit_ns)) {
         *abort_flag = 1u;
         atomicOr(status, ST_TIMEOUT);
         return false;
