@@ -278,7 +278,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
     // one lane waits, the warp learns the outcome
     auto warp_wait = [&](unsigned long long* bar, uint32_t parity) -> bool {
       uint32_t good = 1u;
-      if (lane == 0) good = wait(bar, parity) ? 1u : 0u;
+      if (lane == 0)
+        good = mbar_wait_bounded<1>(smem_u32(bar), parity, &ctrl->abort, &ctrl->wait_ns, P.status) ? 1u : 0u;
       return __shfl_sync(0xffffffffu, good, 0) != 0u;
     };
     // the two warps of a lane quarter meet (bounded like every other wait: false once the CTA is aborting)

@@ -171,6 +171,15 @@ __device__ __forceinline__ int tile_slot(const Params& P, int n0) {
   return P.slab ? P.L.slot_of_sec[n0 / P.L.width] : -1;
 }
 
+// Position in the operand ring: stage and phase advance by counting, so the per-k-block path of the
+// producer, the MMA issuer and the decode warps carries no division (the stage count is a run-time value).
+struct RingPos {
+  uint32_t s = 0, ph = 0;
+  __device__ __forceinline__ void advance(uint32_t stages) {
+    if (++s == stages) { s = 0; ph ^= 1u; }
+  }
+};
+
 // SPLIT 0: every CTA (pair) computes whole tiles.  Split K, for launches with far fewer tiles than SMs
 // whose cost is the stream of weights (small batches), takes two launches of this kernel: SPLIT 1
 // computes one K range of a tile per unit of work and stores the fp32 accumulator to scratch; SPLIT 2
@@ -277,6 +286,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0 && SPLIT != 2) {
       uint32_t issued = 0;
+      RingPos rp;
       bool ok = true, withheld = false;
       for (int tile = t_first; tile < t_end && ok && !withheld; tile += t_step) {
         int tm, tn;
@@ -286,11 +296,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int brow1 = P.swiglu ? P.N + brow0 : brow0 + 128;
         int ks, kb0, kb1;
         kb_range(tile, ks, kb0, kb1);
-        for (int kb = kb0; kb < kb1; ++kb, ++issued) {
+        for (int kb = kb0; kb < kb1; ++kb, ++issued, rp.advance(STAGES)) {
           // failure-detection test: this producer goes silent (nothing armed, nothing in flight), so the
           // MMA warp's wait for the stage runs out and the CTA takes its abort path
           if (!PAIR && P.withhold && blockIdx.x == 0 && issued == (kb1 - kb0 > 1 ? 1u : 0u)) { withheld = true; break; }
-          const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
+          const uint32_t s = rp.s, ph = rp.ph;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
           const uint32_t sa = tiles_base + s * STAGE_BYTES;
@@ -310,9 +320,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         const int lslot = ks != 0 ? -1 : tile_slot(P, brow0);   // the LoRA block rides with the first K range
-        for (int lkb = 0; ok && !withheld && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued) {
+        for (int lkb = 0; ok && !withheld && lslot >= 0 && lkb < P.kslot / BK; ++lkb, ++issued, rp.advance(STAGES)) {
           // LoRA k-blocks: only the A operand (packed U) travels through the ring
-          const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
+          const uint32_t s = rp.s, ph = rp.ph;
           if (!mbar_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u, ctrl, P.status)) { ok = false; break; }
           const uint32_t bar = smem_u32(&ctrl->full[s]);
           if (PAIR) {
@@ -335,7 +345,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && rank == 0 && SPLIT != 2) {
-      uint32_t consumed = 0, titer = 0, ltiles = 0;
+      uint32_t titer = 0, ltiles = 0;
+      RingPos rp;
+      const uint32_t idesc_main = PAIR ? IDESC_PAIR : (P.n_half ? IDESC_N128 : IDESC);
       bool ok = true;
       for (int tile = t_first; tile < t_end && ok; tile += t_step, ++titer) {
         const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -344,8 +356,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const uint32_t d_tmem = tmem_base + a * BN;
         int ks, kb0, kb1;
         kb_range(tile, ks, kb0, kb1);
-        for (int kb = kb0; kb < kb1; ++kb, ++consumed) {
-          const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
+        for (int kb = kb0; kb < kb1; ++kb, rp.advance(STAGES)) {
+          const uint32_t s = rp.s, ph = rp.ph;
           if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = tiles_base + s * STAGE_BYTES;
@@ -353,10 +365,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
           for (int k = 0; k < BK / 16; ++k) {
             if (PAIR)
-              tc_mma_pair(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), IDESC_PAIR,
+              tc_mma_pair(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), idesc_main,
                           (uint32_t)(((kb - kb0) | k) != 0));
             else
-              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), P.n_half ? IDESC_N128 : IDESC,
+              tc_mma(d_tmem, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), idesc_main,
                      (uint32_t)(((kb - kb0) | k) != 0));
           }
           // frees the stage (in both CTAs of a pair) once these MMAs retire
@@ -367,8 +379,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           int tm, tn;
           coords(tile, tm, tn);
           if (ks == 0 && tile_slot(P, tn * ncol_tile) >= 0) {
-            for (int lkb = 0; lkb < P.kslot / BK; ++lkb, ++consumed) {
-              const uint32_t s = consumed % STAGES, ph = (consumed / STAGES) & 1u;
+            for (int lkb = 0; lkb < P.kslot / BK; ++lkb, rp.advance(STAGES)) {
+              const uint32_t s = rp.s, ph = rp.ph;
               if (!mbar_wait(smem_u32(&ctrl->full[s]), ph, ctrl, P.status) ||
                   (lkb == 0 && !mbar_wait(smem_u32(&ctrl->lfull), ltiles & 1u, ctrl, P.status))) { ok = false; break; }
               tc_fence_after();
@@ -465,7 +477,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // writes each k-block as eight 16-byte chunks of bf16 into the stage, in the swizzled K-major layout
     // of the TMA path.  One fp32 product and one rounding per weight, as the stand-alone decoder does.
     // The warps run independently (each polls the barriers itself, one lane per warp).
-    uint32_t dissued = 0;                            // stages used so far (mirrors the TMA producer's count)
+    RingPos dq;                                      // ring position (mirrors the TMA producer's)
     uint32_t rgroups = 0;                            // code groups consumed so far (slot and phase of the ring)
     bool dq_ok = true;                               // this warp's waits so far succeeded
     auto warp_wait = [&](uint32_t bar, uint32_t parity) -> bool {   // one lane waits, all lanes learn the outcome
@@ -522,7 +534,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int gi = 0; gi < 4; ++gi) {
           const int kb = g0 + gi;
           if (gi < DQ_G && kb < kb1 && dq_ok) {       // uniform over the warp
-            const uint32_t s = dissued % STAGES, ph = (dissued / STAGES) & 1u;
+            const uint32_t s = dq.s, ph = dq.ph;
             dq_ok = warp_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u);
             if (dq_ok) {
               uint8_t* brow = smem + s * STAGE_BYTES + A_BYTES + et * 128;
@@ -572,7 +584,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the tensor core
               __syncwarp();
               if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
-              ++dissued;
+              dq.advance(STAGES);
             }
           }
         }
@@ -585,11 +597,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // the LoRA k-blocks of the unit bring only their A operand through the ring: arrive for the stage
       if (ks == 0 && tile_slot(P, brow0) >= 0) {
         for (int lkb = 0; lkb < P.kslot / BK && dq_ok; ++lkb) {
-          const uint32_t s = dissued % STAGES, ph = (dissued / STAGES) & 1u;
+          const uint32_t s = dq.s, ph = dq.ph;
           dq_ok = warp_wait(smem_u32(&ctrl->empty[s]), ph ^ 1u);
           if (dq_ok) {
             if (lane == 0) mbar_arrive(smem_u32(&ctrl->full[s]));
-            ++dissued;
+            dq.advance(STAGES);
           }
         }
       }

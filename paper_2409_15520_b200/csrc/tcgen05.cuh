@@ -172,9 +172,16 @@ __device__ __forceinline__ void unpack8(const uint4 v, float* f) {
 // the CTA, or another CTA of the launch, already did.  The limit is read through `limit_ns` only on the
 // slow path: a wait that succeeds at once costs one try_wait and nothing else (the MMA issuer waits once
 // per k-block).
+// FAST polls are made before the clock is read for the first time: the waits of a producer or an MMA issuer
+// sit on the latency chain of an operand ring and the global timer is a slow register, so they poll a few
+// times first; warps that share a scheduler with working warps keep FAST = 1, where the slow read doubles
+// as a back-off.
+template <int FAST = 16>
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
                                                   const unsigned long long* limit_ns, uint32_t* status) {
-  if (mbar_try(bar, parity)) return true;
+#pragma unroll 1
+  for (int i = 0; i < FAST; ++i)
+    if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = gtimer();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try(bar, parity)) return true;
