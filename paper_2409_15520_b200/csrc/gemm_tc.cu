@@ -431,7 +431,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int repg = P.L.rep_base + P.L.rep_stride * ((tm * TILE_M) / P.L.rows_per_replica);
       const int kgroups = (P.L.r + 7) / 8;
       constexpr int CQ = PAIR ? 32 : 64;               // column quads of the operand rows this CTA holds
-      for (int unit_i = et; unit_i < CQ * kgroups; unit_i += EP_THREADS) {
+      // the operand is generated by the four epilogue warps that share no scheduler with the TMA producer
+      // (warp 0) and the MMA issuer (warp 1): the Philox / Box-Muller bursts then cost those two no issue
+      // slots, and their waits sit on the latency chain of the operand ring
+      const int gen_i = (warp & 2) ? ((warp >> 2) & 1) * 64 + (warp & 1) * 32 + lane : -1;   // warps 2, 3, 6, 7
+      for (int unit_i = gen_i; unit_i >= 0 && unit_i < CQ * kgroups; unit_i += EP_THREADS / 2) {
         const int c4l = (unit_i % CQ) * 4, k0 = (unit_i / CQ) * 8;
         const int c4 = c4l + (PAIR ? (int)rank * 128 : 0);       // column inside the 256-column tile
         float bb[8][4], zz[8][4];
