@@ -1064,6 +1064,21 @@ int tc_make_map_bf16(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows,
   return make_map(m, ptr, K, rows, pitch_elems);
 }
 
+int tc_make_map_bf16_nd(CUtensorMap* m, const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                        const uint32_t* box) {
+  if (!g_encode) {
+    const int e = gemm_tc_init();
+    if (e) return e;
+  }
+  cuuint64_t d[3], st[2];
+  cuuint32_t b[3], es[3] = {1u, 1u, 1u};
+  for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; }
+  for (int i = 0; i + 1 < rank; ++i) st[i] = strides_bytes[i];
+  return (int)g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(ptr), d, st, b, es,
+                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
 // 2-D byte tensor map over quantised codes: rows x row_bytes, box 128 rows x 128 bytes, 128-byte swizzle.
 static int make_code_map(CUtensorMap* m, const void* ptr, uint64_t row_bytes, uint64_t rows) {
   const cuuint64_t dims[2] = {row_bytes, rows};

@@ -103,10 +103,11 @@ void launch_lora_apply(cudaStream_t st, int bf, const void* base, int ldb, int b
 // Shared-input expansion on the bf16 path: out[j, t, :] = base[t, :] + s U[t, :] (B + k eps z) for the n
 // replicas of a pass (base and U on the T shared rows; out rows j * rows_per_replica + t), written with
 // full-line stores.  Supported when every section is a multiple of 128 columns, r <= 64 and rows are
-// 16-byte aligned.
+// 16-byte aligned.  Rank <= 16 moves its tiles with bulk tensor copies, whose bounded waits report to
+// the device status word.
 bool lora_expand_supported(const void* base, int ldb, const void* out, int ldo, const LoraDesc& L);
 void launch_lora_expand(cudaStream_t st, const void* base, int ldb, void* out, int ldo, int n, int T,
-                        const LoraDesc& L, int nsec, int n_sms);
+                        const LoraDesc& L, int nsec, int n_sms, uint32_t* status);
 void launch_rope_table(cudaStream_t st, float* tab, int max_seq, int dh, float theta);
 void launch_rope(cudaStream_t st, int bf, void* qkv, int rows, int Tp, SeqLayout sl, int d, int H,
                  const float* tab);

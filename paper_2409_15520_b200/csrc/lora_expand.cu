@@ -12,12 +12,34 @@
 #include "kernels.h"
 #include "lora_operand.cuh"
 #include "mma.cuh"
+#include "tcgen05.cuh"
 
 namespace zo {
 namespace {
 
 constexpr int XT = 128;                 // rows and columns of one tile
 constexpr int LDC = XT + 8;             // pitch of a staged base/output tile (elements)
+
+// Row tiles one CTA sweeps.  Two CTAs fit an SM, so the grid runs in waves of 2 n_sms CTAs; a (replica,
+// column tile) pair swept whole by one CTA leaves the last wave mostly empty at the usual shapes
+// (672 pairs on 296 places: 2.3 waves).  The sweep is cut into equal parts: the longest part (the
+// generated operand is amortised over it) whose waves are at least 93 % full, else the fullest cut.
+int tiles_per_cta(int pairs, int ntile, int n_sms) {
+  const long long wave = 2LL * n_sms;
+  int best = ntile;
+  double best_eff = 0.0;
+  for (int z = 1; z <= ntile; ++z) {
+    const int per = (ntile + z - 1) / z, parts = (ntile + per - 1) / per;
+    const long long waves = ((long long)pairs * parts + wave - 1) / wave;
+    const double eff = (double)pairs * ntile / (double)wave / ((double)per * (double)waves);
+    if (eff >= 0.93) return per;
+    if (eff > best_eff) {
+      best_eff = eff;
+      best = per;
+    }
+  }
+  return best;
+}
 
 template <int KT>                       // K extent of the generated operand (>= 2r, multiple of 16)
 __global__ void __launch_bounds__(256, 2)
@@ -156,18 +178,239 @@ lora_expand_kernel(const bf16* __restrict__ base, int ldb, bf16* __restrict__ ou
   cp_wait<0>();
 }
 
+
+// ---- rank <= 16: bulk-tensor form ------------------------------------------------------------------
+// The same operation with the tile traffic taken off the load/store pipe.  A warp owns 32 rows x 64
+// columns of each 128 x 128 tile (one 4 KB box, 128-byte swizzle) and runs a private pipeline on it:
+// a bulk tensor load brings the base rows (rows beyond T arrive as zeros), the warp reads them once in
+// accumulator-fragment order (ldmatrix), adds the rank-2r product [U|U] x operand (m16n8k16, fp32
+// accumulate, operand fragments held in registers for the whole sweep), rounds once to bf16, writes
+// the block back in place (stmatrix) and hands the box to a bulk tensor store (rows beyond T of the
+// replica are clipped by the 3-D map).  Three boxes per warp: one being loaded, one in work, one being
+// stored.  Waits on the load barriers are bounded.
+constexpr int WR = 32, WC = 64;         // rows and columns of a warp's box
+constexpr int NBOX = 3;
+constexpr uint32_t BOX_BYTES = WR * WC * 2;
+
+struct ExpandCtrl {
+  unsigned long long full[8][NBOX];
+  unsigned long long wait_ns;
+  uint32_t abort_flag;
+};
+
+template <int KT, bool DUP>          // DUP: 2r == KT, the two halves of [U|U] are the same registers
+__global__ void __launch_bounds__(256, 2)
+lora_expand_tma_kernel(const __grid_constant__ CUtensorMap base_map, const __grid_constant__ CUtensorMap out_map,
+                       int T, LoraDesc L, int tiles_per_cta, unsigned long long wait_ns, uint32_t* status) {
+  constexpr int LDB = KT + 8;
+  constexpr int NKS = KT / 16;
+  extern __shared__ uint8_t sm_dyn[];
+  uint8_t* boxes = sm_dyn + ((1024u - (tc::smem_u32(sm_dyn) & 1023u)) & 1023u);   // [8 warps][NBOX][4 KB], 1024-byte aligned
+  bf16* Bs = reinterpret_cast<bf16*>(boxes + 8 * NBOX * BOX_BYTES);   // [XT columns][LDB]: operand, K contiguous
+  ExpandCtrl* ctl = reinterpret_cast<ExpandCtrl*>(Bs + XT * LDB);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int wr0 = (warp >> 1) * WR, wc0 = (warp & 1) * WC;
+  const int col0 = blockIdx.x * XT;
+  const int sec = col0 / L.width, cs = col0 - sec * L.width;
+  const int slot = sec == 0 ? L.slot_of_sec[0] : (sec == 1 ? L.slot_of_sec[1] : L.slot_of_sec[2]);
+  const int n = blockIdx.y;
+  const int r = L.r;
+  const int ntile = (T + XT - 1) / XT;
+  const int tile0 = blockIdx.z * tiles_per_cta;
+  // the warp's last tile is the last one whose first row of the warp's share exists
+  const int tile1 = min(min(ntile, tile0 + tiles_per_cta), (T - wr0 + XT - 1) / XT);
+
+  const uint32_t box0 = tc::smem_u32(boxes + (size_t)warp * NBOX * BOX_BYTES);
+  const uint32_t bar0 = tc::smem_u32(&ctl->full[warp][0]);
+  if (threadIdx.x == 0) {
+    ctl->wait_ns = wait_ns;
+    ctl->abort_flag = 0u;
+  }
+  if (lane == 0) {
+#pragma unroll
+    for (int b = 0; b < NBOX; ++b) tc::mbar_init(bar0 + 8 * b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (tile0 < tile1) {
+      tc::mbar_expect_tx(bar0, BOX_BYTES);
+      tc::tma_load_2d(box0, &base_map, col0 + wc0, tile0 * XT + wr0, bar0);
+    }
+  }
+
+  if (slot >= 0) {
+    // operand of this (replica, column tile): K index k holds s B[k, col], K index r + k holds
+    // s k_n eps z[k, col]; the rest of the K extent is zero
+    for (int i = threadIdx.x; i < XT * LDB / 8; i += 256) reinterpret_cast<uint4*>(Bs)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+    const int rid = L.rep_base + L.rep_stride * n;
+    for (int i = threadIdx.x; i < r * (XT / 4); i += 256) {
+      const int k = i / (XT / 4), c4 = (i % (XT / 4)) * 4;
+      float4 b, z;
+      lora_operand(L, slot, (size_t)k * L.width + cs + c4, rid, b, z);
+      const float bb[4] = {b.x, b.y, b.z, b.w}, zz[4] = {z.x, z.y, z.z, z.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        Bs[(c4 + j) * LDB + k] = __float2bfloat16_rn(bb[j] * L.scale);
+        Bs[(c4 + j) * LDB + r + k] = __float2bfloat16_rn(zz[j] * L.scale);
+      }
+    }
+  }
+  __syncthreads();                                     // operand and control words complete
+  if (tile0 >= tile1) return;
+
+  // operand fragments of the warp's 64 columns: [k-step][pair of 8-column tiles] -> {b0, b1 | b0, b1}
+  uint32_t bfrag[NKS][WC / 16][4];
+  if (slot >= 0) {
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks)
+#pragma unroll
+      for (int jp = 0; jp < WC / 16; ++jp) {
+        const int col = wc0 + jp * 16 + (lane & 7) + (lane >> 4) * 8;
+        const int c = ks * 16 + ((lane >> 3) & 1) * 8;
+        ldsm_x4(tc::smem_u32(Bs + col * LDB + c), bfrag[ks][jp][0], bfrag[ks][jp][1], bfrag[ks][jp][2],
+                bfrag[ks][jp][3]);
+      }
+  }
+
+  // A = [U | U | 0] of the warp's two 16-row blocks in the fragment order of the m16n8k16 A operand.
+  // With 2r == KT every fragment register is one aligned pair of U (rows g and g + 8, columns 2t and
+  // 8 + 2t of each 16-wide group; the second half of the K extent repeats the first), fetched one tile
+  // ahead as raw fp32 pairs and rounded to bf16 when its tile comes up.  Other ranks gather by element.
+  // Rows beyond T repeat row T - 1: their outputs are clipped by the store.
+  constexpr int NU = KT / 8;                           // distinct fragment registers of a 16-row block
+  float2 raw[2][DUP ? NU : 1];
+  auto fetch_u = [&](int tile) {
+#pragma unroll
+    for (int mb = 0; mb < 2; ++mb) {
+      const int ra = tile * XT + wr0 + mb * 16 + g;
+      const float* ua = L.U + (size_t)min(ra, T - 1) * L.ldu + slot * r + 2 * t;
+      const float* ub = L.U + (size_t)min(ra + 8, T - 1) * L.ldu + slot * r + 2 * t;
+#pragma unroll
+      for (int j = 0; j < NU / 2; ++j) {
+        raw[mb][2 * j] = *reinterpret_cast<const float2*>(ua + 8 * j);
+        raw[mb][2 * j + 1] = *reinterpret_cast<const float2*>(ub + 8 * j);
+      }
+    }
+  };
+  auto load_a = [&](int tile, int mb, uint32_t (&af)[NKS][4]) {
+    const int ra = tile * XT + wr0 + mb * 16 + g, rb = ra + 8;
+    const float* ua = L.U + (size_t)min(ra, T - 1) * L.ldu + slot * r;
+    const float* ub = L.U + (size_t)min(rb, T - 1) * L.ldu + slot * r;
+    auto aval = [&](const float* u, int kk) -> float { return kk < 2 * r ? u[kk < r ? kk : kk - r] : 0.f; };
+#pragma unroll
+    for (int ks = 0; ks < NKS; ++ks) {
+      const int k0 = ks * 16 + 2 * t;
+      af[ks][0] = pack2(aval(ua, k0), aval(ua, k0 + 1));
+      af[ks][1] = pack2(aval(ub, k0), aval(ub, k0 + 1));
+      af[ks][2] = pack2(aval(ua, k0 + 8), aval(ua, k0 + 9));
+      af[ks][3] = pack2(aval(ub, k0 + 8), aval(ub, k0 + 9));
+    }
+  };
+  if (DUP && slot >= 0) fetch_u(tile0);
+
+  // lane's 16-byte cell of a 16 x 16 block at (row block mb, column pair jp) inside a swizzled box:
+  // row = mb*16 + (lane & 15), 16-byte chunk = 2 jp + (lane >> 4), chunk index XORed with row & 7
+  const int lrow = lane & 15, lchunk = lane >> 4;
+  int b = 0;                                           // box of the current tile
+  uint32_t ph = 0;                                     // its barrier phase
+  for (int tile = tile0; tile < tile1; ++tile) {
+    const int nb = b + 1 == NBOX ? 0 : b + 1;
+    if (lane == 0 && tile + 1 < tile1) {
+      tc::tma_store_wait_read<1>();                    // the store that last used box nb (two tiles back) has read it
+      tc::mbar_expect_tx(bar0 + 8 * nb, BOX_BYTES);
+      tc::tma_load_2d(box0 + nb * BOX_BYTES, &base_map, col0 + wc0, (tile + 1) * XT + wr0, bar0 + 8 * nb);
+    }
+    uint32_t af[2][NKS][4];
+    if (slot >= 0) {
+      if constexpr (DUP) {
+#pragma unroll
+        for (int mb = 0; mb < 2; ++mb)
+#pragma unroll
+          for (int ks = 0; ks < NKS; ++ks)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float2 v = raw[mb][(ks * 4 + i) % NU];
+              af[mb][ks][i] = pack2(v.x, v.y);
+            }
+        if (tile + 1 < tile1) fetch_u(tile + 1);       // in flight under this tile's arithmetic
+      } else {
+        load_a(tile, 0, af[0]);
+        load_a(tile, 1, af[1]);
+      }
+    }
+    if (!tc::mbar_wait_bounded(bar0 + 8 * b, ph, &ctl->abort_flag, &ctl->wait_ns, status)) break;
+    const uint32_t box = box0 + b * BOX_BYTES;
+    if (slot >= 0) {
+#pragma unroll
+      for (int mb = 0; mb < 2; ++mb) {
+#pragma unroll
+        for (int jp = 0; jp < WC / 16; ++jp) {
+          const int row = mb * 16 + lrow;
+          const uint32_t caddr = box + row * 128 + (((2 * jp + lchunk) ^ (row & 7)) << 4);
+          uint32_t c0, c1, c2, c3;
+          ldsm_x4(caddr, c0, c1, c2, c3);
+          float a0[4] = {__uint_as_float(c0 << 16), __uint_as_float(c0 & 0xFFFF0000u),
+                         __uint_as_float(c1 << 16), __uint_as_float(c1 & 0xFFFF0000u)};
+          float a1[4] = {__uint_as_float(c2 << 16), __uint_as_float(c2 & 0xFFFF0000u),
+                         __uint_as_float(c3 << 16), __uint_as_float(c3 & 0xFFFF0000u)};
+#pragma unroll
+          for (int ks = 0; ks < NKS; ++ks) {
+            if (ks * 16 >= 2 * r) break;               // nothing but zeros from here on
+            mma_bf16(a0, af[mb][ks][0], af[mb][ks][1], af[mb][ks][2], af[mb][ks][3], bfrag[ks][jp][0],
+                     bfrag[ks][jp][1]);
+            mma_bf16(a1, af[mb][ks][0], af[mb][ks][1], af[mb][ks][2], af[mb][ks][3], bfrag[ks][jp][2],
+                     bfrag[ks][jp][3]);
+          }
+          stsm_x4(caddr, pack2(a0[0], a0[1]), pack2(a0[2], a0[3]), pack2(a1[0], a1[1]), pack2(a1[2], a1[3]));
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the block as the bulk store will read it
+    }
+    __syncwarp();
+    if (lane == 0) {
+      tc::tma_store_3d(&out_map, col0 + wc0, tile * XT + wr0, n, box);
+      tc::tma_store_commit();
+    }
+    if (nb == 0) ph ^= 1u;
+    b = nb;
+  }
+  if (lane == 0) tc::tma_store_wait_read<0>();         // shared memory stays until the last store has read it
+}
+
+template <int KT, bool DUP>
+int launch_tma(cudaStream_t st, const void* base, int ldb, void* out, int ldo, int n, int T, const LoraDesc& L,
+               int nsec, int n_sms, unsigned long long wait_ns, uint32_t* status) {
+  const uint64_t ncols = (uint64_t)nsec * L.width;
+  CUtensorMap bm, om;
+  {
+    const uint64_t dims[2] = {ncols, (uint64_t)T}, strides[1] = {(uint64_t)ldb * 2};
+    const uint32_t box[2] = {WC, WR};
+    if (tc_make_map_bf16_nd(&bm, base, 2, dims, strides, box)) return 1;
+  }
+  {
+    const uint64_t dims[3] = {ncols, (uint64_t)T, (uint64_t)n};
+    const uint64_t strides[2] = {(uint64_t)ldo * 2, (uint64_t)L.rows_per_replica * ldo * 2};
+    const uint32_t box[3] = {WC, WR, 1};
+    if (tc_make_map_bf16_nd(&om, out, 3, dims, strides, box)) return 1;
+  }
+  const size_t smem = 8 * NBOX * BOX_BYTES + (size_t)XT * (KT + 8) * sizeof(bf16) + sizeof(ExpandCtrl) + 1024;
+  cudaFuncSetAttribute(lora_expand_tma_kernel<KT, DUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const int ctiles = (int)(ncols / XT), ntile = (T + XT - 1) / XT;
+  const int per = tiles_per_cta(ctiles * n, ntile, n_sms);
+  dim3 grid(ctiles, n, (ntile + per - 1) / per);
+  lora_expand_tma_kernel<KT, DUP><<<grid, 256, smem, st>>>(bm, om, T, L, per, wait_ns, status);
+  return 0;
+}
+
 template <int KT>
 void launch_t(cudaStream_t st, const void* base, int ldb, void* out, int ldo, int n, int T,
               const LoraDesc& L, int nsec, int n_sms) {
   const size_t smem = (size_t)(XT * (KT + 8) + 2 * XT * LDC) * sizeof(bf16);
   cudaFuncSetAttribute(lora_expand_kernel<KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   const int ctiles = nsec * L.width / XT, ntile = (T + XT - 1) / XT;
-  // enough CTAs for a few waves; beyond that, longer row sweeps amortise the generated operand
-  int z = (4 * n_sms + ctiles * n - 1) / (ctiles * n);
-  z = z < 1 ? 1 : (z > ntile ? ntile : z);
-  const int per = (ntile + z - 1) / z;
-  z = (ntile + per - 1) / per;
-  dim3 grid(ctiles, n, z);
+  const int per = tiles_per_cta(ctiles * n, ntile, n_sms);
+  dim3 grid(ctiles, n, (ntile + per - 1) / per);
   lora_expand_kernel<KT><<<grid, 256, smem, st>>>((const bf16*)base, ldb, (bf16*)out, ldo, T, L, per);
 }
 
@@ -179,8 +422,16 @@ bool lora_expand_supported(const void* base, int ldb, const void* out, int ldo, 
 }
 
 void launch_lora_expand(cudaStream_t st, const void* base, int ldb, void* out, int ldo, int n, int T,
-                        const LoraDesc& L, int nsec, int n_sms) {
+                        const LoraDesc& L, int nsec, int n_sms, uint32_t* status) {
   if (n <= 0 || T <= 0) return;
+  if (L.r <= 16 && status != nullptr) {                // bulk-tensor form; the form below if a map cannot be made
+    int e;
+    if (L.r == 8) e = launch_tma<16, true>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms, 2000000000ull, status);
+    else if (L.r == 16) e = launch_tma<32, true>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms, 2000000000ull, status);
+    else if (L.r < 8) e = launch_tma<16, false>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms, 2000000000ull, status);
+    else e = launch_tma<32, false>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms, 2000000000ull, status);
+    if (e == 0) return;
+  }
   if (L.r <= 8) launch_t<16>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms);
   else if (L.r <= 16) launch_t<32>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms);
   else if (L.r <= 32) launch_t<64>(st, base, ldb, out, ldo, n, T, L, nsec, n_sms);

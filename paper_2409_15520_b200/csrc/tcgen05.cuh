@@ -11,6 +11,10 @@ namespace zo {
 // 2-D bf16 tensor map (host): rows x K elements with K contiguous and a row pitch of pitch_elems; boxes of
 // 128 rows x 64 columns, 128-byte swizzle, out-of-range elements read as zero.  0 = ok.
 int tc_make_map_bf16(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, uint64_t pitch_elems);
+// General bf16 tensor map (host) of rank 2 or 3 with the 128-byte swizzle: dims / box in elements (innermost
+// first, inner box 64), strides in bytes for dimensions 1 and 2.  0 = ok.
+int tc_make_map_bf16_nd(CUtensorMap* m, const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                        const uint32_t* box);
 
 namespace tc {
 
@@ -68,6 +72,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       " [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
+}
+// Bulk tensor store shared -> global (3-D map; out-of-range coordinates are clipped), tracked by bulk groups.
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, int x, int y, int z, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(map), "r"(x),
+               "r"(y), "r"(z), "r"(src)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// waits until at most N of this thread's bulk groups still have to READ their shared-memory source
+template <int N> __device__ __forceinline__ void tma_store_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
 // Pair variant: data lands in this CTA's shared memory, completion is signalled on the barrier
 // at the same offset in the leader (even-ranked) CTA.  No multicast.

@@ -417,7 +417,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
   L.rep_base = ps.base; L.rep_stride = ps.stride;
   if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && lora_expand_supported(base, ko, Y, ko, L)) {
-    PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, base, ko, Y, ko, n, T, L, 1, c->n_sms));
+    PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, base, ko, Y, ko, n, T, L, 1, c->n_sms, status));
   } else {
     PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
   }
@@ -532,7 +532,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(G);
       if (tcore && lora_expand_supported(qkv0, 3 * d, qkv, 3 * d, L)) {
         // expansion to the 2q outputs of the pass: bound by the output stream, full-line stores
-        PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, qkv0, 3 * d, qkv, 3 * d, n, T, L, 3, c->n_sms));
+        PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, qkv0, 3 * d, qkv, 3 * d, n, T, L, 3, c->n_sms, status));
       } else {
         PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
       }
@@ -1020,7 +1020,7 @@ static zo_status mp_lora_linear_impl(void* cuda_stream, int32_t precision, const
     s = run_gemm(nullptr, st, bf, flags, G, status, sms, &launches, err, sizeof(err));
     if (s) return s;
     if (bf && !(flags & ZO_FLAG_SIMT_GEMM) && lora_expand_supported(base, k_out, Y, k_out, L)) {
-      launch_lora_expand(st, base, k_out, Y, k_out, n, T, L, 1, sms);
+      launch_lora_expand(st, base, k_out, Y, k_out, n, T, L, 1, sms, status);
     } else {
       launch_lora_apply(st, bf, base, k_out, 1, Y, k_out, n, T, L, 1);
     }
