@@ -51,10 +51,10 @@ lora_expand_kernel(const bf16* __restrict__ base, int ldb, bf16* __restrict__ ou
   bf16* Cs = Bs + XT * LDB;                            // [2][XT rows][LDC]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
-  const int col0 = blockIdx.x * XT;
+  const int col0 = blockIdx.y * XT;
   const int sec = col0 / L.width, cs = col0 - sec * L.width;
   const int slot = sec == 0 ? L.slot_of_sec[0] : (sec == 1 ? L.slot_of_sec[1] : L.slot_of_sec[2]);   // uniform over the CTA
-  const int n = blockIdx.y;
+  const int n = blockIdx.x;   // replicas of one base tile are neighbours in launch order: the tile comes from DRAM once
   const int Tp = L.rows_per_replica, r = L.r;
   const int ntile = (T + XT - 1) / XT;
   const int tile0 = blockIdx.z * tiles_per_cta, tile1 = min(ntile, tile0 + tiles_per_cta);
@@ -211,10 +211,10 @@ lora_expand_tma_kernel(const __grid_constant__ CUtensorMap base_map, const __gri
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
   const int wr0 = (warp >> 1) * WR, wc0 = (warp & 1) * WC;
-  const int col0 = blockIdx.x * XT;
+  const int col0 = blockIdx.y * XT;
   const int sec = col0 / L.width, cs = col0 - sec * L.width;
   const int slot = sec == 0 ? L.slot_of_sec[0] : (sec == 1 ? L.slot_of_sec[1] : L.slot_of_sec[2]);
-  const int n = blockIdx.y;
+  const int n = blockIdx.x;   // replicas of one base tile are neighbours in launch order: the tile comes from DRAM once
   const int r = L.r;
   const int ntile = (T + XT - 1) / XT;
   const int tile0 = blockIdx.z * tiles_per_cta;
@@ -398,7 +398,7 @@ int launch_tma(cudaStream_t st, const void* base, int ldb, void* out, int ldo, i
   cudaFuncSetAttribute(lora_expand_tma_kernel<KT, DUP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   const int ctiles = (int)(ncols / XT), ntile = (T + XT - 1) / XT;
   const int per = tiles_per_cta(ctiles * n, ntile, n_sms);
-  dim3 grid(ctiles, n, (ntile + per - 1) / per);
+  dim3 grid(n, ctiles, (ntile + per - 1) / per);
   lora_expand_tma_kernel<KT, DUP><<<grid, 256, smem, st>>>(bm, om, T, L, per, wait_ns, status);
   return 0;
 }
@@ -410,7 +410,7 @@ void launch_t(cudaStream_t st, const void* base, int ldb, void* out, int ldo, in
   cudaFuncSetAttribute(lora_expand_kernel<KT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   const int ctiles = nsec * L.width / XT, ntile = (T + XT - 1) / XT;
   const int per = tiles_per_cta(ctiles * n, ntile, n_sms);
-  dim3 grid(ctiles, n, (ntile + per - 1) / per);
+  dim3 grid(n, ctiles, (ntile + per - 1) / per);
   lora_expand_kernel<KT><<<grid, 256, smem, st>>>((const bf16*)base, ldb, (bf16*)out, ldo, T, L, per);
 }
 
