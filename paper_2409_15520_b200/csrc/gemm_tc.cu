@@ -210,8 +210,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   // quantised weights: two slots of raw codes (a group of k-blocks: 256 rows x 128 bytes each) behind the slab area
   constexpr uint32_t RAW_BYTES = 2 * BOX_BYTES;
   uint8_t* raw_ring = smem + STAGES * STAGE_BYTES + (P.kslot > 64 ? 2 : 1) * SLAB_BYTES;
-  // NF4: code byte -> (level of its high nibble, level of its low nibble): one 8-byte look-up per two weights
-  float2* nf4_pairs = reinterpret_cast<float2*>(raw_ring + 2 * RAW_BYTES);
   const uint32_t tiles_base = smem_u32(smem);
   const uint32_t rank = PAIR ? cluster_rank() : 0u;    // 0 = leader of the pair
   const int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
@@ -259,8 +257,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (WQ)
-    for (int i = threadIdx.x; i < 256; i += THREADS) nf4_pairs[i] = make_float2(c_nf4_levels[i >> 4], c_nf4_levels[i & 15]);
   if (warp == 1 && SPLIT != 2) {
     if (PAIR) {
       asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(
@@ -544,25 +540,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
               uint8_t* brow = smem + s * STAGE_BYTES + A_BYTES + et * 128;
               if (!(P.n_half && et >= 128)) {
                 if (nf4) {
+                  // The 16 possible values of this (row, k-block), level x scale rounded to bf16 exactly as
+                  // the stand-alone decode rounds them, held as byte planes in registers: lo[m] / hi[m] are
+                  // the low / high bytes of entries 4m .. 4m + 3.  A weight is then two byte selections
+                  // (no table in shared memory, no multiply per weight).
                   const float sc = csc[gi];
+                  uint32_t lo[4], hi[4];
+#pragma unroll
+                  for (int m = 0; m < 4; ++m) {
+                    const uint32_t t0 = pack_bf16(c_nf4_levels[4 * m] * sc, c_nf4_levels[4 * m + 1] * sc);
+                    const uint32_t t1 = pack_bf16(c_nf4_levels[4 * m + 2] * sc, c_nf4_levels[4 * m + 3] * sc);
+                    lo[m] = __byte_perm(t0, t1, 0x6420);
+                    hi[m] = __byte_perm(t0, t1, 0x7531);
+                  }
 #pragma unroll
                   for (int h = 0; h < 2; ++h) {       // 16 code bytes = 32 weights = 4 output chunks
                     const uint4 q4 = *reinterpret_cast<const uint4*>(rrow + (((2 * gi + h) ^ (et & 7)) << 4));
                     const uint32_t cw[4] = {q4.x, q4.y, q4.z, q4.w};
-                    float w[32];
+                    uint32_t o[16];
 #pragma unroll
-                    for (int i = 0; i < 16; ++i) {    // byte i: element 2i in the high nibble, 2i + 1 in the low one
-                      const float2 pr = nf4_pairs[(cw[i >> 2] >> (8 * (i & 3))) & 0xFFu];
-                      w[2 * i] = pr.x;
-                      w[2 * i + 1] = pr.y;
+                    for (int i = 0; i < 4; ++i) {     // one code word = 8 weights = one output chunk
+                      // byte b of the word: element 2b in the high nibble, 2b + 1 in the low one, so the four
+                      // nibbles of a 16-bit half are elements 1, 0, 3, 2.  Selector a picks entry (code & 7)
+                      // of either half of the table, selector b then takes the half that bit 3 names.
+                      const uint32_t a32 = cw[i] & 0x77777777u;
+                      const uint32_t b32 = ((cw[i] >> 1) & 0x44444444u) | 0x32103210u;
+#pragma unroll
+                      for (int hh = 0; hh < 2; ++hh) {
+                        const uint32_t a = hh ? a32 >> 16 : a32, b = hh ? b32 >> 16 : b32;
+                        const uint32_t l = __byte_perm(__byte_perm(lo[0], lo[1], a), __byte_perm(lo[2], lo[3], a), b);
+                        const uint32_t u = __byte_perm(__byte_perm(hi[0], hi[1], a), __byte_perm(hi[2], hi[3], a), b);
+                        o[4 * i + 2 * hh] = __byte_perm(l, u, 0x4051);        // elements 0 | 1
+                        o[4 * i + 2 * hh + 1] = __byte_perm(l, u, 0x6273);    // elements 2 | 3
+                      }
                     }
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) w[i] *= sc;
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
                       *reinterpret_cast<uint4*>(brow + (((4 * h + c) ^ (et & 7)) << 4)) =
-                          make_uint4(pack_bf16(w[8 * c], w[8 * c + 1]), pack_bf16(w[8 * c + 2], w[8 * c + 3]),
-                                     pack_bf16(w[8 * c + 4], w[8 * c + 5]), pack_bf16(w[8 * c + 6], w[8 * c + 7]));
+                          make_uint4(o[4 * c], o[4 * c + 1], o[4 * c + 2], o[4 * c + 3]);
                   }
                 } else {
 #pragma unroll
