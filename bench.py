@@ -33,6 +33,24 @@ METRIC, UNIT = "perturbed_fwd_tokens_per_s", "tokens/s"
 GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 117662.0}   # (794.43 + 169.43) MB / 8192 rows
 
 
+def hbm_kernel_rates(spec, prof, peaks, steps):
+    """{class: {ms and GB per step, GB/s, frac of the measured copy peak}} for the classes the library books bytes for;
+    the LoRA down-projection is booked in flops 2*rows*J*K and reads rows*K elements."""
+    out = {}
+    es = 2 if spec.bf16 else 4
+    for k in ("attention", "norm", "lora_apply", "rope", "lora_down"):
+        ms, work, cnt = prof.get(k, (0.0, 0.0, 0))
+        if not cnt or ms <= 0 or work <= 0:
+            continue
+        if k == "lora_down":
+            work = work / (2.0 * (spec.n_targets if spec.arch != 0 else 1) * spec.lora_rank) * es
+        gbs = work / (ms * 1e-3) / 1e9
+        out[k] = {"ms_per_step": round(ms / steps, 3), "launches_per_step": cnt // steps,
+                  "GB_per_step": round(work / steps / 1e9, 3), "GB/s": round(gbs, 1),
+                  "frac": round(gbs / peaks["hbm_gbs"], 3) if peaks.get("hbm_gbs") else None}
+    return out
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -522,6 +540,9 @@ def main():
                      "traffic_note": "gate|up launch (the largest GEMM class of the step): ncu capture of that launch at 8192 token rows, scaled by rows"},
         "gemm_tflops_by_class": {k: round(prof[k][1] / (prof[k][0] * 1e-3) / 1e12, 1)
                                  for k in gemm_classes if prof[k][0] > 0},
+        # memory-bound kernels: algorithmic bytes (inputs read once, outputs written once) over their
+        # CUDA-event time in the instrumented pass, against the measured copy bandwidth
+        "hbm_kernels": hbm_kernel_rates(spec, prof, peaks, prof_steps),
         "kernel_time_share": {k: round(v[0] / total_prof, 4) for k, v in prof.items() if v[2]},
         "kernel_ms_per_step": {k: round(v[0] / prof_steps, 3) for k, v in prof.items() if v[2]},
         "loss_mean": float(np.mean(losses)),

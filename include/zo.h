@@ -381,8 +381,10 @@ ZO_API int32_t zo_launch_count(const zo_ctx* ctx);
 
 /* Profiling aid.  While enabled, every kernel launch of zo_step is bracketed by CUDA events
  * on the context's stream.  zo_profile_read synchronises the stream and returns, per kernel
- * class, the summed device time in ms, the summed algorithmic flops 2*M*N*K (GEMM classes
- * only) and the number of launches since the previous read.  Arrays of ZO_PROFILE_CLASSES.
+ * class, the summed device time in ms, the summed algorithmic work and the number of launches
+ * since the previous read.  Work is flops 2*M*N*K for the GEMM classes and LORA_DOWN, and bytes that
+ * must cross HBM (inputs read once, outputs written once) for ATTENTION, NORM, LORA_APPLY and ROPE;
+ * 0 for the rest.  Arrays of ZO_PROFILE_CLASSES.
  * Decoder GEMMs are booked under their own classes (QKV, O, FC1, FC2, HEAD); ZO_PROF_GEMM_TC
  * holds the tensor-core GEMMs of ZO_ARCH_LINEAR. */
 enum { ZO_PROF_GEMM_TC = 0, ZO_PROF_GEMM_SIMT, ZO_PROF_ATTENTION, ZO_PROF_NORM, ZO_PROF_LORA_DOWN,

@@ -1,14 +1,16 @@
 // Shared-input MP-LoRA expansion for the bf16 path (first perturbed layer, Eq. 6 with X^(n) = X):
 //   out[n, t, :] = base[t, :] + s * U[t, :] (B + k_n eps z_{n/2})      for the n replicas of a pass,
 // where base = X W^T (+ bias) and U = X A^T were computed once on the shared rows.  The op writes
-// n*T*k_out outputs from T*k_out inputs: it is bound by the output stream, so everything is arranged
-// for full-line accesses.  One CTA owns a (replica, 128-column tile) pair, generates that pair's
-// operand [s B ; s k eps z] (bf16, rank index along K) once, and sweeps row tiles of 128 tokens.
-// Inside a tile every warp runs a private pipeline on its 16 rows: the base rows arrive through
-// cp.async (double-buffered, one tile ahead), the rank-2r product [U|U] x operand runs on warp-level
-// tensor-core MMAs (m16n8k16, fp32 accumulate), the sum is rounded once to bf16 and leaves through
-// shared memory as 16 bytes per lane on contiguous row segments.  Sections that carry
-// no adapter are copied through the same pipeline.
+// n*T*k_out outputs from T*k_out inputs: it is bound by the output stream.  One CTA owns a (replica,
+// 128-column tile) pair, generates that pair's operand [s B ; s k eps z] (bf16, rank index along K) once
+// and sweeps row tiles of 128 tokens; the rank-2r product [U|U] x operand runs on warp-level tensor-core
+// MMAs (m16n8k16, fp32 accumulate) and the sum is rounded once to bf16.  Replicas are the fastest grid
+// dimension: the CTAs that expand one base tile run together and the tile comes from DRAM once.
+// Sections that carry no adapter are copied through the same pipeline.  Two forms:
+//   * rank <= 16 (lora_expand_tma_kernel): tiles move by bulk tensor copies in both directions, so the
+//     load/store pipe carries one ldmatrix and one stmatrix per 16 x 16 block and nothing else;
+//   * rank 17 .. 64 (lora_expand_kernel): every warp stages its 16 rows with cp.async (double-buffered, one
+//     tile ahead) and writes 16 bytes per lane on contiguous row segments.
 #include "kernels.h"
 #include "lora_operand.cuh"
 #include "mma.cuh"

@@ -387,6 +387,7 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
                       const void* target, int T, uint64_t seed, int q, float eps, float lr) {
   const zo_config& cf = c->cfg;
   const int bf = c->bf, r = cf.lora_rank, ki = cf.d_model, ko = cf.d_out;
+  const double es = bf ? 2.0 : 4.0;            // bytes per activation element (profile bookkeeping)
   const int Tp = (int)up(T, row_pad(cf));
   cudaStream_t st = c->st;
   uint32_t* status = c->at<uint32_t>(c->plan.status);
@@ -417,9 +418,9 @@ zo_status step_linear(zo_ctx* c, const zo_weights* w, const zo_lora* lora, const
   L.scale = cf.lora_scale; L.eps = eps; L.seed = seed; L.tensor_base = 0; L.rows_per_replica = Tp;
   L.rep_base = ps.base; L.rep_stride = ps.stride;
   if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && lora_expand_supported(base, ko, Y, ko, L)) {
-    PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, base, ko, Y, ko, n, T, L, 1, c->n_sms, status));
+    PROF(PC_LORA_APPLY, es * T * ko * (n + 1), launch_lora_expand(st, base, ko, Y, ko, n, T, L, 1, c->n_sms, status));
   } else {
-    PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
+    PROF(PC_LORA_APPLY, es * T * ko * (n + 1), launch_lora_apply(st, bf, base, ko, 1, Y, ko, n, T, L, 1));
   }
   PROF(PC_LOSS, 0.0, launch_mse_rows(st, bf, Y, (const float*)target, n, T, Tp, ko, rowloss_pass));
   PROF(PC_LOSS, 0.0, launch_replica_mean(st, rowloss_pass, nullptr, n, T, ps.base, ps.stride, rowloss, losses, losses_d, status));
@@ -433,6 +434,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
                        float lr, const int32_t* cu = nullptr, int total_tokens = 0) {
   const zo_config& cf = c->cfg;
   const int bf = c->bf, r = cf.lora_rank, d = cf.d_model, f = cf.d_ffn, H = cf.n_heads;
+  const double es = bf ? 2.0 : 4.0;            // bytes per activation element (profile bookkeeping)
   // packed variable-length batch: T = all tokens, S = longest allowed sequence
   const int T = cu ? total_tokens : E * S, Tp = (int)up(T, row_pad(cf));
   const int nt = c->nt, J = nt * r;
@@ -484,7 +486,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
     const int rows = first ? Tp : M;           // layer 0 still works on the shared block
     void* hin = first ? h0 : h;
     void* xn = first ? x0 : x;
-    PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, hin, xn, W.norm1_g, W.norm1_b, rows, d, cf.norm_eps, nullptr, 0, 0));
+    PROF(PC_NORM, 2.0 * es * rows * d, launch_norm(st, bf, nkind, hin, xn, W.norm1_g, W.norm1_b, rows, d, cf.norm_eps, nullptr, 0, 0));
     LoraDesc L{};
     L.U = U; L.ldu = J; L.B = J ? lora->B[l] : nullptr; L.r = r; L.width = d;
     L.B1 = (J && c->pair_mode) ? L.B + (size_t)nt * r * d : nullptr;
@@ -532,9 +534,9 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(G);
       if (tcore && lora_expand_supported(qkv0, 3 * d, qkv, 3 * d, L)) {
         // expansion to the 2q outputs of the pass: bound by the output stream, full-line stores
-        PROF(PC_LORA_APPLY, 0.0, launch_lora_expand(st, qkv0, 3 * d, qkv, 3 * d, n, T, L, 3, c->n_sms, status));
+        PROF(PC_LORA_APPLY, es * T * 3 * d * (n + 1), launch_lora_expand(st, qkv0, 3 * d, qkv, 3 * d, n, T, L, 3, c->n_sms, status));
       } else {
-        PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
+        PROF(PC_LORA_APPLY, es * T * 3 * d * (n + 1), launch_lora_apply(st, bf, qkv0, 3 * d, 1, qkv, 3 * d, n, T, L, 3));
       }
     } else if (J && fused_lora_ok(bf, cf.flags, Tp, d)) {
       G.out = qkv; G.ldo = 3 * d; G.lora = &L;
@@ -547,25 +549,25 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
       GEMM(G);
       if (J) { PROF(PC_LORA_APPLY, 0.0, launch_lora_apply(st, bf, qkv, 3 * d, 0, qkv, 3 * d, n, T, L, 3)); }
     }
-    if (!rope_done) { PROF(PC_ROPE, 0.0, launch_rope(st, bf, qkv, M, Tp, sl, d, H, rope)); }
+    if (!rope_done) { PROF(PC_ROPE, 4.0 * es * M * d, launch_rope(st, bf, qkv, M, Tp, sl, d, H, rope)); }   // q and k, read and written
     if (tcore && !(cf.flags & ZO_FLAG_ATTN_WARP_MMA) && attention_tc_supported(d / H, S)) {
       int ae = 0;
-      PROF(PC_ATTN, 0.0, ae = launch_attention_tc(st, qkv, x, n, sl, Tp, d, H, status, c->n_sms));
+      PROF(PC_ATTN, 4.0 * es * M * d, ae = launch_attention_tc(st, qkv, x, n, sl, Tp, d, H, status, c->n_sms));
       if (ae) {
         snprintf(c->err, sizeof(c->err), "tensor-core attention launch failed (code %d)", ae);
         return ZO_ERR_CUDA;
       }
     } else if (bf && !(cf.flags & ZO_FLAG_SIMT_GEMM) && attention_mma_supported(d / H)) {
-      PROF(PC_ATTN, 0.0, launch_attention_mma(st, qkv, x, n, sl, Tp, d, H));
+      PROF(PC_ATTN, 4.0 * es * M * d, launch_attention_mma(st, qkv, x, n, sl, Tp, d, H));
     } else {
-      PROF(PC_ATTN, 0.0, launch_attention_simt(st, bf, qkv, x, n, sl, Tp, d, H));
+      PROF(PC_ATTN, 4.0 * es * M * d, launch_attention_simt(st, bf, qkv, x, n, sl, Tp, d, H));
     }
     GemmDesc O{};
     O.A = x; O.lda = d; O.M = M; O.N = d; O.K = d; O.out = h; O.ldo = d;
     set_weight(O, W.w_o, W.s_o, d, d);
     O.bias = W.b_o; O.res = hin; O.ldr = d; O.res_mod = first ? Tp : 0; O.prof_class = PC_GEMM_O;
     GEMM(O);
-    PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0));
+    PROF(PC_NORM, 2.0 * es * M * d, launch_norm(st, bf, nkind, h, x, W.norm2_g, W.norm2_b, M, d, cf.norm_eps, nullptr, 0, 0));
     GemmDesc F1{};
     F1.A = x; F1.lda = d; F1.M = M; F1.K = d; F1.bias = W.b_fc1; F1.prof_class = PC_GEMM_FC1;
     set_weight(F1, W.w_fc1, W.s_fc1, opt ? f : 2 * f, d);
@@ -590,7 +592,7 @@ zo_status step_decoder(zo_ctx* c, const zo_weights* w, const zo_lora* lora, cons
   // per-replica loss on the labelled rows only
   const int Mh = n * EP;
   void* xh = c->at<uint8_t>(c->plan.xh);
-  PROF(PC_NORM, 0.0, launch_norm(st, bf, nkind, h, xh, w->final_norm_g, w->final_norm_b, Mh, d, cf.norm_eps, lab_idx, EP, Tp));
+  PROF(PC_NORM, 2.0 * es * Mh * d, launch_norm(st, bf, nkind, h, xh, w->final_norm_g, w->final_norm_b, Mh, d, cf.norm_eps, lab_idx, EP, Tp));
   const void* head = cf.tie_lm_head ? w->tok_emb : w->lm_head;
   if (fused_ce(cf)) {
     // LM head and log-softmax in one pass: the logits stay in tensor memory and registers

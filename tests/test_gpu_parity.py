@@ -243,11 +243,13 @@ def test_mp_lora_linear_bf16_tensor_core(x_replicated, r):
     _mp_lora_linear_case(x_replicated, r, T=256, ki=328, ko=544, q=2)
 
 
-@pytest.mark.parametrize("r", [5, 8, 16, 32, 64])
+@pytest.mark.parametrize("r", [5, 8, 12, 16, 32, 64])
 def test_mp_lora_linear_shared_input_expansion(r):
-    """Shared input with k_out a multiple of 128: the expansion kernel (operand generated once per
-    replica and column tile, warp-level tensor-core product, staged full-line stores) for every rank
-    class, a rank that is not a multiple of 4 or 8, and a ragged last row tile (T = 200)."""
+    """Shared input with k_out a multiple of 128: the expansion kernels (operand generated once per
+    replica and column tile, warp-level tensor-core product) for every rank class: the bulk-tensor
+    form with the duplicated operand half in shared registers (8, 16) and with the element-wise
+    gather (5, 12: not a multiple of 8), the cp.async form (32, 64); a ragged last row tile (T = 200:
+    the last tile has 72 rows, so one warp's box is clipped by the store and one is skipped)."""
     outs = _mp_lora_linear_case(0, r, T=200, ki=328, ko=384, q=3)
     # the CUDA-core expansion computes the same sums in fp32 from unrounded operands: the two agree to bf16 rounding
     assert np.max(np.abs(outs[0] - outs[SIMT])) < 2.0 ** -6 * np.max(np.abs(outs[SIMT]))
