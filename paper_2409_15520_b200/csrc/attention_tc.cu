@@ -320,12 +320,23 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
           if (two) tc_ld32(scol + (j + 2) * 32, w);
           tc_ld_wait();
           const int lim = klim - j * 32;             // elements 0 .. lim of the piece count (>= 31: all of them)
+          // a piece that lies below the diagonal for every row of the warp needs no mask (most pieces do)
+          if (klim_lo - j * 32 >= 31) {
 #pragma unroll
-          for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], i <= lim ? __uint_as_float(v[i]) : -INFINITY);
+            for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(v[i]));
+          } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], i <= lim ? __uint_as_float(v[i]) : -INFINITY);
+          }
           if (two) {
+            if (klim_lo - j * 32 >= 95) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i)
-              m4[i & 3] = fmaxf(m4[i & 3], i + 64 <= lim ? __uint_as_float(w[i]) : -INFINITY);
+              for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(w[i]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                m4[i & 3] = fmaxf(m4[i & 3], i + 64 <= lim ? __uint_as_float(w[i]) : -INFINITY);
+            }
           }
         }
         float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
@@ -348,12 +359,22 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
             tc_ld32(scol + j * 32, v);
             tc_ld_wait();
             const int lim = klim - j * 32;
+            if (klim_lo - j * 32 >= 31) {             // unmasked piece
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float p0 = i <= lim ? ex2f(fmaf(__uint_as_float(v[i]), P.scale_log2e, -ms)) : 0.f;
-              const float p1 = i + 1 <= lim ? ex2f(fmaf(__uint_as_float(v[i + 1]), P.scale_log2e, -ms)) : 0.f;
-              l4[(i >> 1) & 3] += p0 + p1;
-              pk[i >> 1] = pack_bf16(p0, p1);
+              for (int i = 0; i < 32; i += 2) {
+                const float p0 = ex2f(fmaf(__uint_as_float(v[i]), P.scale_log2e, -ms));
+                const float p1 = ex2f(fmaf(__uint_as_float(v[i + 1]), P.scale_log2e, -ms));
+                l4[(i >> 1) & 3] += p0 + p1;
+                pk[i >> 1] = pack_bf16(p0, p1);
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < 32; i += 2) {
+                const float p0 = i <= lim ? ex2f(fmaf(__uint_as_float(v[i]), P.scale_log2e, -ms)) : 0.f;
+                const float p1 = i + 1 <= lim ? ex2f(fmaf(__uint_as_float(v[i + 1]), P.scale_log2e, -ms)) : 0.f;
+                l4[(i >> 1) & 3] += p0 + p1;
+                pk[i >> 1] = pack_bf16(p0, p1);
+              }
             }
           }
 #pragma unroll
