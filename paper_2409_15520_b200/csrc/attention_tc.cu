@@ -347,7 +347,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
         float l4[4] = {0.f, 0.f, 0.f, 0.f};
         for (int c = 0; c < nch && ok; ++c, ++pc) {
           const uint32_t slot = pc & 1u;
-          if (!warp_wait(&ctrl->p_empty[slot], ((pc >> 1) & 1u) ^ 1u)) { ok = false; break; }
           uint8_t* prow = smem + L::P_OFF + slot * BOX + r * 128;
           const int j = 2 * c + half;                // this thread's half of the 64-key chunk
           uint32_t pk[16];                           // P of the piece, bf16 pairs
@@ -377,6 +376,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
               }
             }
           }
+          // the slot is needed only now: the piece's arithmetic ran under the P V product that still read it
+          if (!warp_wait(&ctrl->p_empty[slot], ((pc >> 1) & 1u) ^ 1u)) { ok = false; break; }
 #pragma unroll
           for (int q4 = 0; q4 < 4; ++q4)             // 16-byte chunk half*4 + q4 of the row's 128 bytes: 8 keys per chunk
             *reinterpret_cast<uint4*>(prow + (((half * 4 + q4) ^ (r & 7)) << 4)) =
