@@ -46,7 +46,7 @@ namespace zo {
 namespace tc {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int MAX_STAGES = 6;
+constexpr int MAX_STAGES = 9;                   // narrow-output launches with a 32-row weight box: nine stages of 20 KiB
 constexpr uint32_t A_BYTES = BM * BK * 2;       // 16 KiB
 constexpr uint32_t BOX_BYTES = 128 * BK * 2;    // one 128-row box of the weight tile, 16 KiB
 template <bool PAIR> struct Cfg {
@@ -92,7 +92,9 @@ struct Params {
   int pack_r;
   LoraDesc L;
   uint32_t* status;
-  int n_half;               // 1: at most 128 output columns in all: one weight box per stage, MMAs of N = 128
+  int n_half;               // 1: at most 128 output columns in all: one weight box per stage, MMAs of N = bbox
+  int bbox;                 // rows of that box (32, 64 or 128: the smallest that holds N): a down-projection is a
+                            // stream of activations, and the bytes not spent on weight rows are stages in flight
   int ksplit;               // > 1: the K range of every tile is cut into ksplit units of work
   float4* part;             // ksplit > 1: fp32 partial accumulators, [unit][64 column quads][128 rows]
   // Cross-entropy head: instead of storing the tile, every thread folds the logits of its row into a
@@ -128,9 +130,10 @@ __device__ __forceinline__ void ep_bar() { asm volatile("bar.sync 1, %0;" ::"n"(
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                            ((uint32_t)(BM >> 4) << 24);
 // The pair instruction spans both CTAs: M = 256.
-// The same with N = 128 (launches with at most 128 output columns, e.g. the LoRA down-projection).
-constexpr uint32_t IDESC_N128 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) |
-                                ((uint32_t)(BM >> 4) << 24);
+// The same with N = 32, 64 or 128 (launches with at most 128 output columns, e.g. the LoRA down-projection).
+__device__ __forceinline__ constexpr uint32_t idesc_n(uint32_t n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
 constexpr uint32_t IDESC_PAIR = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) |
                                 ((uint32_t)((2 * BM) >> 4) << 24);
 
@@ -198,8 +201,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const bool narrow = !PAIR && P.n_half;
   // (the kernels that decode quantised weights keep two stages: the other two hold the ring of raw codes)
   const int STAGES = PAIR ? Cfg<PAIR>::STAGES
-                          : (narrow && !WQ ? 6 : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0) - (WQ ? 2 : 0));
-  const uint32_t STAGE_BYTES = narrow && !WQ ? A_BYTES + BOX_BYTES : Cfg<PAIR>::STAGE_BYTES;
+                          : (narrow && !WQ ? (P.bbox == 32 ? 9 : (P.bbox == 64 ? 8 : 6))
+                                           : Cfg<PAIR>::STAGES - (P.slab && P.kslot > 64 ? 1 : 0) - (WQ ? 2 : 0));
+  const uint32_t STAGE_BYTES = narrow && !WQ ? A_BYTES + (uint32_t)P.bbox * 128u : Cfg<PAIR>::STAGE_BYTES;
   constexpr int TILE_M = PAIR ? 2 * BM : BM;           // rows of one scheduled tile
   const int GROUP_M = PAIR ? (P.group_m + 1) / 2 : P.group_m;   // row tiles of a raster group
   extern __shared__ uint8_t smem_raw[];
@@ -309,7 +313,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_expect_tx(bar, A_BYTES);            // the B operand of the stage comes from the decode warps
             tma_load_2d(sa, &tmA, kb * BK, m0, bar);
           } else {
-            mbar_expect_tx(bar, P.n_half ? A_BYTES + BOX_BYTES : Cfg<PAIR>::TX_BYTES);
+            mbar_expect_tx(bar, P.n_half ? A_BYTES + (uint32_t)P.bbox * 128u : Cfg<PAIR>::TX_BYTES);
             tma_load_2d(sa, &tmA, kb * BK, m0, bar);
             tma_load_2d(sa + A_BYTES, &tmB, kb * BK, brow0, bar);
             if (!P.n_half) tma_load_2d(sa + A_BYTES + BOX_BYTES, &tmB, kb * BK, brow1, bar);
@@ -343,7 +347,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (lane == 0 && rank == 0 && SPLIT != 2) {
       uint32_t titer = 0, ltiles = 0;
       RingPos rp;
-      const uint32_t idesc_main = PAIR ? IDESC_PAIR : (P.n_half ? IDESC_N128 : IDESC);
+      const uint32_t idesc_main = PAIR ? IDESC_PAIR : (P.n_half ? idesc_n((uint32_t)P.bbox) : IDESC);
       bool ok = true;
       for (int tile = t_first; tile < t_end && ok; tile += t_step, ++titer) {
         const uint32_t a = titer & 1u, aph = (titer >> 1) & 1u;
@@ -1061,10 +1065,11 @@ int gemm_tc_init() {
 
 // 2-D bf16 tensor map: rows x K (K contiguous), box 128 rows x 64 columns, 128-byte swizzle;
 // out-of-range elements read as zero.
-static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, uint64_t pitch_elems) {
+static int make_map(CUtensorMap* m, const void* ptr, uint64_t K, uint64_t rows, uint64_t pitch_elems,
+                    uint32_t box_rows = 128u) {
   const cuuint64_t dims[2] = {K, rows};
   const cuuint64_t strides[1] = {pitch_elems * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)tc::BK, 128u};
+  const cuuint32_t box[2] = {(cuuint32_t)tc::BK, box_rows};
   const cuuint32_t es[2] = {1u, 1u};
   return (int)g_encode(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides,
                        box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1194,6 +1199,13 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
                                          tiles2 >= 8LL * max_clusters &&
                                          2.0 * (double)G.M * (double)G.N * (double)G.K <= 3.0e12));
   P.n_half = (!pair && !G.swiglu && !P.slab && P.N <= 128) ? 1 : 0;
+  P.bbox = 128;
+  if (P.n_half && !G.wfmt && P.N <= 64) {
+    // a narrow product streams its activations: the smallest weight box leaves the most stages in flight
+    P.bbox = P.N <= 32 ? 32 : 64;
+    e = make_map(&tmB, G.W, (uint64_t)G.K, (uint64_t)G.N, (uint64_t)G.K, (uint32_t)P.bbox);
+    if (e) return 10000 + e;
+  }
   if (pair) {
     // pairs of CTAs (clusters of 2) on 256-row tiles
     const int pairs = (int)(tiles2 < max_clusters ? tiles2 : max_clusters);
