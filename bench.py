@@ -523,6 +523,10 @@ def main():
         "zo_steps_per_s": jobs * args.steps / (ms * 1e-3),
         "step_tflops": algorithmic_flops_per_step(spec) * args.steps / (ms * 1e-3) / 1e12,
         "clocks": clocks,
+        # step time x median SM clock (ms x GHz = millions of SM clocks per step): separates what a change did to
+        # the work per clock from what the power cap did to the clock
+        "mclk_per_step": (round(ms / args.steps * clocks["sm_mhz"] / 1e3, 1)
+                          if clocks.get("sm_mhz") else None),
         "e2e": {"value": whole_job_value(jobs, tokens_per_step, args.steps, ms_e2e), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches,
