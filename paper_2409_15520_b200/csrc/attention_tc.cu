@@ -410,14 +410,18 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
           tc_ld32(lane_base + 384u + j * 64 + 32, v1);
           tc_ld_wait();
           if (qpos < S_len) {
+            // a lane writes its own row, so a store instruction touches 32 rows whatever its width: 32-byte
+            // stores (whole sectors) halve the number of such instructions
 #pragma unroll
-            for (int q4 = 0; q4 < 8; ++q4) {
-              const uint32_t* v = q4 < 4 ? v0 + 8 * q4 : v1 + 8 * (q4 - 4);
-              *reinterpret_cast<uint4*>(orow + j * 64 + q4 * 8) = make_uint4(
-                  pack_bf16(__uint_as_float(v[0]) * inv, __uint_as_float(v[1]) * inv),
-                  pack_bf16(__uint_as_float(v[2]) * inv, __uint_as_float(v[3]) * inv),
-                  pack_bf16(__uint_as_float(v[4]) * inv, __uint_as_float(v[5]) * inv),
-                  pack_bf16(__uint_as_float(v[6]) * inv, __uint_as_float(v[7]) * inv));
+            for (int q8 = 0; q8 < 4; ++q8) {
+              const uint32_t* v = q8 < 2 ? v0 + 16 * q8 : v1 + 16 * (q8 - 2);
+              uint32_t o[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                o[i] = pack_bf16(__uint_as_float(v[2 * i]) * inv, __uint_as_float(v[2 * i + 1]) * inv);
+              asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(orow + j * 64 + q8 * 16),
+                           "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                           : "memory");
             }
           }
         }
@@ -466,6 +470,7 @@ int launch_attention_tc(cudaStream_t st, const void* qkv, void* ctx, int n, SeqL
   const int dh = d / H;
   const int n_jobs = n * sl.E * H;
   if (n_jobs <= 0) return 0;
+  if ((reinterpret_cast<uintptr_t>(ctx) & 31) != 0 || d % 16 != 0) return (int)cudaErrorMisalignedAddress;   // 32-byte output stores
   CUtensorMap tm;
   // rows of the replicated q|k|v buffer x 3d columns; boxes of 128 rows x 64 columns, 128-byte swizzle
   const int me = tc_make_map_bf16(&tm, qkv, (uint64_t)3 * d, (uint64_t)n * Tp, (uint64_t)3 * d);
