@@ -416,6 +416,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int et = threadIdx.x - 64;               // 0..EP_THREADS-1
     const int half = (warp - 2) >> 2;              // which of the quarter's two warps: even or odd chunks
     const bool out_vec_ok = ((uintptr_t)P.out & 15) == 0 && (P.ldo % (P.out_f32 ? 4 : 8)) == 0;
+    // a lane reads and writes its own row, so an access instruction touches 32 rows whatever its width:
+    // 32-byte accesses (whole sectors) halve the number of such instructions of a bf16 tile
+    const bool out_wide_ok = !P.out_f32 && ((uintptr_t)P.out & 31) == 0 && P.ldo % 16 == 0;
+    const bool res_wide_ok = ((uintptr_t)P.res & 31) == 0 && P.ldr % 16 == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
     uint8_t* slab = smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES);
     // Slab mode: build the B operand [s B ; s k eps z] of a tile's LoRA k-block: 256 rows (output
@@ -736,7 +740,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (!P.res) return;
         const bool full_chunk = col0 + 32 <= P.N;
         const bf16* rp = P.res + (size_t)rrow * P.ldr + col0;
-        if (full_chunk && res_vec_ok) {
+        if (full_chunk && res_wide_ok) {
+#pragma unroll
+          for (int j16 = 0; j16 < 2; ++j16) {
+            uint32_t w[8];
+            asm volatile("ld.global.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                         : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7])
+                         : "l"(rp + 16 * j16));
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              f[16 * j16 + 2 * j] += __uint_as_float(w[j] << 16);
+              f[16 * j16 + 2 * j + 1] += __uint_as_float(w[j] & 0xFFFF0000u);
+            }
+          }
+        } else if (full_chunk && res_vec_ok) {
 #pragma unroll
           for (int j8 = 0; j8 < 4; ++j8) {
             float t[8];
@@ -769,7 +786,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         } else {
           bf16* op = (bf16*)P.out + (size_t)row * P.ldo + col0;
-          if (vec_out) {
+          if (full_chunk && out_wide_ok) {
+#pragma unroll
+            for (int j16 = 0; j16 < 2; ++j16) {
+              uint32_t o[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) o[j] = pack_bf16(f[16 * j16 + 2 * j], f[16 * j16 + 2 * j + 1]);
+              asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(op + 16 * j16), "r"(o[0]), "r"(o[1]),
+                           "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                           : "memory");
+            }
+          } else if (vec_out) {
 #pragma unroll
             for (int j8 = 0; j8 < 4; ++j8)
               *reinterpret_cast<uint4*>(op + 8 * j8) =
