@@ -950,16 +950,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           const float* cs = P.rope_tab + (size_t)(P.rope_pos ? P.rope_pos[row % P.rope_tp] : (row % P.rope_tp) % P.rope_s) * dh;   // cos[0..hd) | sin[0..hd)
           if (po > 0) {
             const int h0 = col0 % dh;                  // head-local index of this chunk's first column (< hd)
+            // every lane reads the table row of its own position: 32-byte loads, for the same reason as the stores
 #pragma unroll
-            for (int j4 = 0; j4 < 8; ++j4) {
-              const float4 c4 = *reinterpret_cast<const float4*>(cs + h0 + 4 * j4);
-              const float4 s4 = *reinterpret_cast<const float4*>(cs + hd + h0 + 4 * j4);
-              const float cc[4] = {c4.x, c4.y, c4.z, c4.w}, ss[4] = {s4.x, s4.y, s4.z, s4.w};
+            for (int j8 = 0; j8 < 4; ++j8) {
+              float cc[8], ss[8];
+              asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                           : "=f"(cc[0]), "=f"(cc[1]), "=f"(cc[2]), "=f"(cc[3]), "=f"(cc[4]), "=f"(cc[5]), "=f"(cc[6]), "=f"(cc[7])
+                           : "l"(cs + h0 + 8 * j8));
+              asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                           : "=f"(ss[0]), "=f"(ss[1]), "=f"(ss[2]), "=f"(ss[3]), "=f"(ss[4]), "=f"(ss[5]), "=f"(ss[6]), "=f"(ss[7])
+                           : "l"(cs + hd + h0 + 8 * j8));
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float x1 = f[4 * j4 + j], x2 = f2[4 * j4 + j];
-                f[4 * j4 + j] = x1 * cc[j] - x2 * ss[j];
-                f2[4 * j4 + j] = x2 * cc[j] + x1 * ss[j];
+              for (int j = 0; j < 8; ++j) {
+                const float x1 = f[8 * j8 + j], x2 = f2[8 * j8 + j];
+                f[8 * j8 + j] = x1 * cc[j] - x2 * ss[j];
+                f2[8 * j8 + j] = x2 * cc[j] + x1 * ss[j];
               }
             }
           } else if (dh == 32) {                       // both halves inside this chunk
@@ -1173,6 +1178,7 @@ int launch_gemm_tc(cudaStream_t st, const GemmDesc& G, uint32_t* status, int n_s
   P.pack_out = (bf16*)G.pack_out; P.pack_ld = G.pack_ld; P.pack_r = G.pack_r;
   CUtensorMap tmU = tmA;
   P.group_m = G.group_m > 0 ? G.group_m : 16;
+  if (G.rope_tab && ((uintptr_t)G.rope_tab & 31) != 0) return (int)cudaErrorMisalignedAddress;   // 32-byte table loads
   P.rope_tab = G.rope_tab; P.rope_cols = G.rope_cols; P.rope_dh = G.rope_dh; P.rope_s = G.rope_s; P.rope_tp = G.rope_tp; P.rope_pos = G.rope_pos;
   if (P.slab) {
     e = make_map(&tmU, G.pack_u, (uint64_t)G.pack_ld, (uint64_t)G.M, (uint64_t)G.pack_ld);
