@@ -420,6 +420,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // 32-byte accesses (whole sectors) halve the number of such instructions of a bf16 tile
     const bool out_wide_ok = !P.out_f32 && ((uintptr_t)P.out & 31) == 0 && P.ldo % 16 == 0;
     const bool res_wide_ok = ((uintptr_t)P.res & 31) == 0 && P.ldr % 16 == 0;
+    const bool out_f32_wide_ok = P.out_f32 && ((uintptr_t)P.out & 31) == 0 && P.ldo % 8 == 0;
+    const bool pack_wide_ok = ((uintptr_t)P.pack_out & 31) == 0 && P.pack_ld % 16 == 0 && P.kslot % 16 == 0 &&
+                              P.khalf % 16 == 0 && P.N % 8 == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
     uint8_t* slab = smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES);
     // Slab mode: build the B operand [s B ; s k eps z] of a tile's LoRA k-block: 256 rows (output
@@ -774,7 +777,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const bool vec_out = full_chunk && out_vec_ok;
         if (P.out_f32) {
           float* op = (float*)P.out + (size_t)row * P.ldo + col0;
-          if (vec_out) {
+          if (full_chunk && out_f32_wide_ok) {
+#pragma unroll
+            for (int j8 = 0; j8 < 4; ++j8)
+              asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(op + 8 * j8), "f"(f[8 * j8]),
+                           "f"(f[8 * j8 + 1]), "f"(f[8 * j8 + 2]), "f"(f[8 * j8 + 3]), "f"(f[8 * j8 + 4]), "f"(f[8 * j8 + 5]),
+                           "f"(f[8 * j8 + 6]), "f"(f[8 * j8 + 7])
+                           : "memory");
+          } else if (vec_out) {
 #pragma unroll
             for (int j4 = 0; j4 < 8; ++j4)
               *reinterpret_cast<float4*>(op + 4 * j4) =
@@ -989,14 +999,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           // bf16 copy of U for the tensor-core LoRA k-block: rank index k of slot t goes to
           // K = t*kslot + k and again to K = t*kslot + khalf + k
           bf16* pr = P.pack_out + (size_t)row * P.pack_ld;
+          if (P.pack_r == 16 && pack_wide_ok) {
+            // a slot's 16 values are one 32-byte run, written at K = t*kslot and again at K = t*kslot + khalf
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int col = col0 + j;
-            if (col < P.N) {
-              const int t = col / P.pack_r, k = col - t * P.pack_r;
-              const bf16 hv = __float2bfloat16_rn(f[j]);
-              pr[t * P.kslot + k] = hv;
-              pr[t * P.kslot + P.khalf + k] = hv;
+            for (int u = 0; u < 2; ++u) {
+              if (col0 + 16 * u + 16 <= P.N) {
+                uint32_t o[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) o[j] = pack_bf16(f[16 * u + 2 * j], f[16 * u + 2 * j + 1]);
+                bf16* dst = pr + (col0 / 16 + u) * P.kslot;
+                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(o[0]), "r"(o[1]), "r"(o[2]),
+                             "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                             : "memory");
+                asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst + P.khalf), "r"(o[0]), "r"(o[1]),
+                             "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7])
+                             : "memory");
+              }
+            }
+          } else if (P.pack_r == 8 && pack_wide_ok) {
+            // rank 8: 16-byte runs
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              if (col0 + 8 * u + 8 <= P.N) {
+                const uint4 o = make_uint4(pack_bf16(f[8 * u], f[8 * u + 1]), pack_bf16(f[8 * u + 2], f[8 * u + 3]),
+                                           pack_bf16(f[8 * u + 4], f[8 * u + 5]), pack_bf16(f[8 * u + 6], f[8 * u + 7]));
+                bf16* dst = pr + (col0 / 8 + u) * P.kslot;
+                *reinterpret_cast<uint4*>(dst) = o;
+                *reinterpret_cast<uint4*>(dst + P.khalf) = o;
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int col = col0 + j;
+              if (col < P.N) {
+                const int t = col / P.pack_r, k = col - t * P.pack_r;
+                const bf16 hv = __float2bfloat16_rn(f[j]);
+                pr[t * P.kslot + k] = hv;
+                pr[t * P.kslot + P.khalf + k] = hv;
+              }
             }
           }
         }
