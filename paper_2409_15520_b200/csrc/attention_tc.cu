@@ -6,7 +6,7 @@
 //   * persistent CTAs, one per SM; a job is one (sequence, head).  Warp 0 is the copy engine's
 //     producer (cp.async.bulk.tensor boxes of 128 rows x 64 columns, 128-byte swizzle, no multicast),
 //     warp 1 issues tcgen05.mma, warps 2-9 are two threads per query row (softmax and output), each taking
-//     one half of every 64-key chunk of the row; pieces that the causal mask blanks for a whole warp are skipped,
+//     one half of every 64-key chunk of the row's P (one of the two takes the row maximum, the other writes the output); pieces that the causal mask blanks for a whole warp are skipped,
 //     and the next piece is requested from tensor memory while the current one is worked on.
 //   * a sequence of <= 256 tokens is at most two query tiles and two key tiles, so the scores of a
 //     whole query tile fit in tensor memory (128 + 256 columns for the two tiles): the row maximum is
@@ -311,13 +311,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
         // later ones).  The loops are kept rolled: ten warps in four roles share one instruction cache.
         // (four independent running maxima / sums: a single chain of 32 dependent operations would leave the
         // two warps of a scheduler waiting on arithmetic latency)
+        // The row maximum is taken by the odd-half thread of the row alone, over all pieces: the even-half warps
+        // are still writing the previous tile's output when the scores of this tile arrive, and the odd-half
+        // warps would only wait for them.
         float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-        for (int j = half; j < 2 * nch; j += 4) {    // two pieces per round trip to tensor memory
+        for (int j = 0; half && j < 2 * nch; j += 2) {    // two pieces per round trip to tensor memory
           if (j * 32 > klim_hi) break;
-          const bool two = j + 2 < 2 * nch && (j + 2) * 32 <= klim_hi;
+          const bool two = (j + 1) * 32 <= klim_hi;
           uint32_t v[32], w[32];
           tc_ld32(scol + j * 32, v);
-          if (two) tc_ld32(scol + (j + 2) * 32, w);
+          if (two) tc_ld32(scol + (j + 1) * 32, w);
           tc_ld_wait();
           const int lim = klim - j * 32;             // elements 0 .. lim of the piece count (>= 31: all of them)
           // a piece that lies below the diagonal for every row of the warp needs no mask (most pieces do)
@@ -329,20 +332,20 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tm, const Params P) {
             for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], i <= lim ? __uint_as_float(v[i]) : -INFINITY);
           }
           if (two) {
-            if (klim_lo - j * 32 >= 95) {
+            if (klim_lo - j * 32 >= 63) {
 #pragma unroll
               for (int i = 0; i < 32; ++i) m4[i & 3] = fmaxf(m4[i & 3], __uint_as_float(w[i]));
             } else {
 #pragma unroll
               for (int i = 0; i < 32; ++i)
-                m4[i & 3] = fmaxf(m4[i & 3], i + 64 <= lim ? __uint_as_float(w[i]) : -INFINITY);
+                m4[i & 3] = fmaxf(m4[i & 3], i + 32 <= lim ? __uint_as_float(w[i]) : -INFINITY);
             }
           }
         }
         float m = fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3]));
-        ctrl->xmax[half][r] = m;
+        if (half) ctrl->xmax[1][r] = m;
         if (!pair_sync()) { ok = false; break; }
-        m = fmaxf(m, ctrl->xmax[half ^ 1][r]);       // (key 0 counts for every row: the maximum is finite)
+        if (!half) m = ctrl->xmax[1][r];             // (key 0 counts for every row: the maximum is finite)
         const float ms = m * P.scale_log2e;
         float l4[4] = {0.f, 0.f, 0.f, 0.f};
         for (int c = 0; c < nch && ok; ++c, ++pc) {
