@@ -182,11 +182,14 @@ norm_vec_kernel(const T* __restrict__ x, T* __restrict__ out, const T* __restric
   }
 }
 
-// One warp per row: the row is read once (16-byte accesses, all issued before the first use),
-// kept packed in registers, reduced with shuffles only.  Requires d % VEC == 0, d <= 32*VEC*NV.
-template <typename T, int NV>
+// One warp per row, four rows per block: the row is read once (16-byte accesses, all issued before the
+// first use), kept packed in registers (NV vectors per lane), reduced with shuffles only: no barrier and
+// no shared memory.  Default for bf16 rows of up to 4096 elements (NV = 16: 153 registers, 12 rows of
+// 8 KB in flight per SM).  Against one block per row, CUDA events inside the step: d = 4096 -6 %,
+// d = 2048 -19 %, d = 768 -11 %.  KIND 0 = LayerNorm, 1 = RMSNorm.  Requires d % VEC == 0, d <= 32*VEC*NV.
+template <typename T, int NV, int KIND>
 __global__ void __launch_bounds__(128)
-norm_warp_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
+norm_warp_kernel(const T* __restrict__ x, T* __restrict__ out, const T* __restrict__ g,
                  const T* __restrict__ b, int rows, int d, float eps,
                  const int32_t* __restrict__ lab_idx, int EP, int Tp) {
   constexpr int VEC = 16 / sizeof(T);
@@ -219,12 +222,12 @@ norm_warp_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T
 #pragma unroll
     for (int j = 0; j < VEC; ++j) {
       const float t = to_f(e[j]);
-      s += kind == 0 ? t : t * t;
+      s += KIND == 0 ? t : t * t;
     }
   }
   s = warp_sum(s);
   float mu = 0.f, rstd;
-  if (kind == 0) {
+  if (KIND == 0) {
     mu = s / d;
     float q = 0.f;
 #pragma unroll
@@ -249,14 +252,14 @@ norm_warp_kernel(int kind, const T* __restrict__ x, T* __restrict__ out, const T
       const uint4 graw = *reinterpret_cast<const uint4*>(g + v * VEC);
       const T* ge = reinterpret_cast<const T*>(&graw);
       uint4 braw = make_uint4(0, 0, 0, 0);
-      if (kind == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
+      if (KIND == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
       const T* be = reinterpret_cast<const T*>(&braw);
       const T* e = reinterpret_cast<const T*>(&raw[i]);
       uint4 oraw;
       T* oe = reinterpret_cast<T*>(&oraw);
 #pragma unroll
       for (int j = 0; j < VEC; ++j)
-        oe[j] = from_f<T>((to_f(e[j]) - mu) * rstd * to_f(ge[j]) + ((kind == 0 && b) ? to_f(be[j]) : 0.f));
+        oe[j] = from_f<T>((to_f(e[j]) - mu) * rstd * to_f(ge[j]) + ((KIND == 0 && b) ? to_f(be[j]) : 0.f));
       *reinterpret_cast<uint4*>(o + v * VEC) = oraw;
     }
   }
@@ -269,14 +272,23 @@ static void norm_dispatch(cudaStream_t st, int kind, const void* x, void* out, c
   constexpr int VEC = 16 / sizeof(T);
   const bool aligned = (((uintptr_t)x | (uintptr_t)out | (uintptr_t)g | (uintptr_t)b) & 15) == 0;
   const int nvec = d / VEC;
-  if (aligned && d % VEC == 0 && nvec <= 64) {
-    // short rows: one warp per row, four rows per block
+  if (aligned && d % VEC == 0 && nvec <= (sizeof(T) == 2 ? 512 : 64)) {
+    // one warp per row, four rows per block (bf16: up to 4096 elements; fp32: up to 256)
     const int nv = (nvec + 31) / 32;
     const int grid = (rows + 3) / 4;
-    if (nv <= 1)
-      norm_warp_kernel<T, 1><<<grid, 128, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp);
-    else
-      norm_warp_kernel<T, 2><<<grid, 128, 0, st>>>(kind, (const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp);
+#define ZO_NW(NV)                                                                                              \
+  do {                                                                                                         \
+    if (kind == 0)                                                                                             \
+      norm_warp_kernel<T, NV, 0><<<grid, 128, 0, st>>>((const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp); \
+    else                                                                                                       \
+      norm_warp_kernel<T, NV, 1><<<grid, 128, 0, st>>>((const T*)x, (T*)out, (const T*)g, (const T*)b, rows, d, eps, lab_idx, EP, Tp); \
+  } while (0)
+    if (nv <= 1) ZO_NW(1);
+    else if (nv == 2) ZO_NW(2);
+    else if (nv <= 4) ZO_NW(4);
+    else if (nv <= 8) ZO_NW(8);
+    else ZO_NW(16);
+#undef ZO_NW
     return;
   }
   if (aligned && d % VEC == 0 && nvec <= 256 * 4) {
