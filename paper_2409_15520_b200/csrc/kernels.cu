@@ -182,6 +182,30 @@ norm_vec_kernel(const T* __restrict__ x, T* __restrict__ out, const T* __restric
   }
 }
 
+// Packed fp32 pairs (sm_100: one instruction multiplies two floats) for the bf16 RMSNorm, which is bound
+// by instruction issue: a bf16 pair widens to an fp32 pair with two logic operations.
+__device__ __forceinline__ unsigned long long f2_from_bf2(uint32_t w) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(w << 16), "r"(w & 0xFFFF0000u));
+  return r;
+}
+__device__ __forceinline__ unsigned long long f2_mul(unsigned long long a, unsigned long long b) {
+  unsigned long long r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ unsigned long long f2_fma(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint32_t bf2_from_f2(unsigned long long a) {
+  uint32_t lo, hi, r;
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(a));
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(__uint_as_float(hi)), "f"(__uint_as_float(lo)));
+  return r;
+}
+
 // One warp per row, four rows per block: the row is read once (16-byte accesses, all issued before the
 // first use), kept packed in registers (NV vectors per lane), reduced with shuffles only: no barrier and
 // no shared memory.  Default for bf16 rows of up to 4096 elements (NV = 16: 153 registers, 12 rows of
@@ -214,6 +238,84 @@ norm_warp_kernel(const T* __restrict__ x, T* __restrict__ out, const T* __restri
   for (int i = 0; i < NV; ++i) {
     const int v = lane + 32 * i;
     raw[i] = v < nvec ? *reinterpret_cast<const uint4*>(xr + v * VEC) : make_uint4(0, 0, 0, 0);
+  }
+  if constexpr (sizeof(T) == 2) {
+    // bf16 rows on packed fp32 pairs: per element the same products and roundings as the scalar form below
+    // ((x - mean) * rstd, then * g + b fused); the sums run in two interleaved chains
+    auto hsum = [](unsigned long long a) {
+      float s0, s1;
+      asm("mov.b64 {%0, %1}, %2;" : "=f"(s0), "=f"(s1) : "l"(a));
+      return s0 + s1;
+    };
+    auto dup = [](float a) {
+      unsigned long long r;
+      asm("mov.b64 %0, {%1, %1};" : "=l"(r) : "f"(a));
+      return r;
+    };
+    // every sweep widens the packed row again: carrying the widened copy from one sweep to the next would
+    // cost 8 registers per vector, and the rows in flight per SM with them
+    auto forget = [&]() {
+#pragma unroll
+      for (int i = 0; i < NV; ++i)
+        asm volatile("" : "+r"(raw[i].x), "+r"(raw[i].y), "+r"(raw[i].z), "+r"(raw[i].w));
+    };
+    unsigned long long acc = 0ull;
+    const unsigned long long one2 = dup(1.f);
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const unsigned long long t = f2_from_bf2(w[j]);
+        acc = KIND == 0 ? f2_fma(t, one2, acc) : f2_fma(t, t, acc);       // vectors past the row are zero
+      }
+    }
+    forget();
+    float mu = 0.f, rs;
+    if (KIND == 0) {
+      mu = warp_sum(hsum(acc)) / d;
+      const unsigned long long nmu2 = dup(-mu);
+      unsigned long long q2 = 0ull;
+#pragma unroll
+      for (int i = 0; i < NV; ++i) {
+        if (lane + 32 * i < nvec) {
+          const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const unsigned long long t = f2_fma(f2_from_bf2(w[j]), one2, nmu2);
+            q2 = f2_fma(t, t, q2);
+          }
+        }
+      }
+      forget();
+      rs = rsqrtf(warp_sum(hsum(q2)) / d + eps);
+    } else {
+      rs = rsqrtf(warp_sum(hsum(acc)) / d + eps);
+    }
+    const unsigned long long rs2 = dup(rs), nmu2 = dup(-mu);
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+      const int v = lane + 32 * i;
+      if (v < nvec) {
+        const uint4 graw = *reinterpret_cast<const uint4*>(g + v * VEC);
+        uint4 braw = make_uint4(0, 0, 0, 0);
+        if (KIND == 0 && b) braw = *reinterpret_cast<const uint4*>(b + v * VEC);
+        const uint32_t w[4] = {raw[i].x, raw[i].y, raw[i].z, raw[i].w};
+        const uint32_t gw[4] = {graw.x, graw.y, graw.z, graw.w};
+        const uint32_t bw[4] = {braw.x, braw.y, braw.z, braw.w};
+        uint32_t ow[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          unsigned long long t = f2_from_bf2(w[j]);
+          if (KIND == 0) t = f2_fma(t, one2, nmu2);
+          t = f2_mul(t, rs2);
+          t = KIND == 0 ? f2_fma(t, f2_from_bf2(gw[j]), f2_from_bf2(bw[j])) : f2_mul(t, f2_from_bf2(gw[j]));
+          ow[j] = bf2_from_f2(t);
+        }
+        *reinterpret_cast<uint4*>(o + v * VEC) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+      }
+    }
+    return;
   }
   float s = 0.f;
 #pragma unroll
