@@ -424,6 +424,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool pack_wide_ok = ((uintptr_t)P.pack_out & 31) == 0 && P.pack_ld % 16 == 0 && P.kslot % 16 == 0 &&
                               P.khalf % 16 == 0 && P.N % 8 == 0;
     const bool res_vec_ok = ((uintptr_t)P.res & 15) == 0 && (P.ldr % 8) == 0;
+    const bool bias_vec_ok = ((uintptr_t)P.bias & 15) == 0;   // col0 is a multiple of 32 elements
     uint8_t* slab = smem + (SPLIT == 2 ? 0 : STAGES * STAGE_BYTES);
     // Slab mode: build the B operand [s B ; s k eps z] of a tile's LoRA k-block: 256 rows (output
     // columns) x 64 K-elements, K-major with the 128-byte swizzle.  Rank index k sits at K = k
@@ -912,9 +913,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
           if (P.bias) {
+            if (col0 + 32 <= P.N && bias_vec_ok) {
+              // the chunk's 32 bias values as four 16-byte loads (every lane reads the same addresses)
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (col0 + j < P.N) f[j] += to_f(P.bias[col0 + j]);
+              for (int j8 = 0; j8 < 4; ++j8) {
+                float t[8];
+                unpack8(__ldg(reinterpret_cast<const uint4*>(P.bias + col0 + 8 * j8)), t);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) f[8 * j8 + j] += t[j];
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < P.N) f[j] += to_f(P.bias[col0 + j]);
+            }
           }
           if (P.act == ACT_RELU) {
 #pragma unroll
