@@ -728,6 +728,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(sacc[j]);
       };
       const int rrow = P.res ? (P.res_mod > 0 ? row % P.res_mod : row) : 0;
+      // the rotary table row of this thread's token, once per tile (two divisions by run-time values)
+      const float* rope_row = nullptr;
+      if (P.rope_tab && row_ok)
+        rope_row = P.rope_tab + (size_t)(P.rope_pos ? P.rope_pos[row % P.rope_tp] : (row % P.rope_tp) % P.rope_s) * P.rope_dh;
       // per-tile LoRA constants: all rows of the tile belong to one replica
       const int rep = P.has_lora ? P.L.rep_base + P.L.rep_stride * (m0 / P.L.rows_per_replica) : 0;
       const float* urow = P.has_lora ? P.L.U + (size_t)min(row, P.M - 1) * P.L.ldu : nullptr;
@@ -973,9 +977,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (have2) add_res(col0 + po * 32, f2);
         if (rope_here) {
           const int dh = P.rope_dh, hd = dh >> 1;
-          const float* cs = P.rope_tab + (size_t)(P.rope_pos ? P.rope_pos[row % P.rope_tp] : (row % P.rope_tp) % P.rope_s) * dh;   // cos[0..hd) | sin[0..hd)
+          const float* cs = rope_row;                  // cos[0..hd) | sin[0..hd) of this row's position
           if (po > 0) {
-            const int h0 = col0 % dh;                  // head-local index of this chunk's first column (< hd)
+            const int h0 = col0 & (dh - 1);            // head-local index of this chunk's first column (< hd); dh is 64 or 128 here
             // every lane reads the table row of its own position: 32-byte loads, for the same reason as the stores
 #pragma unroll
             for (int j8 = 0; j8 < 4; ++j8) {
