@@ -30,7 +30,7 @@ METRIC, UNIT = "perturbed_fwd_tokens_per_s", "tokens/s"
 # capture (dram__bytes_read.sum + dram__bytes_write.sum) of that launch at 8192 token rows; activations,
 # outputs and one weight-panel read per raster group all grow with the rows, so a full launch is scaled
 # by rows.  None = the kernel changed since the counters were taken.
-GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 119701.0}   # (809.63 + 170.95) MB / 8192 rows
+GEMM_FC1_DRAM_BYTES_PER_ROW = {"llama7b": 117485.0}   # (791.41 + 171.03) MB / 8192 rows
 
 
 def hbm_kernel_rates(spec, prof, peaks, steps):
